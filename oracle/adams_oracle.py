@@ -1,0 +1,111 @@
+"""ctypes front end of the CPU oracle (TEST INFRASTRUCTURE, not a product path).
+
+Only tests, the smoke check and the benchmark's CPU-baseline / reference legs
+may import this module.  It takes and returns numpy arrays; it never touches a
+GPU and never imports the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes
+from dataclasses import dataclass
+
+import numpy as np
+
+from . import build_oracle
+
+# Flag values of the oracle (see adams_oracle.c).
+F_RESELECT = 1
+F_COUNT_FLIPS = 2
+F_META_BITMASK = 4
+F_V_KEPT_FROM_G = 8
+F_EMIT_DENSE = 16
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build_oracle.build())
+        for name in ("oracle_adams_step_f64", "oracle_adams_step_f32"):
+            fn = getattr(lib, name)
+            fn.restype = ctypes.c_int
+            fn.argtypes = [
+                ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,   # w m v g
+                ctypes.c_void_p, ctypes.c_void_p,                                     # w_fwd meta
+                ctypes.c_void_p, ctypes.c_int,                                        # scale n_seg
+                ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int,           # rows cols N M
+                ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                ctypes.c_int64, ctypes.c_int64,                                       # step total_steps
+                ctypes.c_uint32, ctypes.c_void_p,                                     # flags flip_count
+            ]
+        _lib = lib
+    return _lib
+
+
+@dataclass
+class Hyper:
+    """Hyper-parameters of one step.  Values are rounded to fp32 first, because
+    the CUDA entry points take them as fp32: both sides then see the same numbers."""
+    lr: float = 1e-4
+    beta1: float = 0.9
+    beta2: float = 0.95
+    eps: float = 1e-8
+    l1_coeff: float = 1e-3
+    step: int = 1000
+    total_steps: int = 30000
+
+    def as_f32(self):
+        f = lambda x: float(np.float32(x))
+        return f(self.lr), f(self.beta1), f(self.beta2), f(self.eps), f(self.l1_coeff)
+
+
+def adams_step_inplace(w, m, v, g_bits, w_fwd_bits, meta, scale, rows, cols, N, M, hyper: Hyper,
+                       flags: int, precision: str = "f64") -> int:
+    """Run the oracle in place on C-contiguous numpy arrays.
+
+    w, m, v: float32 [rows*cols]; g_bits, w_fwd_bits: uint16 (raw bf16);
+    meta: uint32 [rows*cols/32]; scale: float32 [rows, n_seg] or None.
+    Returns the number of mask flips counted (0 unless F_COUNT_FLIPS)."""
+    lib = _load()
+    fn = lib.oracle_adams_step_f64 if precision == "f64" else lib.oracle_adams_step_f32
+    for a, dt in ((w, np.float32), (m, np.float32), (v, np.float32), (g_bits, np.uint16),
+                  (w_fwd_bits, np.uint16), (meta, np.uint32)):
+        assert a.dtype == dt and a.flags["C_CONTIGUOUS"], (a.dtype, dt)
+    assert w.size == rows * cols and meta.size == rows * cols // 32
+    n_seg = 1
+    scale_ptr = None
+    if scale is not None:
+        assert scale.dtype == np.float32 and scale.flags["C_CONTIGUOUS"] and scale.shape[0] == rows
+        n_seg = scale.shape[1]
+        scale_ptr = scale.ctypes.data
+    flips = ctypes.c_uint64(0)
+    lr, b1, b2, eps, lam = hyper.as_f32()
+    rc = fn(w.ctypes.data, m.ctypes.data, v.ctypes.data, g_bits.ctypes.data,
+            w_fwd_bits.ctypes.data, meta.ctypes.data, scale_ptr, n_seg,
+            rows, cols, N, M, lr, b1, b2, eps, lam, hyper.step, hyper.total_steps,
+            flags, ctypes.addressof(flips))
+    if rc != 0:
+        raise ValueError(f"oracle rejected its arguments (status {rc})")
+    return int(flips.value)
+
+
+def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELECT,
+               meta_in=None, precision: str = "f64"):
+    """Out-of-place convenience wrapper for 2-D inputs.
+
+    Returns dict(w, m, v, w_fwd (uint16 bf16 bits), meta (uint32 [rows, cols/32]), flips)."""
+    rows, cols = w.shape
+    w2 = np.ascontiguousarray(w, dtype=np.float32).copy().reshape(-1)
+    m2 = np.ascontiguousarray(m, dtype=np.float32).copy().reshape(-1)
+    v2 = np.ascontiguousarray(v, dtype=np.float32).copy().reshape(-1)
+    g2 = np.ascontiguousarray(g_bits, dtype=np.uint16).reshape(-1)
+    fwd = np.zeros(rows * cols, dtype=np.uint16)
+    if meta_in is None:
+        meta = np.zeros(rows * cols // 32, dtype=np.uint32)
+    else:
+        meta = np.ascontiguousarray(meta_in, dtype=np.uint32).copy().reshape(-1)
+    sc = None if scale is None else np.ascontiguousarray(scale, dtype=np.float32)
+    flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision)
+    return dict(w=w2.reshape(rows, cols), m=m2.reshape(rows, cols), v=v2.reshape(rows, cols),
+                w_fwd=fwd.reshape(rows, cols), meta=meta.reshape(rows, cols // 32), flips=flips)

@@ -1,0 +1,434 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests re-types the oracle's loop: each one compares it with a
+brute-force enumeration, a value the paper prints, a closed form that holds at
+special parameter values, or a library routine (torch.optim.Adam, torch's bf16
+conversion).  They run without a GPU.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import adams_oracle as orc
+from oracle.adams_oracle import Hyper
+from helpers import bf16_bits_to_f32, keep_mask_from_meta, torch_bf16_bits
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+NM_CASES = [(1, 2), (1, 4), (2, 4), (3, 4), (4, 4), (4, 8), (2, 8), (1, 8), (5, 16), (8, 16)]
+
+
+def zeros_like_state(rows, cols):
+    z = np.zeros((rows, cols), dtype=np.float32)
+    return z.copy(), z.copy(), np.zeros((rows, cols), dtype=np.uint16)
+
+
+def run(w, m=None, v=None, g=None, scale=None, N=2, M=4, hyper=None, flags=orc.F_RESELECT | orc.F_META_BITMASK,
+        meta_in=None, precision="f64"):
+    rows, cols = w.shape
+    zm, zv, zg = zeros_like_state(rows, cols)
+    m = zm if m is None else m
+    v = zv if v is None else v
+    g = zg if g is None else g
+    hyper = hyper or Hyper()
+    return orc.adams_step(w, m, v, g, scale, N, M, hyper, flags, meta_in, precision)
+
+
+def bf16_exact(x):
+    """fp32 array whose values are exactly representable in bf16, and their bits."""
+    bits = torch_bf16_bits(np.asarray(x, dtype=np.float32))
+    return bf16_bits_to_f32(bits), bits
+
+
+# --------------------------------------------------------------------------- selection (Eq. 3, 4, 6)
+
+def adversarial_groups(rng, n_groups, M):
+    w = rng.normal(0, 0.02, size=(n_groups, M)).astype(np.float32)
+    # exact ties, equal magnitudes of opposite sign, zeros of both signs, all-equal groups
+    w[0::7, 1 % M] = w[0::7, 0]
+    w[1::7, M - 1] = -w[1::7, 0]
+    w[2::7, :] = 0.0
+    w[3::7, 0] = -0.0
+    w[4::7, :] = 0.125
+    w[5::7, M // 2] = 0.0
+    return w
+
+
+@pytest.mark.parametrize("N,M", NM_CASES)
+def test_selection_is_the_brute_force_maximum(N, M):
+    rng = np.random.default_rng(100 * N + M)
+    n_groups = 32 * 12
+    groups = adversarial_groups(rng, n_groups, M)
+    cols = 64 if M <= 16 else 128
+    w = groups.reshape(-1, cols)
+    out = run(w, N=N, M=M, hyper=Hyper(lr=0.0))
+    keep = keep_mask_from_meta(out["meta"], cols, M, bitmask=True).reshape(n_groups, M)
+    a = np.abs(groups.astype(np.float64))
+    combos = [np.array(c) for c in itertools.combinations(range(M), N)]
+    for gi in range(n_groups):
+        assert keep[gi].sum() == N                                        # Eq. 4
+        sums = np.array([a[gi, c].sum() for c in combos])
+        assert a[gi, keep[gi]].sum() == sums.max()                        # Eq. 6: the N largest magnitudes
+        if len(np.unique(a[gi])) == M:                                    # no ties: the mask is unique
+            assert set(np.flatnonzero(keep[gi])) == set(combos[int(sums.argmax())])
+        else:                                                             # ties go to the lower column
+            order = sorted(range(M), key=lambda j: (-a[gi, j], j))
+            assert set(np.flatnonzero(keep[gi])) == set(order[:N])
+
+
+def test_paper_one_two_example():
+    rows = []
+    with open(os.path.join(GOLDEN, "one_two_example.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            lhs, rhs = line.split("->")
+            rows.append(([float(x) for x in lhs.split()], [float(x) for x in rhs.split()]))
+    assert len(rows) == 2
+    for theta, fwd in rows:
+        w = np.tile(np.array(theta, dtype=np.float32), 16)[None, :]          # 32 columns: 16 copies of the pair
+        out = run(w, N=1, M=2, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT | orc.F_META_BITMASK)
+        got = bf16_bits_to_f32(out["w_fwd"])[0, :2]
+        expect = bf16_bits_to_f32(torch_bf16_bits(np.array(fwd, dtype=np.float32)))
+        assert np.array_equal(got, expect)
+        keep = keep_mask_from_meta(out["meta"], 32, 2, True)[0, :2]
+        assert list(keep) == [f != 0 for f in fwd]
+
+
+@pytest.mark.parametrize("N,M", NM_CASES)
+def test_every_group_keeps_exactly_n(N, M):
+    rng = np.random.default_rng(7)
+    w = rng.normal(0, 0.02, size=(5, 96 if M < 32 else 128)).astype(np.float32)
+    cols = w.shape[1]
+    if cols % M:
+        pytest.skip("shape")
+    out = run(w, N=N, M=M)
+    keep = keep_mask_from_meta(out["meta"], cols, M, True)
+    assert np.all(keep.reshape(5, cols // M, M).sum(-1) == N)
+    assert out["meta"].nbytes == w.size // 8                                # one bit per parameter
+    fwd = bf16_bits_to_f32(out["w_fwd"])
+    assert np.all(fwd[~keep] == 0) and np.all(out["w_fwd"][~keep] == 0)      # pruned slots are +0
+
+
+# --------------------------------------------------------------------------- Adam core
+
+def torch_adam_reference(w0, grads, lr, beta1, beta2, eps):
+    p = torch.nn.Parameter(torch.from_numpy(w0.astype(np.float64)))
+    opt = torch.optim.Adam([p], lr=lr, betas=(beta1, beta2), eps=eps, weight_decay=0.0)
+    for g in grads:
+        p.grad = torch.from_numpy(g.astype(np.float64))
+        opt.step()
+    st = opt.state[p]
+    return p.detach().numpy(), st["exp_avg"].numpy(), st["exp_avg_sq"].numpy()
+
+
+@pytest.mark.parametrize("beta1,flags_extra", [(0.0, 0), (0.9, orc.F_V_KEPT_FROM_G)])
+def test_reduces_to_textbook_adam(beta1, flags_extra):
+    """l1_coeff = 0 and full density (N = M): the literal update equals Adam when beta1 = 0
+    (v is fed by the first moment, Eq. 8); with kept entries feeding g^2 it equals Adam for any beta1."""
+    rng = np.random.default_rng(3)
+    rows, cols, steps = 6, 64, 6
+    w0 = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    grads = [bf16_exact(rng.normal(0, 1e-3, size=(rows, cols)))[0] for _ in range(steps)]
+    h = dict(lr=1e-3, beta1=beta1, beta2=0.95, eps=1e-8)
+    hf = {k: float(np.float32(x)) for k, x in h.items()}
+    ref_w, ref_m, ref_v = torch_adam_reference(w0, grads, hf["lr"], hf["beta1"], hf["beta2"], hf["eps"])
+    w, m, v = w0.copy(), np.zeros_like(w0), np.zeros_like(w0)
+    for t, g in enumerate(grads, start=1):
+        out = run(w, m, v, torch_bf16_bits(g), N=4, M=4,
+                  hyper=Hyper(l1_coeff=0.0, step=t, total_steps=1000, **h),
+                  flags=orc.F_RESELECT | orc.F_META_BITMASK | flags_extra)
+        w, m, v = out["w"], out["m"], out["v"]
+    np.testing.assert_allclose(w, ref_w, rtol=2e-6, atol=1e-10)
+    np.testing.assert_allclose(m, ref_m, rtol=2e-6, atol=5e-11)     # fp32 storage of m, cancellation
+    np.testing.assert_allclose(v, ref_v, rtol=2e-6, atol=1e-18)
+
+
+def test_literal_reading_differs_from_adam_when_beta1_nonzero():
+    """Guard on the reading itself: with beta1 = 0.9 the literal second moment (from mu^2) is not Adam's."""
+    rng = np.random.default_rng(4)
+    w0 = rng.normal(0, 0.02, size=(2, 32)).astype(np.float32)
+    g, gb = bf16_exact(rng.normal(0, 1e-3, size=(2, 32)))
+    out = run(w0, g=gb, N=4, M=4, hyper=Hyper(l1_coeff=0.0, step=1, total_steps=10))
+    _, _, ref_v = torch_adam_reference(w0, [g], 1e-4, float(np.float32(0.9)), float(np.float32(0.95)), 1e-8)
+    assert np.all(out["v"] < 0.02 * ref_v + 1e-30)          # (1-beta1)^2 = 0.01 of g^2
+
+
+def test_first_step_closed_form_kept_entry():
+    """t = 1, m0 = v0 = 0, kept entry: dw = -lr g / ((1-beta1)|g| + eps); under the g^2 reading -lr g/(|g| + eps)."""
+    g, gb = bf16_exact(np.array([[3e-3, -2e-3, 5e-4, -7e-5] * 8]))
+    w0 = np.full((1, 32), 0.5, dtype=np.float32)
+    h = Hyper(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, l1_coeff=0.3, step=1, total_steps=50)
+    lr, b1, b2, eps, _ = h.as_f32()
+    out = run(w0, g=gb, N=4, M=4, hyper=h)
+    expect = 0.5 - lr * g.astype(np.float64) / ((1 - b1) * np.abs(g) + eps)
+    np.testing.assert_allclose(out["w"], expect, rtol=1e-7)
+    out2 = run(w0, g=gb, N=4, M=4, hyper=h, flags=orc.F_RESELECT | orc.F_META_BITMASK | orc.F_V_KEPT_FROM_G)
+    expect2 = 0.5 - lr * g.astype(np.float64) / (np.abs(g) + eps)
+    np.testing.assert_allclose(out2["w"], expect2, rtol=1e-7)
+
+
+# --------------------------------------------------------------------------- proportional L1 decay (Eq. 7)
+
+def group_with_known_mask(sign=1.0):
+    """2:4 groups (4, 3, 2, 1) * 0.01 * sign: columns 0, 1 kept, columns 2, 3 masked."""
+    return (np.tile(np.array([4, 3, 2, 1], dtype=np.float32), 8)[None, :] * np.float32(0.01) * np.float32(sign))
+
+
+@pytest.mark.parametrize("sign", [1.0, -1.0])
+def test_decay_closed_form_at_alpha_one(sign):
+    """alpha = 1 (t = T), g = 0, m = 0, v0 = lambda^2, masked entry: mu~ = lambda Sign(w), v stays
+    lambda^2, dw = -lr (lambda/bc1) Sign(w) / (lambda/sqrt(bc2) + eps); kept entries do not move."""
+    w0 = group_with_known_mask(sign)
+    lam = float(np.float32(2e-3))
+    h = Hyper(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, l1_coeff=lam, step=20, total_steps=20)
+    lr, b1, b2, eps, _ = h.as_f32()
+    v0 = np.full_like(w0, np.float32(lam) ** 2)
+    out = run(w0, v=v0, N=2, M=4, hyper=h)
+    bc1, bc2 = 1 - b1 ** 20, 1 - b2 ** 20
+    v_expect = b2 * float(v0[0, 0]) + (1 - b2) * lam * lam
+    step_size = lr * (lam / bc1) / (np.sqrt(v_expect / bc2) + eps)
+    masked = np.tile(np.array([False, False, True, True]), 8)[None, :]
+    expect = w0.astype(np.float64) - np.where(masked, sign * step_size, 0.0)
+    np.testing.assert_allclose(out["w"], expect, rtol=2e-7)
+    np.testing.assert_allclose(out["v"][masked], v_expect, rtol=2e-7)
+    np.testing.assert_allclose(out["v"][~masked], b2 * float(v0[0, 0]), rtol=2e-7)
+    assert np.all(out["m"] == 0)                                   # the stored moment carries no decay
+
+
+def test_decay_mixes_moment_and_sign_with_alpha():
+    """t = 1 of T = 4 (alpha = 1/4), m0 = v0 = 0: mu = (1-b1) g, mu~ = 3/4 mu + 1/4 lambda Sign(w),
+    v^ = mu~^2, so dw = -lr mu~ / ((1-b1)(|mu~| + eps... )) with the bias corrections of t = 1."""
+    w0 = group_with_known_mask(1.0)
+    g, gb = bf16_exact(np.full((1, 32), -6e-3))
+    lam = float(np.float32(1e-3))
+    h = Hyper(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, l1_coeff=lam, step=1, total_steps=4)
+    lr, b1, b2, eps, _ = h.as_f32()
+    out = run(w0, g=gb, N=2, M=4, hyper=h)
+    mu = (1 - b1) * g.astype(np.float64)
+    masked = np.tile(np.array([False, False, True, True]), 8)[None, :]
+    mu_t = np.where(masked, 0.75 * mu + 0.25 * lam * 1.0, mu)
+    expect_w = w0 - lr * (mu_t / (1 - b1)) / (np.abs(mu_t) + eps)
+    np.testing.assert_allclose(out["w"], expect_w, rtol=2e-7)
+    np.testing.assert_allclose(out["m"], mu, rtol=2e-7)            # stored first moment is undecayed
+    np.testing.assert_allclose(out["v"], (1 - b2) * mu_t ** 2, rtol=3e-7)
+
+
+def test_kept_entries_ignore_lambda_and_stored_moment_is_plain_ema():
+    rng = np.random.default_rng(11)
+    w0 = rng.normal(0, 0.02, size=(4, 64)).astype(np.float32)
+    m0 = rng.normal(0, 1e-4, size=(4, 64)).astype(np.float32)
+    v0 = (rng.normal(0, 1e-3, size=(4, 64)) ** 2).astype(np.float32)
+    g, gb = bf16_exact(rng.normal(0, 1e-3, size=(4, 64)))
+    a = run(w0, m0, v0, gb, N=2, M=4, hyper=Hyper(l1_coeff=0.0))
+    b = run(w0, m0, v0, gb, N=2, M=4, hyper=Hyper(l1_coeff=0.5))
+    keep = keep_mask_from_meta(a["meta"], 64, 4, True)
+    assert np.array_equal(a["meta"], b["meta"])
+    for k in ("w", "v", "w_fwd"):
+        assert np.array_equal(a[k][keep], b[k][keep])
+    assert not np.any(a["w"][~keep] == b["w"][~keep])
+    assert np.array_equal(a["m"], b["m"])
+    b1 = float(np.float32(0.9))
+    ema = b1 * m0.astype(np.float64) + (1 - b1) * g.astype(np.float64)
+    np.testing.assert_allclose(a["m"], ema, rtol=1e-6, atol=1e-12)
+
+
+def test_alpha_to_zero_masked_path_meets_kept_path():
+    rng = np.random.default_rng(12)
+    w0 = rng.normal(0, 0.02, size=(4, 64)).astype(np.float32)
+    m0 = rng.normal(0, 1e-4, size=(4, 64)).astype(np.float32)
+    v0 = (rng.normal(0, 1e-3, size=(4, 64)) ** 2).astype(np.float32)
+    _, gb = bf16_exact(rng.normal(0, 1e-3, size=(4, 64)))
+    h = Hyper(l1_coeff=1e-3, step=1, total_steps=10 ** 15)
+    sparse = run(w0, m0, v0, gb, N=2, M=4, hyper=h)
+    dense = run(w0, m0, v0, gb, N=4, M=4, hyper=h)
+    np.testing.assert_allclose(sparse["w"], dense["w"], rtol=2e-7, atol=1e-12)
+    np.testing.assert_allclose(sparse["v"], dense["v"], rtol=2e-7, atol=1e-20)
+
+
+def test_sign_of_zero_is_zero_and_sign_follows_the_weight_immediately():
+    w0 = group_with_known_mask(1.0)
+    w0[0, 2] = 0.0          # masked (smallest magnitudes of its group are columns 2, 3)
+    w0[0, 6] = -0.0
+    rng = np.random.default_rng(13)
+    m0 = rng.normal(0, 1e-4, size=w0.shape).astype(np.float32)
+    v0 = np.full_like(w0, 1e-6)
+    h = Hyper(l1_coeff=0.05, step=10, total_steps=20)
+    with_decay = run(w0, m0, v0, N=2, M=4, hyper=h)
+    # at a zero weight the decay term vanishes: same as lambda = 0
+    no_lambda = run(w0, m0, v0, N=2, M=4, hyper=Hyper(l1_coeff=0.0, step=10, total_steps=20))
+    for c in (2, 6):
+        assert with_decay["w"][0, c] == no_lambda["w"][0, c]
+        assert with_decay["v"][0, c] == no_lambda["v"][0, c]
+    assert with_decay["w"][0, 3] != no_lambda["w"][0, 3]
+    # the decay direction is read from the current weight, not from accumulated momentum:
+    # a masked weight just below zero is pushed up although its neighbour just above zero is pushed down
+    w1 = group_with_known_mask(1.0)
+    w1[0, 2], w1[0, 3] = 1e-5, -1e-5
+    out = run(w1, v=v0, N=2, M=4, hyper=Hyper(lr=1e-6, l1_coeff=0.05, step=20, total_steps=20))
+    assert out["w"][0, 2] < w1[0, 2] and out["w"][0, 3] > w1[0, 3]
+    assert np.isclose(w1[0, 2] - out["w"][0, 2], out["w"][0, 3] - w1[0, 3], rtol=1e-3)
+
+
+# --------------------------------------------------------------------------- weight scaling, emission (Eq. 11, 12)
+
+def edge_floats():
+    rng = np.random.default_rng(21)
+    vals = [0.0, -0.0, 1.0, -1.0, 1.00390625, 1.01171875, 1.005859375, 1.0058593, 1.0058594,   # ties and near ties
+            3.3895314e38, 3.4e38, 1e-38, 1e-40, 9.1835e-41, 4.5e-41, 1e-45, 65504.0, 0.1, -0.3, 255.5, 256.5, 257.5]
+    x = np.array(vals, dtype=np.float32)
+    # every bf16 mid-point pattern: low 16 bits = 0x8000 (tie), 0x7FFF, 0x8001 around random upper halves
+    hi = rng.integers(0x0000, 0x7F00, size=600, dtype=np.uint32) << 16
+    lows = np.array([0x8000, 0x7FFF, 0x8001, 0x0000, 0xFFFF, 0x0001], dtype=np.uint32)
+    bits = (hi[:, None] | lows[None, :]).reshape(-1)
+    sign = (rng.integers(0, 2, size=bits.size, dtype=np.uint32) << 31)
+    y = (bits | sign).astype(np.uint32).view(np.float32)
+    z = rng.normal(0, 1, size=2000).astype(np.float32) * np.float32(10.0) ** rng.integers(-30, 30, size=2000).astype(np.float32)
+    allv = np.concatenate([x, y, z.astype(np.float32)])
+    pad = (-allv.size) % 32
+    return np.concatenate([allv, np.ones(pad, dtype=np.float32)])[None, :]
+
+
+@pytest.mark.parametrize("precision", ["f64", "f32"])
+def test_bf16_rounding_matches_library_conversion(precision):
+    w0 = edge_floats()
+    out = run(w0, N=4, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT | orc.F_META_BITMASK | orc.F_EMIT_DENSE,
+              precision=precision)
+    assert np.array_equal(out["w"].view(np.uint32), w0.view(np.uint32))       # lr = 0 leaves w untouched
+    assert np.array_equal(out["w_fwd"], torch_bf16_bits(w0))
+
+
+def test_unit_scale_emits_masked_bf16_of_updated_weight_and_pow2_scale_is_exact():
+    rng = np.random.default_rng(22)
+    rows, cols = 6, 128
+    w0 = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    m0 = rng.normal(0, 1e-4, size=(rows, cols)).astype(np.float32)
+    v0 = (rng.normal(0, 1e-3, size=(rows, cols)) ** 2).astype(np.float32)
+    _, gb = bf16_exact(rng.normal(0, 1e-3, size=(rows, cols)))
+    none = run(w0, m0, v0, gb, scale=None)
+    ones = run(w0, m0, v0, gb, scale=np.ones((rows, 2), dtype=np.float32))
+    keep = keep_mask_from_meta(none["meta"], cols, 4, True)
+    expect = np.where(keep, torch_bf16_bits(none["w"]), np.uint16(0))
+    assert np.array_equal(none["w_fwd"], expect) and np.array_equal(ones["w_fwd"], expect)
+    for k in (3, -2):
+        sc = np.full((rows, 2), 2.0 ** k, dtype=np.float32)
+        out = run(w0, m0, v0, gb, scale=sc)
+        assert np.array_equal(out["w"], none["w"])                           # the optimizer acts on raw W
+        assert np.array_equal(bf16_bits_to_f32(out["w_fwd"]), bf16_bits_to_f32(expect) * np.float32(2.0 ** k))
+
+
+@pytest.mark.parametrize("n_seg", [1, 2, 4])
+def test_scale_segment_of_a_column(n_seg):
+    """Eq. 12: row r is cut into n contiguous segments of C/n columns; segment s uses A[r, s]."""
+    rows, cols = 3, 128
+    w0 = np.full((rows, cols), 0.5, dtype=np.float32)
+    scale = (2.0 ** (np.arange(rows)[:, None] * 4 + np.arange(n_seg)[None, :])).astype(np.float32)
+    out = run(w0, scale=scale, N=4, M=4, hyper=Hyper(lr=0.0))
+    got = bf16_bits_to_f32(out["w_fwd"])
+    for r in range(rows):
+        for c in range(cols):
+            assert got[r, c] == 0.5 * scale[r, c // (cols // n_seg)]
+
+
+def test_dense_emission_keeps_masked_entries():
+    w0 = group_with_known_mask(1.0)
+    out = run(w0, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT | orc.F_META_BITMASK | orc.F_EMIT_DENSE)
+    assert np.array_equal(out["w_fwd"], torch_bf16_bits(w0))
+
+
+# --------------------------------------------------------------------------- metadata, mask reuse, flips
+
+def test_index_and_bitmask_encodings_describe_the_same_mask():
+    rng = np.random.default_rng(31)
+    w0 = rng.normal(0, 0.02, size=(7, 96)).astype(np.float32)
+    a = run(w0, N=2, M=4, flags=orc.F_RESELECT | orc.F_META_BITMASK, hyper=Hyper(lr=0.0))
+    b = run(w0, N=2, M=4, flags=orc.F_RESELECT, hyper=Hyper(lr=0.0))
+    nonzero = bf16_bits_to_f32(a["w_fwd"]) != 0        # weights are nonzero, so kept <=> emitted nonzero
+    assert np.array_equal(keep_mask_from_meta(a["meta"], 96, 4, True), nonzero)
+    assert np.array_equal(keep_mask_from_meta(b["meta"], 96, 4, False), nonzero)
+    nibbles = (b["meta"][:, :, None] >> (4 * np.arange(8, dtype=np.uint32))[None, None, :]) & 0xF
+    assert np.all((nibbles & 3) < (nibbles >> 2))                          # lower position first
+    assert a["meta"].nbytes == b["meta"].nbytes == w0.size // 8
+
+
+def test_hand_packed_word_layout():
+    """One row of 64 columns, 2:4: keep columns {1,2} in group 0, {0,3} in group 8, {2,3} in group 15."""
+    w0 = np.tile(np.array([4, 3, 2, 1], dtype=np.float32), 16)[None, :].copy()     # default: keep {0,1}
+    w0[0, 0:4] = [1, 4, 3, 2]
+    w0[0, 32:36] = [4, 1, 2, 3]
+    w0[0, 60:64] = [1, 2, 3, 4]
+    bm = run(w0, N=2, M=4, hyper=Hyper(lr=0.0))["meta"]
+    ix = run(w0, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT)["meta"]
+    word0_bm = sum(0b0011 << (4 * k) for k in range(1, 8)) | 0b0110
+    word1_bm = sum(0b0011 << (4 * k) for k in range(1, 7)) | 0b1001 | (0b1100 << 28)
+    idx = lambda lo, hi: lo | (hi << 2)
+    word0_ix = sum(idx(0, 1) << (4 * k) for k in range(1, 8)) | idx(1, 2)
+    word1_ix = sum(idx(0, 1) << (4 * k) for k in range(1, 7)) | idx(0, 3) | (idx(2, 3) << 28)
+    assert [int(x) for x in bm[0]] == [word0_bm, word1_bm]
+    assert [int(x) for x in ix[0]] == [word0_ix, word1_ix]
+
+
+@pytest.mark.parametrize("bitmask", [True, False])
+def test_reused_mask_is_decoded_and_flips_are_counted(bitmask):
+    enc = orc.F_META_BITMASK if bitmask else 0
+    rng = np.random.default_rng(32)
+    w0 = rng.normal(0, 0.02, size=(4, 64)).astype(np.float32)
+    first = run(w0, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT | enc)
+    # same weights again: no flips
+    again = run(w0, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT | orc.F_COUNT_FLIPS | enc, meta_in=first["meta"])
+    assert again["flips"] == 0 and np.array_equal(again["meta"], first["meta"])
+    # a hand-made previous mask: every group keeps {0, 1}
+    field = 0b0011 if bitmask else (0 | 1 << 2)
+    prev = np.full((4, 2), sum(field << (4 * k) for k in range(8)), dtype=np.uint32)
+    keep = keep_mask_from_meta(first["meta"], 64, 4, bitmask)
+    hand = int(np.sum(keep != np.tile(np.array([True, True, False, False]), 16)[None, :]))
+    cnt = run(w0, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT | orc.F_COUNT_FLIPS | enc, meta_in=prev)
+    assert cnt["flips"] == hand and hand > 0
+    # mask reuse (no reselection): the given mask gates decay and emission even though it is not the top-2
+    reuse = run(w0, N=2, M=4, hyper=Hyper(lr=0.0), flags=enc, meta_in=prev)
+    assert np.array_equal(reuse["meta"], prev)
+    assert np.array_equal(bf16_bits_to_f32(reuse["w_fwd"]) != 0, np.tile(np.array([True, True, False, False]), 16)[None, :].repeat(4, 0))
+
+
+# --------------------------------------------------------------------------- numerics and long-run behaviour
+
+def test_fp32_order_stays_within_tolerance_of_fp64():
+    rng = np.random.default_rng(41)
+    rows, cols = 16, 256
+    w0 = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    m0 = rng.normal(0, 1e-4, size=(rows, cols)).astype(np.float32)
+    v0 = (rng.normal(0, 1e-3, size=(rows, cols)) ** 2).astype(np.float32)
+    _, gb = bf16_exact(rng.normal(0, 1e-3, size=(rows, cols)))
+    sc = (1 + 0.1 * rng.random((rows, 2))).astype(np.float32)
+    a = run(w0, m0, v0, gb, scale=sc, precision="f64")
+    b = run(w0, m0, v0, gb, scale=sc, precision="f32")
+    assert np.array_equal(a["meta"], b["meta"])
+    for k in ("w", "m", "v"):
+        err = np.abs(a[k].astype(np.float64) - b[k]) / np.maximum(1e-6 * np.abs(a[k]), 1e-9)
+        assert err.max() < 0.5, (k, err.max())
+    da = bf16_bits_to_f32(a["w_fwd"]).astype(np.float64)
+    db = bf16_bits_to_f32(b["w_fwd"])
+    assert np.all(np.abs(da - db) <= np.abs(da) * 2.0 ** -7)
+
+
+def test_masked_weights_shrink_as_alpha_ramps():
+    """Smoke test of the long-run behaviour the paper describes (App. C: the kept share of the
+    magnitude tends to 1); exact trajectories are not printed anywhere, so nothing is compared."""
+    rng = np.random.default_rng(42)
+    rows, cols, T = 8, 64, 300
+    w = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    m = np.zeros_like(w)
+    v = np.zeros_like(w)
+    meta = None
+    ratios = []
+    for t in range(1, T + 1):
+        _, gb = bf16_exact(rng.normal(0, 1e-4, size=(rows, cols)))
+        flags = orc.F_META_BITMASK | (orc.F_RESELECT if (t == 1 or t % 10 == 0) else 0)
+        out = run(w, m, v, gb, hyper=Hyper(lr=2e-3, l1_coeff=1e-4, step=t, total_steps=T), flags=flags, meta_in=meta)
+        w, m, v, meta = out["w"], out["m"], out["v"], out["meta"]
+        keep = keep_mask_from_meta(meta, cols, 4, True)
+        ratios.append(np.abs(w[keep]).sum() / np.abs(w).sum())
+    assert ratios[-1] > 0.97 and ratios[-1] > ratios[0] + 0.1
