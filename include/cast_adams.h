@@ -1,0 +1,192 @@
+/*
+ * cast_adams.h -- C ABI of the fused AdamS N:M optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * One call performs, for every parameter of a row-major weight matrix W (rows x cols,
+ * cols = input dimension), one iteration of the AdamS optimizer of CAST (arxiv 2509.25996):
+ *
+ *   - N:M magnitude selection per group of M consecutive columns            (Eq. 3, 4, 6)
+ *   - first moment           mu   = beta1 m + (1 - beta1) g                  (Alg. 1 / Eq. 8)
+ *   - proportional L1 decay  mu~  = (1 - a) mu + a lambda Sign(w), a = t/T,
+ *                            on entries outside the kept set, mu~ = mu inside (Eq. 7, Alg. 1)
+ *   - second moment          v    = beta2 v + (1 - beta2) mu~^2               (Eq. 8)
+ *   - bias-corrected update  w    = w - lr (mu~/(1-beta1^t)) / (sqrt(v/(1-beta2^t)) + eps)
+ *   - forward weight         Diag(A~) W~ (Eq. 12), pruned by the mask (Alg. 2, final loop), as bf16
+ *   - mask metadata, one bit per parameter (Remark of Sec. 4.1), optional flip count (App. C)
+ *
+ * Conventions shared by every entry point
+ *   - Returns CAST_OK (0) or a negative status.  Nothing throws, aborts or synchronises the
+ *     device; all argument checks run on the host before any launch.  After CAST_ERR_CUDA,
+ *     cast_last_cuda_error() gives the cudaError_t that was seen on this thread.
+ *   - "device pointer" = memory reachable from the current CUDA device; "host pointer" = ordinary
+ *     host memory.  The caller owns every buffer and keeps it alive until `stream` has passed the
+ *     work.  Buffers of one matrix must not overlap each other.
+ *   - w, m, v are updated IN PLACE.  Non-finite inputs are not checked; results are then
+ *     unspecified (the paper is silent).
+ *   - Shapes: cols % 32 == 0 (a metadata word describes 32 consecutive columns of one row),
+ *     cols % M == 0, M in {2, 4, 8, 16, 32}, 1 <= N <= M, rows*cols < 2^31 per matrix.
+ *     Every device pointer is 16-byte aligned.
+ *   - bf16 values are passed as raw 16-bit patterns (cast_bf16).
+ *
+ * Metadata layout (the paper fixes only its size; the layout is defined here):
+ *   uint32 words, row-major, cols/32 words per row.  Group i of row r owns the M-bit field at
+ *   bit offset (i*M) mod 32 of word r*(cols/32) + (i*M)/32.
+ *     bitmask form (CAST_F_META_BITMASK, any N:M): bit j of the field is set iff column i*M+j is kept.
+ *     index form   (default, 2:4 only):            field = lo | hi << 2 with lo < hi the positions
+ *                                                   (0..3) of the two kept columns.
+ */
+#ifndef CAST_ADAMS_H
+#define CAST_ADAMS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define CAST_API __attribute__((visibility("default")))
+#else
+#define CAST_API
+#endif
+
+typedef uint16_t cast_bf16;      /* raw bfloat16 bits                        */
+typedef void*    cast_stream_t;  /* a cudaStream_t (NULL = the default stream) */
+
+enum cast_status {
+    CAST_OK         =  0,
+    CAST_ERR_NULL   = -1,   /* a required pointer is NULL                                   */
+    CAST_ERR_SHAPE  = -2,   /* rows/cols/segment sizes violate the shape rules              */
+    CAST_ERR_ALIGN  = -3,   /* a device pointer is not 16-byte aligned                      */
+    CAST_ERR_NM     = -4,   /* unsupported N:M, or index-form metadata asked for N:M != 2:4 */
+    CAST_ERR_HYPER  = -5,   /* hyper-parameter out of range (see cast_adams_step)           */
+    CAST_ERR_CUDA   = -6,   /* a CUDA runtime call failed; see cast_last_cuda_error()       */
+    CAST_ERR_PLAN   = -7,   /* invalid plan / context handle, or it is too small            */
+    CAST_ERR_ALIAS  = -8,   /* two buffers of one matrix overlap                            */
+    CAST_ERR_MEMORY = -9    /* a pointer is not of the required kind (device / host)        */
+};
+
+enum cast_flags {
+    CAST_F_RESELECT      = 1u << 0, /* choose the kept set from |w_{t-1}| now (Eq. 6).  Without it the
+                                       kept set is decoded from `meta` (mask reuse between the refreshes
+                                       the paper makes every T1 = 10 iterations, Sec. 4.1)             */
+    CAST_F_COUNT_FLIPS   = 1u << 1, /* add ||mask_t - mask_{t-1}||_0 (numerator of the flip rate r_t,
+                                       App. C) to *flip_count; mask_{t-1} is read from `meta`          */
+    CAST_F_META_BITMASK  = 1u << 2, /* bitmask-form metadata (required unless N:M == 2:4)              */
+    CAST_F_V_KEPT_FROM_G = 1u << 3, /* alternate reading of Eq. 8: kept entries feed g^2 (textbook Adam)
+                                       into v; entries outside the kept set still feed mu~^2           */
+    CAST_F_EMIT_DENSE    = 1u << 4  /* emit Diag(A~) W~ for all entries (the dense training-time forward
+                                       weight of Alg. 2) instead of the pruned product                  */
+};
+
+/*
+ * cast_adams_step -- one AdamS iteration (Alg. 1 loop body, Eq. 6-8; Eq. 12 for the emitted weight)
+ * over one matrix, asynchronous on `stream`.
+ *
+ *   w, m, v      device, fp32 [rows*cols], in/out: master weight, first moment (stored undecayed),
+ *                second moment.
+ *   g            device, bf16 [rows*cols], in: gradient of this iteration.
+ *   w_fwd_bf16   device, bf16 [rows*cols], out: bf16(A[r, c / (cols/scale_groups)] * w_new[r, c]) where
+ *                kept, +0.0 (0x0000) elsewhere (all entries with CAST_F_EMIT_DENSE).  Rounding is to
+ *                nearest even of the fp32 product.
+ *   meta         device, uint32 [rows*cols/32], in/out (layout above).  Read when CAST_F_RESELECT is
+ *                absent or CAST_F_COUNT_FLIPS is set; always written.
+ *   scale        device, fp32 [rows][scale_groups] (the matrix A of Eq. 12, n = scale_groups), or NULL
+ *                for A = 1.  Requires scale_groups >= 1, cols % scale_groups == 0 and
+ *                (cols/scale_groups) % max(M, 8) == 0.
+ *   N, M         keep N of every M consecutive columns; the kept set is chosen on the weights before
+ *                this update, larger magnitude first, lower column first among equal magnitudes.
+ *   lr           finite.  beta1, beta2 in [0, 1).  eps > 0.  l1_coeff (lambda of Eq. 7) finite.
+ *   step         t >= 1;  total_steps  T >= t;  the decay weight is alpha_t = t/T.
+ *   flags        OR of cast_flags.
+ *   flip_count   device, one unsigned 64-bit counter the step ADDS to (the caller zeroes it); may be
+ *                NULL unless CAST_F_COUNT_FLIPS is set.
+ *
+ * Errors: any violated rule above returns its status and launches nothing.
+ */
+CAST_API int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
+                    cast_bf16* w_fwd_bf16, uint32_t* meta,
+                    const float* scale, int scale_groups,
+                    int64_t rows, int64_t cols, int N, int M,
+                    float lr, float beta1, float beta2, float eps, float l1_coeff,
+                    int64_t step, int64_t total_steps,
+                    uint32_t flags, unsigned long long* flip_count,
+                    cast_stream_t stream);
+
+/* One matrix of a multi-tensor plan; fields as the arguments of cast_adams_step. */
+typedef struct cast_tensor {
+    float* w; float* m; float* v;
+    const cast_bf16* g;
+    cast_bf16* w_fwd;
+    uint32_t* meta;
+    const float* scale;      /* may be NULL */
+    int32_t scale_groups;    /* ignored when scale is NULL */
+    int64_t rows, cols;
+} cast_tensor_t;
+
+/* Hyper-parameters of one iteration (Alg. 1 inputs); ranges as in cast_adams_step. */
+typedef struct cast_hyper {
+    float lr, beta1, beta2, eps, l1_coeff;
+    int64_t step, total_steps;
+    uint32_t flags;
+} cast_hyper_t;
+
+/*
+ * Multi-tensor plan: the AdamS iteration of Alg. 1 over "each parameter theta in Theta", i.e. over
+ * every prunable matrix of the model, in ONE kernel launch.
+ *
+ * cast_plan_create  validates `n_tensors` descriptors (host array, copied), uploads a descriptor table
+ *                   to the current device (one allocation, one blocking copy) and returns an opaque
+ *                   handle in *plan_out.  All matrices share N:M.  The buffers named by the descriptors
+ *                   stay owned by the caller and must outlive the plan's use.
+ * cast_plan_step    launches one grid over all matrices on `stream`; arguments as cast_adams_step.
+ *                   The plan may be stepped any number of times, on any stream of its device; two
+ *                   steps of one plan must not overlap in time (they update the same state).
+ * cast_plan_destroy frees the table.  The caller makes sure no step is still running.
+ */
+CAST_API int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out);
+CAST_API int cast_plan_step(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
+                   cast_stream_t stream);
+CAST_API int cast_plan_destroy(void* plan);
+
+/*
+ * Host-resident optimizer state (the same iteration of Alg. 1, with w, m, v, g, w_fwd, meta and scale
+ * in HOST memory): the matrix is cut into blocks of whole rows that are copied to device staging
+ * buffers, updated by the same kernel and copied back, with copies and kernels of consecutive blocks
+ * overlapped on the context's own streams.
+ *
+ * cast_host_ctx_create  allocates the staging buffers for blocks of up to `max_block_params`
+ *                       parameters (a multiple of 32, >= 1024) in `n_slots` (2..8) slots on the current
+ *                       device.  Device memory used: about 28.2 bytes * max_block_params * n_slots.
+ * cast_host_step        arguments as cast_adams_step but every pointer is a HOST pointer (page-locked
+ *                       memory makes the copies asynchronous; pageable memory works and is slower).
+ *                       flip_count is a host counter that is added to.  The call returns when all work
+ *                       is queued; results are valid after cast_host_ctx_sync.  A matrix whose rows are
+ *                       longer than max_block_params is rejected with CAST_ERR_PLAN.
+ * cast_host_ctx_sync    waits for everything queued through the context and folds the flip counts.
+ * cast_host_ctx_destroy waits, then frees streams and buffers.
+ */
+CAST_API int cast_host_ctx_create(int64_t max_block_params, int n_slots, void** ctx_out);
+CAST_API int cast_host_step(void* ctx,
+                   float* w, float* m, float* v, const cast_bf16* g,
+                   cast_bf16* w_fwd_bf16, uint32_t* meta,
+                   const float* scale, int scale_groups,
+                   int64_t rows, int64_t cols, int N, int M,
+                   float lr, float beta1, float beta2, float eps, float l1_coeff,
+                   int64_t step, int64_t total_steps,
+                   uint32_t flags, unsigned long long* flip_count);
+CAST_API int cast_host_ctx_sync(void* ctx);
+CAST_API int cast_host_ctx_destroy(void* ctx);
+
+/* Static description of a status code (never NULL). */
+CAST_API const char* cast_strerror(int status);
+
+/* The cudaError_t behind the last CAST_ERR_CUDA returned on the calling thread (0 if none). */
+CAST_API int cast_last_cuda_error(void);
+
+/* Number of kernels this library has launched in the calling process (for launch accounting). */
+CAST_API unsigned long long cast_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAST_ADAMS_H */

@@ -1,0 +1,211 @@
+"""ctypes binding of libcast_adams.so: the same names as the C ABI, argument marshalling only.
+
+Every function returns the library's integer status (0 = CAST_OK); `check()` turns a
+non-zero status into a CastError.  Pointer arguments accept a torch tensor, a numpy
+array, an integer address or None.  There is no fallback: if the shared library has
+not been built, loading raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libcast_adams.so")
+
+# status codes
+CAST_OK = 0
+CAST_ERR_NULL = -1
+CAST_ERR_SHAPE = -2
+CAST_ERR_ALIGN = -3
+CAST_ERR_NM = -4
+CAST_ERR_HYPER = -5
+CAST_ERR_CUDA = -6
+CAST_ERR_PLAN = -7
+CAST_ERR_ALIAS = -8
+CAST_ERR_MEMORY = -9
+
+# flags
+CAST_F_RESELECT = 1 << 0
+CAST_F_COUNT_FLIPS = 1 << 1
+CAST_F_META_BITMASK = 1 << 2
+CAST_F_V_KEPT_FROM_G = 1 << 3
+CAST_F_EMIT_DENSE = 1 << 4
+
+EXPORTS = (
+    "cast_adams_step", "cast_plan_create", "cast_plan_step", "cast_plan_destroy",
+    "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
+    "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
+)
+
+
+class CastError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"cast_adams status {status}: {message}")
+        self.status = status
+
+
+class cast_tensor_t(ctypes.Structure):
+    _fields_ = [
+        ("w", ctypes.c_void_p), ("m", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("g", ctypes.c_void_p), ("w_fwd", ctypes.c_void_p), ("meta", ctypes.c_void_p),
+        ("scale", ctypes.c_void_p), ("scale_groups", ctypes.c_int32),
+        ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+    ]
+
+
+class cast_hyper_t(ctypes.Structure):
+    _fields_ = [
+        ("lr", ctypes.c_float), ("beta1", ctypes.c_float), ("beta2", ctypes.c_float),
+        ("eps", ctypes.c_float), ("l1_coeff", ctypes.c_float),
+        ("step", ctypes.c_int64), ("total_steps", ctypes.c_int64), ("flags", ctypes.c_uint32),
+    ]
+
+
+_lib = None
+
+_STEP_ARGS = [
+    ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,      # w m v g
+    ctypes.c_void_p, ctypes.c_void_p,                                        # w_fwd meta
+    ctypes.c_void_p, ctypes.c_int,                                           # scale scale_groups
+    ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int,              # rows cols N M
+    ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float,
+    ctypes.c_int64, ctypes.c_int64,                                          # step total_steps
+    ctypes.c_uint32, ctypes.c_void_p,                                        # flags flip_count
+]
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it has not been built (there is no other path)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2509_25996_b200.build_ext` "
+            "(this package has no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    lib.cast_adams_step.restype = ctypes.c_int
+    lib.cast_adams_step.argtypes = _STEP_ARGS + [ctypes.c_void_p]
+    lib.cast_plan_create.restype = ctypes.c_int
+    lib.cast_plan_create.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                     ctypes.POINTER(ctypes.c_void_p)]
+    lib.cast_plan_step.restype = ctypes.c_int
+    lib.cast_plan_step.argtypes = [ctypes.c_void_p, ctypes.POINTER(cast_hyper_t), ctypes.c_void_p, ctypes.c_void_p]
+    lib.cast_plan_destroy.restype = ctypes.c_int
+    lib.cast_plan_destroy.argtypes = [ctypes.c_void_p]
+    lib.cast_host_ctx_create.restype = ctypes.c_int
+    lib.cast_host_ctx_create.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
+    lib.cast_host_step.restype = ctypes.c_int
+    lib.cast_host_step.argtypes = [ctypes.c_void_p] + _STEP_ARGS
+    lib.cast_host_ctx_sync.restype = ctypes.c_int
+    lib.cast_host_ctx_sync.argtypes = [ctypes.c_void_p]
+    lib.cast_host_ctx_destroy.restype = ctypes.c_int
+    lib.cast_host_ctx_destroy.argtypes = [ctypes.c_void_p]
+    lib.cast_strerror.restype = ctypes.c_char_p
+    lib.cast_strerror.argtypes = [ctypes.c_int]
+    lib.cast_last_cuda_error.restype = ctypes.c_int
+    lib.cast_last_cuda_error.argtypes = []
+    lib.cast_kernel_launch_count.restype = ctypes.c_ulonglong
+    lib.cast_kernel_launch_count.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _ptr(x) -> Optional[int]:
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(f"cannot take the address of {type(x)!r}")
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream          # torch.cuda.Stream
+
+
+def cast_strerror(status: int) -> str:
+    return load_library().cast_strerror(int(status)).decode()
+
+
+def cast_last_cuda_error() -> int:
+    return int(load_library().cast_last_cuda_error())
+
+
+def cast_kernel_launch_count() -> int:
+    return int(load_library().cast_kernel_launch_count())
+
+
+def check(status: int) -> None:
+    if status != CAST_OK:
+        msg = cast_strerror(status)
+        if status == CAST_ERR_CUDA:
+            msg += f" (cudaError {cast_last_cuda_error()})"
+        raise CastError(status, msg)
+
+
+def cast_adams_step(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols, N, M,
+                    lr, beta1, beta2, eps, l1_coeff, step, total_steps, flags, flip_count=None, stream=None) -> int:
+    return load_library().cast_adams_step(
+        _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
+        int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
+        int(flags), _ptr(flip_count), _stream(stream))
+
+
+def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols) -> cast_tensor_t:
+    return cast_tensor_t(_ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd), _ptr(meta), _ptr(scale),
+                         int(scale_groups), int(rows), int(cols))
+
+
+def cast_plan_create(tensors: Sequence[cast_tensor_t], N: int, M: int):
+    """Returns (status, plan handle or None)."""
+    n = len(tensors)
+    arr = (cast_tensor_t * max(n, 1))(*tensors)
+    out = ctypes.c_void_p(None)
+    rc = load_library().cast_plan_create(arr if n else None, n, int(N), int(M), ctypes.byref(out))
+    return rc, (out.value if rc == CAST_OK else None)
+
+
+def make_hyper(lr, beta1, beta2, eps, l1_coeff, step, total_steps, flags) -> cast_hyper_t:
+    return cast_hyper_t(lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps), int(flags))
+
+
+def cast_plan_step(plan, hyper: Optional[cast_hyper_t], flip_count=None, stream=None) -> int:
+    h = ctypes.byref(hyper) if hyper is not None else None
+    return load_library().cast_plan_step(plan, h, _ptr(flip_count), _stream(stream))
+
+
+def cast_plan_destroy(plan) -> int:
+    return load_library().cast_plan_destroy(plan)
+
+
+def cast_host_ctx_create(max_block_params: int, n_slots: int):
+    """Returns (status, context handle or None)."""
+    out = ctypes.c_void_p(None)
+    rc = load_library().cast_host_ctx_create(int(max_block_params), int(n_slots), ctypes.byref(out))
+    return rc, (out.value if rc == CAST_OK else None)
+
+
+def cast_host_step(ctx, w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols, N, M,
+                   lr, beta1, beta2, eps, l1_coeff, step, total_steps, flags, flip_count=None) -> int:
+    return load_library().cast_host_step(
+        ctx, _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
+        int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
+        int(flags), _ptr(flip_count))
+
+
+def cast_host_ctx_sync(ctx) -> int:
+    return load_library().cast_host_ctx_sync(ctx)
+
+
+def cast_host_ctx_destroy(ctx) -> int:
+    return load_library().cast_host_ctx_destroy(ctx)

@@ -1,0 +1,266 @@
+// Device code of the fused AdamS N:M step (CAST, arxiv 2509.25996: Alg. 1, Eq. 6-8, Eq. 12).
+//
+// Streaming kernel, HBM-bound: 14 B read and 14.125 B written per parameter.  One thread owns
+// a "unit" of 8 consecutive columns (32 B of each fp32 array, 16 B of each bf16 array, one
+// metadata byte), so every group of M <= 8 columns lives in one thread's registers and the
+// top-N selection is a register-only rank network; groups of 16 or 32 columns are shared by 2
+// or 4 neighbouring lanes through warp shuffles.  A warp covers 256 consecutive parameters:
+// 1 KB of each fp32 array, 512 B of each bf16 array and one 32-byte sector of metadata.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cast {
+
+constexpr int kThreads = 256;          // threads per CTA
+constexpr int kUnitElems = 8;          // parameters per thread per tile
+constexpr int kTileUnits = kThreads;   // units per tile (2048 parameters)
+
+// flag bits (values of the public header)
+constexpr uint32_t kReselect = 1u << 0;
+constexpr uint32_t kCountFlips = 1u << 1;
+constexpr uint32_t kMetaBitmask = 1u << 2;
+constexpr uint32_t kVKeptFromG = 1u << 3;
+constexpr uint32_t kEmitDense = 1u << 4;
+
+// One matrix as the kernel sees it.
+struct TensorDesc {
+    float* w;
+    float* m;
+    float* v;
+    const uint16_t* g;
+    uint16_t* w_fwd;
+    uint32_t* meta;
+    const float* scale;        // A[rows][n] or nullptr
+    uint32_t n_units;          // rows * cols / 8
+    uint32_t seg_magic;        // unit / seg_units == (uint64(unit) * seg_magic) >> seg_shift
+    uint32_t seg_shift;
+    uint32_t pad_;
+};
+
+// Scalars of one iteration, folded on the host in double precision.
+struct StepConsts {
+    float beta1;        // beta1
+    float omb1;         // 1 - beta1
+    float beta2;        // beta2
+    float omb2;         // 1 - beta2
+    float c_mu;         // 1 - alpha_t                  (Eq. 7)
+    float c_sign;       // alpha_t * lambda             (Eq. 7)
+    float inv_bc2;      // 1 / (1 - beta2^t)
+    float lr_bc1;       // lr / (1 - beta1^t)
+    float eps;
+    int32_t n_keep;     // N
+    uint32_t flags;
+};
+
+__device__ __forceinline__ float4 ld_f4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ void st_f4(float* p, float4 x) { *reinterpret_cast<float4*>(p) = x; }
+
+// Keep mask (bit j = column j of the unit is kept) of the groups held by this thread.
+// Order inside a group: larger |w| first, lower column first among equal magnitudes (Eq. 6 with
+// exactly N kept, Eq. 4).  Magnitudes are compared as integers: for non-NaN floats the bit
+// pattern without the sign orders exactly like the absolute value, and -0 equals +0.
+template <int M>
+__device__ __forceinline__ uint32_t select_keep(const float (&w)[8], int n_keep)
+{
+    uint32_t a[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) a[i] = __float_as_uint(w[i]) & 0x7FFFFFFFu;
+
+    constexpr int G = (M <= 8) ? M : 8;      // columns of one group held by this thread
+    int rank[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) rank[i] = 0;
+
+    // pairs inside the thread
+#pragma unroll
+    for (int base = 0; base < 8; base += G) {
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+#pragma unroll
+            for (int k = j + 1; k < G; ++k) {
+                const bool j_first = a[base + j] >= a[base + k];   // equal: the lower column wins
+                rank[base + k] += j_first ? 1 : 0;
+                rank[base + j] += j_first ? 0 : 1;
+            }
+        }
+    }
+    // columns of the same group held by neighbouring lanes (M = 16: 2 lanes, M = 32: 4 lanes)
+    if constexpr (M > 8) {
+        constexpr int L = M / 8;
+        const unsigned lane = threadIdx.x & 31u;
+#pragma unroll
+        for (int d = 1; d < L; ++d) {
+            const bool other_lower = ((lane ^ d) < lane);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                const uint32_t ak = __shfl_xor_sync(0xFFFFFFFFu, a[k], d);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const bool k_first = other_lower ? (ak >= a[j]) : (ak > a[j]);
+                    rank[j] += k_first ? 1 : 0;
+                }
+            }
+        }
+    }
+    uint32_t keep = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) keep |= (rank[i] < n_keep ? 1u : 0u) << i;
+    return keep;
+}
+
+// 2:4 index form <-> keep bits, one nibble per group.  Table entry k (a 4-bit keep mask with two
+// bits set) holds lo | hi << 2; entries of other masks are unused.
+__device__ __forceinline__ uint32_t idx2_from_keep_nibble(uint32_t k)
+{
+    // k: 0011->lo0 hi1 = 0x4, 0101->0,2 = 0x8, 0110->1,2 = 0x9, 1001->0,3 = 0xC, 1010->1,3 = 0xD, 1100->2,3 = 0xE
+    constexpr unsigned long long table =
+        (0x4ull << (4 * 0x3)) | (0x8ull << (4 * 0x5)) | (0x9ull << (4 * 0x6)) |
+        (0xCull << (4 * 0x9)) | (0xDull << (4 * 0xA)) | (0xEull << (4 * 0xC));
+    return (uint32_t)(table >> (4 * k)) & 0xFu;
+}
+__device__ __forceinline__ uint32_t keep_nibble_from_idx2(uint32_t f)
+{
+    return (1u << (f & 3u)) | (1u << ((f >> 2) & 3u));
+}
+__device__ __forceinline__ uint32_t meta_byte_from_keep(uint32_t keep, bool bitmask)
+{
+    if (bitmask) return keep;
+    return idx2_from_keep_nibble(keep & 0xFu) | (idx2_from_keep_nibble(keep >> 4) << 4);
+}
+__device__ __forceinline__ uint32_t keep_from_meta_byte(uint32_t b, bool bitmask)
+{
+    if (bitmask) return b;
+    return keep_nibble_from_idx2(b & 0xFu) | (keep_nibble_from_idx2(b >> 4) << 4);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));   // round to nearest even
+    return r;
+}
+
+// The whole per-unit body: loads, selection, moments, decay, update, emission, metadata.
+// `active` is false for threads past the end of the matrix; they take part in the shuffles only.
+template <int M>
+__device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const StepConsts& c,
+                                                 uint32_t unit, bool active)
+{
+    float w[8], m[8], v[8];
+    uint4 graw = make_uint4(0, 0, 0, 0);
+    uint32_t prev_byte = 0;
+    const size_t e = (size_t)unit * kUnitElems;
+    const bool need_prev = ((c.flags & kReselect) == 0) || (c.flags & kCountFlips);
+
+    if (active) {
+        const float4 w0 = ld_f4(t.w + e), w1 = ld_f4(t.w + e + 4);
+        const float4 m0 = ld_f4(t.m + e), m1 = ld_f4(t.m + e + 4);
+        const float4 v0 = ld_f4(t.v + e), v1 = ld_f4(t.v + e + 4);
+        graw = *reinterpret_cast<const uint4*>(t.g + e);
+        if (need_prev) prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[unit];
+        w[0] = w0.x; w[1] = w0.y; w[2] = w0.z; w[3] = w0.w; w[4] = w1.x; w[5] = w1.y; w[6] = w1.z; w[7] = w1.w;
+        m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+        v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w; v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { w[i] = 0.f; m[i] = 0.f; v[i] = 0.f; }
+    }
+
+    const bool bitmask = (c.flags & kMetaBitmask) != 0;
+    const uint32_t prev_keep = keep_from_meta_byte(prev_byte, bitmask);
+    uint32_t keep;
+    if (c.flags & kReselect) keep = select_keep<M>(w, c.n_keep);     // uniform branch: all lanes shuffle
+    else keep = prev_keep;
+
+    float a = 1.0f;
+    if (active && t.scale != nullptr) {
+        const uint32_t seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
+        a = __ldg(t.scale + seg);
+    }
+
+    const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
+    const bool v_from_g = (c.flags & kVKeptFromG) != 0;
+    const bool dense = (c.flags & kEmitDense) != 0;
+    float fwd[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const float g32 = __uint_as_float((i & 1) ? (gw[i >> 1] & 0xFFFF0000u) : (gw[i >> 1] << 16));
+        const bool kept = (keep >> i) & 1u;
+        // first moment, stored undecayed (Alg. 1)
+        const float mu = fmaf(c.beta1, m[i], c.omb1 * g32);
+        m[i] = mu;
+        // proportional L1 decay outside the kept set (Eq. 7); Sign(0) = 0
+        const float sgn_term = (w[i] == 0.0f) ? 0.0f : copysignf(c.c_sign, w[i]);
+        const float mu_t = kept ? mu : fmaf(c.c_mu, mu, sgn_term);
+        // second moment from the decayed first moment (Eq. 8)
+        const float src = (v_from_g && kept) ? g32 : mu_t;
+        const float vn = fmaf(c.beta2, v[i], (c.omb2 * src) * src);
+        v[i] = vn;
+        // bias-corrected update
+        const float denom = sqrtf(vn * c.inv_bc2) + c.eps;
+        const float wn = w[i] - (c.lr_bc1 * mu_t) / denom;
+        w[i] = wn;
+        // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for
+        fwd[i] = (kept || dense) ? a * wn : 0.0f;
+    }
+
+    if (active) {
+        st_f4(t.w + e, make_float4(w[0], w[1], w[2], w[3]));
+        st_f4(t.w + e + 4, make_float4(w[4], w[5], w[6], w[7]));
+        st_f4(t.m + e, make_float4(m[0], m[1], m[2], m[3]));
+        st_f4(t.m + e + 4, make_float4(m[4], m[5], m[6], m[7]));
+        st_f4(t.v + e, make_float4(v[0], v[1], v[2], v[3]));
+        st_f4(t.v + e + 4, make_float4(v[4], v[5], v[6], v[7]));
+        uint4 f;
+        f.x = pack_bf16x2(fwd[0], fwd[1]);
+        f.y = pack_bf16x2(fwd[2], fwd[3]);
+        f.z = pack_bf16x2(fwd[4], fwd[5]);
+        f.w = pack_bf16x2(fwd[6], fwd[7]);
+        *reinterpret_cast<uint4*>(t.w_fwd + e) = f;
+        reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)meta_byte_from_keep(keep, bitmask);
+    }
+    // flips of this unit (App. C: ||M_t - M_{t-1}||_0)
+    return active ? (uint32_t)__popc(keep ^ prev_keep) : 0u;
+}
+
+// Persistent grid: CTA b handles tiles b, b + gridDim.x, ...  For the multi-tensor form the tile
+// index space is the concatenation of all matrices' tiles (each matrix padded to whole tiles);
+// tile_start[k] is the first tile of matrix k and tile_start[n_tensors] the total.  Because a CTA's
+// tile index only grows, the matrix index is found by walking forward, never by searching.
+template <int M, bool MULTI>
+__global__ void __launch_bounds__(kThreads)
+adams_nm_kernel(const __grid_constant__ TensorDesc single,
+                const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ tile_start,
+                uint32_t total_tiles, const __grid_constant__ StepConsts c,
+                unsigned long long* __restrict__ flip_count)
+{
+    uint32_t flips = 0;
+    uint32_t k = 0;
+    for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        if constexpr (MULTI) {
+            while (tile >= __ldg(tile_start + k + 1)) ++k;
+            const TensorDesc t = descs[k];
+            const uint32_t unit = (tile - __ldg(tile_start + k)) * kTileUnits + threadIdx.x;
+            flips += process_unit<M>(t, c, unit, unit < t.n_units);
+        } else {
+            const uint32_t unit = tile * kTileUnits + threadIdx.x;
+            flips += process_unit<M>(single, c, unit, unit < single.n_units);
+        }
+    }
+    if (c.flags & kCountFlips) {
+        flips = __reduce_add_sync(0xFFFFFFFFu, flips);
+        __shared__ uint32_t warp_sums[kThreads / 32];
+        if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = flips;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long total = 0;
+#pragma unroll
+            for (int i = 0; i < kThreads / 32; ++i) total += warp_sums[i];
+            if (total) atomicAdd(flip_count, total);
+        }
+    }
+}
+
+}  // namespace cast

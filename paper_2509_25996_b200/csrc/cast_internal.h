@@ -1,0 +1,50 @@
+// Host-side helpers shared by the entry points of the library (not part of the public ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/cast_adams.h"
+#include "adams_kernel.cuh"
+
+namespace cast {
+
+// Remember a failed CUDA call for cast_last_cuda_error() and return CAST_ERR_CUDA.
+int cuda_failed(cudaError_t e);
+
+#define CAST_CUDA_TRY(expr)                                  \
+    do {                                                     \
+        cudaError_t cast_e_ = (expr);                        \
+        if (cast_e_ != cudaSuccess) return ::cast::cuda_failed(cast_e_); \
+    } while (0)
+
+// N:M, flags and the flip counter pointer.
+int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count);
+
+// Hyper-parameter ranges; on success fills the folded per-iteration scalars.
+int make_step_consts(float lr, float beta1, float beta2, float eps, float l1_coeff,
+                     int64_t step, int64_t total_steps, int N, uint32_t flags, StepConsts* out);
+
+// Shape rules of one matrix (does not look at pointers).
+int check_shape(int64_t rows, int64_t cols, int M, bool has_scale, int scale_groups);
+
+// Null / alignment / overlap rules of one matrix's pointers (addresses only, never dereferenced).
+int check_pointers(const void* w, const void* m, const void* v, const void* g, const void* w_fwd,
+                   const void* meta, const void* scale, int scale_groups, int64_t rows, int64_t cols);
+
+// Every given pointer must be device-accessible memory on the current device.
+int check_device_memory(const void* const* ptrs, int n);
+
+// Kernel-side description of one (already validated) matrix.
+TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
+                     const float* scale, int scale_groups, int64_t rows, int64_t cols);
+
+inline uint32_t tiles_of(const TensorDesc& d) { return (d.n_units + kTileUnits - 1) / kTileUnits; }
+
+// Launch over one matrix (descriptor passed by value) or over a device table of matrices.
+int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count,
+                  cudaStream_t stream);
+int launch_multi(const TensorDesc* d_descs, const uint32_t* d_tile_start, uint32_t total_tiles, int M,
+                 const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
+
+}  // namespace cast

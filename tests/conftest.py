@@ -15,7 +15,7 @@ def pytest_configure(config):
 
 @pytest.fixture(scope="session", autouse=True)
 def _built():
-    """Compile the C oracle once per session."""
-    from oracle import build_oracle
-    build_oracle.build()
+    """Compile the CUDA library (nvcc cross-compiles without a GPU) and the C oracle once per session."""
+    import __graft_entry__
+    __graft_entry__.build()
     yield

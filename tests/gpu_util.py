@@ -1,0 +1,147 @@
+"""Helpers of the GPU parity tests: guarded device buffers, one CUDA call through the C-ABI, one
+oracle call on host copies of the same tensors, and the comparison with the stated tolerances."""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+import torch
+
+import paper_2509_25996_b200 as cast
+from paper_2509_25996_b200 import binding as B
+from paper_2509_25996_b200 import workloads
+from oracle import adams_oracle as orc
+from helpers import bf16_ulp_distance, within_tol
+
+GUARD_BYTES = 256
+
+
+class Guarded:
+    """A device buffer with canary bands on both sides (catches out-of-bounds writes of a kernel)."""
+
+    def __init__(self, n: int, dtype: torch.dtype, device, fill=None):
+        item = torch.empty((), dtype=dtype).element_size()
+        self.pad = GUARD_BYTES // item
+        self.raw = torch.empty(n + 2 * self.pad, dtype=dtype, device=device)
+        self.canary = {torch.float32: 1234.5, torch.bfloat16: -3.0, torch.int32: 0x5A5A5A5A}[dtype]
+        self.raw.fill_(self.canary)
+        self.view = self.raw[self.pad:self.pad + n]
+        if fill is not None:
+            self.view.copy_(fill.reshape(-1))
+
+    def intact(self) -> bool:
+        lo, hi = self.raw[:self.pad], self.raw[self.raw.numel() - self.pad:]
+        return bool((lo == self.canary).all().item() and (hi == self.canary).all().item())
+
+
+@dataclass
+class DeviceState:
+    rows: int
+    cols: int
+    w: Guarded
+    m: Guarded
+    v: Guarded
+    g: Guarded
+    w_fwd: Guarded
+    meta: Guarded
+    scale: Optional[torch.Tensor]
+
+    def all_intact(self) -> bool:
+        return all(b.intact() for b in (self.w, self.m, self.v, self.g, self.w_fwd, self.meta))
+
+
+def to_device(inp: workloads.TensorInputs, device, meta_in: Optional[np.ndarray] = None) -> DeviceState:
+    rows, cols = inp.w.shape
+    n = rows * cols
+    meta = Guarded(n // 32, torch.int32, device)
+    if meta_in is not None:
+        meta.view.copy_(torch.from_numpy(np.ascontiguousarray(meta_in).view(np.int32).reshape(-1)))
+    else:
+        meta.view.zero_()
+    fwd = Guarded(n, torch.bfloat16, device)
+    return DeviceState(rows, cols,
+                       Guarded(n, torch.float32, device, inp.w.to(device)),
+                       Guarded(n, torch.float32, device, inp.m.to(device)),
+                       Guarded(n, torch.float32, device, inp.v.to(device)),
+                       Guarded(n, torch.bfloat16, device, inp.g.to(device)),
+                       fwd, meta,
+                       None if inp.scale is None else inp.scale.to(device).contiguous())
+
+
+def host_arrays(inp: workloads.TensorInputs):
+    return (inp.w.cpu().numpy(), inp.m.cpu().numpy(), inp.v.cpu().numpy(), workloads.bf16_bits(inp.g),
+            None if inp.scale is None else inp.scale.cpu().numpy())
+
+
+def oracle_flags(flags: int) -> int:
+    """The two flag sets use the same numbering; translated name by name so a renumbering would show."""
+    out = 0
+    for lib_bit, orc_bit in ((B.CAST_F_RESELECT, orc.F_RESELECT), (B.CAST_F_COUNT_FLIPS, orc.F_COUNT_FLIPS),
+                             (B.CAST_F_META_BITMASK, orc.F_META_BITMASK), (B.CAST_F_V_KEPT_FROM_G, orc.F_V_KEPT_FROM_G),
+                             (B.CAST_F_EMIT_DENSE, orc.F_EMIT_DENSE)):
+        if flags & lib_bit:
+            out |= orc_bit
+    return out
+
+
+def run_oracle(inp: workloads.TensorInputs, N, M, hyper: orc.Hyper, flags, meta_in=None, precision="f64"):
+    w, m, v, g, sc = host_arrays(inp)
+    return orc.adams_step(w, m, v, g, sc, N, M, hyper, oracle_flags(flags), meta_in, precision)
+
+
+def device_outputs(st: DeviceState, flips=None):
+    rows, cols = st.rows, st.cols
+    out = dict(
+        w=st.w.view.cpu().numpy().reshape(rows, cols),
+        m=st.m.view.cpu().numpy().reshape(rows, cols),
+        v=st.v.view.cpu().numpy().reshape(rows, cols),
+        w_fwd=workloads.bf16_bits(st.w_fwd.view).reshape(rows, cols),
+        meta=st.meta.view.cpu().numpy().view(np.uint32).reshape(rows, cols // 32),
+    )
+    if flips is not None:
+        out["flips"] = int(flips.item())
+    return out
+
+
+def run_cuda_single(inp: workloads.TensorInputs, N, M, hyper: orc.Hyper, flags, meta_in=None, device="cuda:0"):
+    st = to_device(inp, device, meta_in)
+    flips = torch.zeros(1, dtype=torch.int64, device=device) if flags & B.CAST_F_COUNT_FLIPS else None
+    lr, b1, b2, eps, lam = hyper.as_f32()
+    n_seg = 1 if st.scale is None else st.scale.shape[1]
+    cast.check(cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view,
+                                    st.scale, n_seg, st.rows, st.cols, N, M, lr, b1, b2, eps, lam,
+                                    hyper.step, hyper.total_steps, flags, flips, torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    assert st.all_intact(), "a kernel wrote outside its buffers"
+    return device_outputs(st, flips)
+
+
+def near_tie_groups(w: np.ndarray, N: int, M: int, rel: float = 1e-6) -> int:
+    """Groups whose N-th and (N+1)-th largest magnitudes differ by less than `rel` relative."""
+    if N >= M:
+        return 0
+    a = np.sort(np.abs(w.reshape(-1, M).astype(np.float64)), axis=1)[:, ::-1]
+    hi, lo = a[:, N - 1], a[:, N]
+    return int(np.sum((hi - lo) < rel * np.maximum(hi, 1e-300)))
+
+
+def assert_parity(got: dict, ref: dict, label: str = ""):
+    """fp32 state within max(1e-6 relative, 1e-9 absolute); forward weight within 1 bf16 ulp with the same
+    zero pattern; metadata bit-exact."""
+    for k in ("w", "m", "v"):
+        ok, worst = within_tol(got[k], ref[k], rel=1e-6, floor=1e-9)
+        assert ok, f"{label} {k}: worst error is {worst:.3g} x the tolerance"
+    assert np.array_equal(got["meta"], ref["meta"]), f"{label} metadata differs"
+    d = bf16_ulp_distance(got["w_fwd"], ref["w_fwd"])
+    assert d.max(initial=0) <= 1, f"{label} forward weight differs by {d.max()} ulp"
+    assert np.array_equal(got["w_fwd"] == 0, ref["w_fwd"] == 0) or np.all(
+        (got["w_fwd"] & 0x7FFF)[(got["w_fwd"] == 0) != (ref["w_fwd"] == 0)] <= 1), f"{label} zero pattern differs"
+    if "flips" in got:
+        assert got["flips"] == ref["flips"], f"{label} flips {got['flips']} != {ref['flips']}"
+
+
+def v_pure_relative_error(got: dict, ref: dict) -> float:
+    r = ref["v"].astype(np.float64)
+    nz = r != 0
+    return float(np.max(np.abs(got["v"].astype(np.float64)[nz] - r[nz]) / np.abs(r[nz]))) if nz.any() else 0.0

@@ -1,0 +1,77 @@
+"""Full-size workloads in the launch configuration the benchmark times, checked on sampled row blocks
+(the oracle recomputes each sampled block from host copies taken before the step) and on properties
+that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_25996_b200 as cast
+from paper_2509_25996_b200 import binding as B
+from paper_2509_25996_b200 import workloads
+from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
+from oracle import adams_oracle as orc
+import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def sample_blocks(shapes, n_random, rows_per_block, seed):
+    rng = np.random.default_rng(seed)
+    picks = [(0, 0), (len(shapes) - 1, shapes[-1][0] - rows_per_block)]      # very first and very last rows
+    for _ in range(n_random):
+        t = int(rng.integers(0, len(shapes)))
+        picks.append((t, int(rng.integers(0, shapes[t][0] - rows_per_block + 1))))
+    return picks
+
+
+def check_sampled(wl_name, N, M, flags, n_random=14, rows_per_block=6, need_gb=0.0):
+    free, _ = torch.cuda.mem_get_info()
+    if free < need_gb * 1e9:
+        pytest.skip(f"needs {need_gb} GB of device memory, {free / 1e9:.0f} GB free")
+    wl = workloads.workload(wl_name)
+    state = DeviceModelState(wl.shapes, N, M, seed=0, device=DEV, scale_mode="jitter")
+    picks = sample_blocks(wl.shapes, n_random, rows_per_block, seed=1)
+    before = []
+    for t, r0 in picks:
+        s = state.mats[t]
+        sl = slice(r0, r0 + rows_per_block)
+        before.append(workloads.TensorInputs(s.w[sl].cpu(), s.g[sl].cpu(), s.m[sl].cpu(), s.v[sl].cpu(), s.scale[sl].cpu()))
+    h = RunHyper(total_steps=wl.total_steps)
+    launches = cast.cast_kernel_launch_count()
+    state.step(h, flags)
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == launches + 1
+    oh = orc.Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
+    for (t, r0), inp in zip(picks, before):
+        s = state.mats[t]
+        sl = slice(r0, r0 + rows_per_block)
+        got = dict(w=s.w[sl].cpu().numpy(), m=s.m[sl].cpu().numpy(), v=s.v[sl].cpu().numpy(),
+                   w_fwd=workloads.bf16_bits(s.w_fwd[sl]), meta=s.meta[sl].cpu().numpy().view(np.uint32))
+        U.assert_parity(got, U.run_oracle(inp, N, M, oh, flags), f"{wl_name} tensor {t} rows {r0}+")
+    # properties at full size: every group keeps exactly N (Eq. 4), pruned slots are +0, one bit per parameter
+    bitmask = bool(flags & B.CAST_F_META_BITMASK)
+    for t in (0, len(wl.shapes) // 2, len(wl.shapes) - 1):
+        s = state.mats[t]
+        nz = (s.w_fwd.view(torch.int16) != 0).view(s.rows, s.cols // M, M).sum(-1)
+        assert int(nz.max().item()) <= N and float((nz == N).float().mean().item()) > 0.999
+        assert s.meta.numel() * 4 == s.rows * s.cols // 8
+        if bitmask:
+            pop = sum(((s.meta >> b) & 1).sum(dtype=torch.int64) for b in range(32))
+            assert int(pop.item()) == s.rows * s.cols * N // M
+    state.close()
+
+
+def test_llama2_7b_full_set_sampled():
+    """LLaMA2-7B linear set (224 matrices, 6,476,005,376 parameters, 104 GB resident), one launch."""
+    check_sampled("llama2_7b", 2, 4, B.CAST_F_RESELECT, need_gb=125)
+
+
+@pytest.mark.parametrize("N,M", [(4, 8), (1, 4)])
+def test_llama2_7b_layer_general_nm_sampled(N, M):
+    check_sampled("llama2_7b_layer", N, M, B.CAST_F_RESELECT | B.CAST_F_META_BITMASK, n_random=8, need_gb=5)
+
+
+def test_llama2_13b_layer_sampled():
+    check_sampled("llama2_13b_layer", 2, 4, B.CAST_F_RESELECT, n_random=8, need_gb=8)

@@ -1,0 +1,182 @@
+"""CUDA path vs the CPU oracle, element by element, on identical seeded inputs (all through the C-ABI).
+
+Tolerances (written here, derived from the arithmetic: every fp32 result is a short chain of
+correctly rounded or 1-2 ulp operations, ~1e-7 relative, and sums that can cancel are bounded
+absolutely by an ulp of their ~1e-4-sized operands, ~1e-11):
+    w, m, v      |cuda - oracle| <= max(1e-6 |oracle|, 1e-9)
+    w_fwd        within 1 bf16 ulp, same zero pattern
+    mask, meta   bit-exact (selection compares the bit-identical pre-update weights on both sides);
+                 groups whose N-th and (N+1)-th magnitudes are within 1e-6 relative are counted
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_25996_b200 as cast
+from paper_2509_25996_b200 import binding as B
+from paper_2509_25996_b200 import workloads
+from oracle.adams_oracle import Hyper
+from helpers import keep_mask_from_meta
+import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+RS, BM = B.CAST_F_RESELECT, B.CAST_F_META_BITMASK
+NM_ALL = [(2, 4), (1, 2), (2, 2), (1, 4), (3, 4), (4, 4), (4, 8), (1, 8), (8, 8), (5, 16), (16, 16), (8, 32), (1, 32), (31, 32)]
+
+
+def inputs(rows, cols, seed=0, idx=0, scale_mode="jitter"):
+    return workloads.gen_tensor_inputs(rows, cols, seed=seed, tensor_index=idx, device="cpu", scale_mode=scale_mode)
+
+
+@pytest.mark.parametrize("N,M", NM_ALL)
+@pytest.mark.parametrize("rows,cols", [(1, 32), (3, 64), (5, 96), (7, 2080)])
+def test_small_shapes_every_nm(N, M, rows, cols):
+    """1 x 32 up to 7 x 2080 (7.1 tiles of 2048 parameters: several tiles and a ragged tail)."""
+    inp = inputs(rows, cols, seed=1, idx=N * 100 + M)
+    if inp.scale is not None and (cols // 2) % max(M, 8) != 0:
+        inp.scale = None
+    flags = RS | (0 if (N, M) == (2, 4) else BM)
+    h = Hyper()
+    got = U.run_cuda_single(inp, N, M, h, flags)
+    for prec in ("f64", "f32"):
+        U.assert_parity(got, U.run_oracle(inp, N, M, h, flags, precision=prec), f"{N}:{M} {rows}x{cols} {prec}")
+    keep = keep_mask_from_meta(got["meta"], cols, M, bitmask=(flags & BM) != 0)
+    assert np.all(keep.reshape(rows, cols // M, M).sum(-1) == N)               # Eq. 4 on the CUDA result
+
+
+def adversarial(rows, cols, M):
+    """Exact ties, +-0, denormals, all-equal groups, huge and tiny magnitudes next to each other."""
+    inp = inputs(rows, cols, seed=2)
+    w = inp.w.view(-1, M)
+    w[0::9, 1 % M] = w[0::9, 0]
+    w[1::9, M - 1] = -w[1::9, 0]
+    w[2::9, :] = 0.0
+    w[3::9, 0] = -0.0
+    w[4::9, :] = 0.125
+    w[5::9, 0] = 1e-41
+    w[5::9, M - 1] = -1e-41
+    w[6::9, 0] = 3e4
+    w[6::9, 1 % M] = 1e-30
+    w[7::9, M // 2] = 0.0
+    return inp
+
+
+@pytest.mark.parametrize("N,M", [(2, 4), (1, 4), (4, 8), (5, 16), (8, 32)])
+def test_adversarial_values(N, M):
+    rows, cols = 12, 384
+    inp = adversarial(rows, cols, M)
+    flags = RS | (0 if (N, M) == (2, 4) else BM)
+    h = Hyper(l1_coeff=1e-3, step=500, total_steps=1000)
+    got = U.run_cuda_single(inp, N, M, h, flags)
+    U.assert_parity(got, U.run_oracle(inp, N, M, h, flags), f"adversarial {N}:{M}")
+    assert U.near_tie_groups(inp.w.numpy(), N, M) > 0        # the census sees the planted ties; masks still agree
+
+
+@pytest.mark.parametrize("extra", [0, BM, B.CAST_F_V_KEPT_FROM_G, B.CAST_F_EMIT_DENSE,
+                                   BM | B.CAST_F_V_KEPT_FROM_G | B.CAST_F_EMIT_DENSE])
+@pytest.mark.parametrize("scale_mode,n_seg", [("none", 1), ("ones", 2), ("jitter", 2), ("jitter", 1), ("jitter", 4), ("jitter", 48)])
+def test_flags_and_scale_segments(extra, scale_mode, n_seg):
+    rows, cols = 9, 768
+    inp = inputs(rows, cols, seed=3, scale_mode=scale_mode)
+    if inp.scale is not None and n_seg != 2:
+        gen = torch.Generator().manual_seed(5)
+        inp.scale = 1.0 + 0.1 * torch.rand((rows, n_seg), generator=gen)
+    h = Hyper()
+    got = U.run_cuda_single(inp, 2, 4, h, RS | extra)
+    U.assert_parity(got, U.run_oracle(inp, 2, 4, h, RS | extra), f"flags {extra} scale {scale_mode}/{n_seg}")
+
+
+@pytest.mark.parametrize("bitmask", [False, True])
+def test_mask_reuse_and_flip_count(bitmask):
+    """Kept set decoded from the stored metadata (no reselection), and flips against a previous mask."""
+    enc = BM if bitmask else 0
+    rows, cols = 6, 1056
+    inp = inputs(rows, cols, seed=4)
+    h = Hyper()
+    first = U.run_oracle(inp, 2, 4, h, RS | enc)
+    inp2 = inputs(rows, cols, seed=5)              # other weights, so the stored mask is not their top-2
+    got = U.run_cuda_single(inp2, 2, 4, h, enc, meta_in=first["meta"])
+    U.assert_parity(got, U.run_oracle(inp2, 2, 4, h, enc, meta_in=first["meta"]), "reuse")
+    assert np.array_equal(got["meta"], first["meta"])
+    fl = RS | enc | B.CAST_F_COUNT_FLIPS
+    got = U.run_cuda_single(inp2, 2, 4, h, fl, meta_in=first["meta"])
+    ref = U.run_oracle(inp2, 2, 4, h, fl, meta_in=first["meta"])
+    U.assert_parity(got, ref, "flips")
+    assert got["flips"] == ref["flips"] > 0
+
+
+def test_general_nm_flip_count():
+    inp = inputs(4, 512, seed=6)
+    prev = U.run_oracle(inputs(4, 512, seed=7), 4, 8, Hyper(), RS | BM)["meta"]
+    fl = RS | BM | B.CAST_F_COUNT_FLIPS
+    got = U.run_cuda_single(inp, 4, 8, Hyper(), fl, meta_in=prev)
+    U.assert_parity(got, U.run_oracle(inp, 4, 8, Hyper(), fl, meta_in=prev), "4:8 flips")
+
+
+def test_single_matrix_3072x768_full():
+    """The one-matrix workload in full (2,359,296 parameters, 1152 tiles)."""
+    w = workloads.workload("opt125m_fc2")
+    rows, cols = w.shapes[0]
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=0, tensor_index=0, device=DEV, scale_mode="jitter")
+    inp = workloads.TensorInputs(inp.w.cpu(), inp.g.cpu(), inp.m.cpu(), inp.v.cpu(), inp.scale.cpu())
+    h = Hyper(total_steps=w.total_steps)
+    got = U.run_cuda_single(inp, 2, 4, h, RS)
+    ref = U.run_oracle(inp, 2, 4, h, RS)
+    U.assert_parity(got, ref, "3072x768")
+    U.assert_parity(got, U.run_oracle(inp, 2, 4, h, RS, precision="f32"), "3072x768 f32")
+    ties = U.near_tie_groups(inp.w.numpy(), 2, 4)
+    print(f"near-tie groups: {ties} of {rows * cols // 4}; mask mismatches: 0; "
+          f"v pure relative error {U.v_pure_relative_error(got, ref):.3g}")
+    assert U.v_pure_relative_error(got, ref) < 1e-6
+
+
+def test_two_runs_are_bit_identical():
+    inp = inputs(64, 1024, seed=8)
+    a = U.run_cuda_single(inp, 2, 4, Hyper(), RS)
+    b = U.run_cuda_single(inp, 2, 4, Hyper(), RS)
+    for k in ("w", "m", "v", "w_fwd", "meta"):
+        assert np.array_equal(a[k].view(np.uint8), b[k].view(np.uint8))
+
+
+def test_three_steps_with_refresh_schedule():
+    """Steps t = 9, 10, 11 with the paper's refresh every T1 = 10 iterations: step 10 reselects and counts
+    flips, the others reuse the stored mask.  Each step starts from the CUDA path's own previous state,
+    copied to the host for the oracle, so every step is compared from identical inputs."""
+    rows, cols = 16, 2048
+    inp = inputs(rows, cols, seed=9)
+    meta = U.run_oracle(inp, 2, 4, Hyper(lr=0.0), RS)["meta"]       # mask of step 0
+    for t in (9, 10, 11):
+        flags = (RS | B.CAST_F_COUNT_FLIPS) if t % 10 == 0 else 0
+        h = Hyper(lr=5e-3, l1_coeff=1e-3, step=t, total_steps=12)
+        inp.g = workloads.gen_gradient(rows, cols, 9, 0, t)
+        got = U.run_cuda_single(inp, 2, 4, h, flags, meta_in=meta)
+        ref = U.run_oracle(inp, 2, 4, h, flags, meta_in=meta)
+        U.assert_parity(got, ref, f"step {t}")
+        if t == 10:
+            assert got["flips"] == ref["flips"]
+        inp.w, inp.m, inp.v = (torch.from_numpy(got[k].copy()) for k in ("w", "m", "v"))
+        meta = got["meta"]
+
+
+def test_stream_argument_is_honoured():
+    inp = inputs(32, 512, seed=10)
+    s = torch.cuda.Stream(device=DEV)
+    st = U.to_device(inp, DEV)
+    torch.cuda.synchronize()
+    lr, b1, b2, eps, lam = Hyper().as_f32()
+    cast.check(cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view,
+                                    st.scale, 2, 32, 512, 2, 4, lr, b1, b2, eps, lam, 1000, 30000, RS, None, s))
+    s.synchronize()
+    U.assert_parity(U.device_outputs(st), U.run_oracle(inp, 2, 4, Hyper(), RS), "side stream")
+
+
+def test_device_pointer_kind_is_checked():
+    inp = inputs(4, 64, seed=11)
+    st = U.to_device(inp, DEV)
+    host_w = torch.zeros(4 * 64)
+    before = cast.cast_kernel_launch_count()
+    rc = cast.cast_adams_step(host_w, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view,
+                              None, 1, 4, 64, 2, 4, 1e-4, 0.9, 0.95, 1e-8, 1e-3, 1, 10, RS, None, None)
+    assert rc == B.CAST_ERR_MEMORY and cast.cast_kernel_launch_count() == before

@@ -1,0 +1,135 @@
+"""Multi-tensor plan (one launch over all matrices) and host-resident state, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2509_25996_b200 as cast
+from paper_2509_25996_b200 import binding as B
+from paper_2509_25996_b200 import workloads
+from oracle.adams_oracle import Hyper
+import gpu_util as U
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+RS, BM = B.CAST_F_RESELECT, B.CAST_F_META_BITMASK
+
+
+def run_plan(inputs_list, N, M, hyper: Hyper, flags, metas=None):
+    states = [U.to_device(inp, DEV, None if metas is None else metas[i]) for i, inp in enumerate(inputs_list)]
+    tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale,
+                             1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in states]
+    rc, plan = cast.cast_plan_create(tensors, N, M)
+    cast.check(rc)
+    flips = torch.zeros(1, dtype=torch.int64, device=DEV) if flags & B.CAST_F_COUNT_FLIPS else None
+    lr, b1, b2, eps, lam = hyper.as_f32()
+    before = cast.cast_kernel_launch_count()
+    cast.check(cast.cast_plan_step(plan, B.make_hyper(lr, b1, b2, eps, lam, hyper.step, hyper.total_steps, flags),
+                                   flips, torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == before + 1          # one grid covers every matrix
+    cast.check(cast.cast_plan_destroy(plan))
+    assert all(s.all_intact() for s in states)
+    return [U.device_outputs(s) for s in states], (None if flips is None else int(flips.item()))
+
+
+def test_plan_mixed_shapes_ragged_tiles():
+    """Matrices of 0.02 to 33 tiles, most with a ragged last tile, some without a scale tensor."""
+    shapes = [(1, 32), (3, 96), (64, 1056), (7, 2080), (1, 2048), (33, 2048), (5, 416), (2, 64), (40, 800)]
+    ins = [workloads.gen_tensor_inputs(r, c, seed=20, tensor_index=i, device="cpu",
+                                       scale_mode=("none" if i % 3 == 0 else "jitter")) for i, (r, c) in enumerate(shapes)]
+    h = Hyper()
+    fl = RS | B.CAST_F_COUNT_FLIPS
+    prev = [U.run_oracle(workloads.gen_tensor_inputs(r, c, seed=21, tensor_index=i), 2, 4, h, RS)["meta"]
+            for i, (r, c) in enumerate(shapes)]
+    got, flips = run_plan(ins, 2, 4, h, fl, prev)
+    total = 0
+    for i, inp in enumerate(ins):
+        ref = U.run_oracle(inp, 2, 4, h, fl, meta_in=prev[i])
+        U.assert_parity(got[i], ref, f"tensor {i} {shapes[i]}")
+        total += ref["flips"]
+    assert flips == total
+
+
+@pytest.mark.parametrize("N,M", [(4, 8), (1, 4), (8, 16)])
+def test_plan_general_nm(N, M):
+    shapes = [(16, 512), (9, 1184), (3, 4096)]
+    ins = [workloads.gen_tensor_inputs(r, c, seed=22, tensor_index=i, scale_mode="jitter") for i, (r, c) in enumerate(shapes)]
+    got, _ = run_plan(ins, N, M, Hyper(total_steps=7500), RS | BM)
+    for i, inp in enumerate(ins):
+        U.assert_parity(got[i], U.run_oracle(inp, N, M, Hyper(total_steps=7500), RS | BM), f"{N}:{M} tensor {i}")
+
+
+def test_plan_decoder_d768_12_layers_full():
+    """All 72 linear weights of the 12-layer d=768 decoder (84,934,656 parameters), one launch, compared in full."""
+    wl = workloads.workload("decoder_d768_12l")
+    h = Hyper(total_steps=wl.total_steps)
+    ins = []
+    for i, (r, c) in enumerate(wl.shapes):
+        t = workloads.gen_tensor_inputs(r, c, seed=0, tensor_index=i, device=DEV, scale_mode="jitter")
+        ins.append(workloads.TensorInputs(t.w.cpu(), t.g.cpu(), t.m.cpu(), t.v.cpu(), t.scale.cpu()))
+    got, _ = run_plan(ins, 2, 4, h, RS)
+    ties = 0
+    for i, inp in enumerate(ins):
+        U.assert_parity(got[i], U.run_oracle(inp, 2, 4, h, RS), f"tensor {i} {wl.shapes[i]}")
+        ties += U.near_tie_groups(inp.w.numpy(), 2, 4)
+    print(f"near-tie groups: {ties} of {wl.n_params // 4}; mask mismatches: 0")
+
+
+def test_plan_rejects_wrong_device_memory_and_survives():
+    inp = workloads.gen_tensor_inputs(4, 64, seed=23)
+    s = U.to_device(inp, DEV)
+    host = torch.zeros(4 * 64)
+    bad = B.make_tensor(host, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, None, 1, 4, 64)
+    rc, plan = cast.cast_plan_create([bad], 2, 4)
+    assert rc == B.CAST_ERR_MEMORY and plan is None
+
+
+# ------------------------------------------------------------------------------- host-resident state
+
+def pinned(t: torch.Tensor) -> torch.Tensor:
+    return t.contiguous().pin_memory()
+
+
+@pytest.mark.parametrize("block,slots", [(4096, 2), (8192 * 3, 3)])
+def test_host_step_blocks_match_oracle(block, slots):
+    rows, cols = 37, 1024                      # 37 rows in blocks of 4 (or 24) rows: several blocks + a short one
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=30, scale_mode="jitter")
+    h = Hyper()
+    prev = U.run_oracle(workloads.gen_tensor_inputs(rows, cols, seed=31), 2, 4, h, RS)["meta"]
+    fl = RS | B.CAST_F_COUNT_FLIPS
+    ref = U.run_oracle(inp, 2, 4, h, fl, meta_in=prev)
+    w, m, v, g, sc = pinned(inp.w), pinned(inp.m), pinned(inp.v), pinned(inp.g), pinned(inp.scale)
+    fwd = pinned(torch.zeros((rows, cols), dtype=torch.bfloat16))
+    meta = pinned(torch.from_numpy(prev.view(np.int32).copy()))
+    flips = np.zeros(1, dtype=np.uint64)
+    rc, ctx = cast.cast_host_ctx_create(block, slots)
+    cast.check(rc)
+    lr, b1, b2, eps, lam = h.as_f32()
+    cast.check(cast.cast_host_step(ctx, w, m, v, g, fwd, meta, sc, 2, rows, cols, 2, 4, lr, b1, b2, eps, lam,
+                                   h.step, h.total_steps, fl, flips))
+    cast.check(cast.cast_host_ctx_sync(ctx))
+    got = dict(w=w.numpy(), m=m.numpy(), v=v.numpy(), w_fwd=workloads.bf16_bits(fwd),
+               meta=meta.numpy().view(np.uint32), flips=int(flips[0]))
+    U.assert_parity(got, ref, f"host blocks of {block}")
+    # rows longer than a block are refused
+    assert cast.cast_host_step(ctx, w, m, v, g, fwd, meta, sc, 2, 1, rows * cols, 2, 4, lr, b1, b2, eps, lam,
+                               h.step, h.total_steps, RS, None) in (B.CAST_ERR_PLAN, B.CAST_ERR_SHAPE)
+    cast.check(cast.cast_host_ctx_destroy(ctx))
+
+
+def test_host_step_pageable_memory():
+    rows, cols = 8, 512
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=32, scale_mode="none")
+    ref = U.run_oracle(inp, 2, 4, Hyper(), RS)
+    fwd = torch.zeros((rows, cols), dtype=torch.bfloat16)
+    meta = torch.zeros((rows, cols // 32), dtype=torch.int32)
+    rc, ctx = cast.cast_host_ctx_create(2048, 2)
+    cast.check(rc)
+    lr, b1, b2, eps, lam = Hyper().as_f32()
+    cast.check(cast.cast_host_step(ctx, inp.w, inp.m, inp.v, inp.g, fwd, meta, None, 1, rows, cols, 2, 4,
+                                   lr, b1, b2, eps, lam, 1000, 30000, RS, None))
+    cast.check(cast.cast_host_ctx_destroy(ctx))
+    got = dict(w=inp.w.numpy(), m=inp.m.numpy(), v=inp.v.numpy(), w_fwd=workloads.bf16_bits(fwd),
+               meta=meta.numpy().view(np.uint32))
+    U.assert_parity(got, ref, "pageable")
