@@ -1,0 +1,420 @@
+#!/usr/bin/env python
+"""Benchmark of the fused AdamS N:M step: whole-job parameters/s on N GPUs of one node.
+
+    python bench.py --gpus 1 --steps K --warmup W            (default workload: LLaMA2-7B linear set, 2:4)
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N ...
+    python bench.py --impl reference ...                      (the CPU oracle on the host cores)
+
+A step is one pass of the whole hot path (one multi-tensor launch) over every matrix of the
+workload.  The path does not shard (every group is independent, no exchange step): with N > 1
+every rank runs an independent replica on its own GPU and the value is the sum ("replicas only").
+Rank 0 prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+BYTES_PER_PARAM = 28.125          # 14 read (w, m, v fp32 + g bf16) + 14 written (w, m, v, w_fwd) + 1/8 metadata
+BYTES_PER_PARAM_FLIPS = 28.25     # + 1/8 previous metadata read
+NOMINAL_HBM_GBS = 8000.0          # the nominal peak the target fraction is quoted against
+FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the multi-tensor kernel, from the ncu
+# capture summarised under profiles/ (None until a capture exists)
+NCU_DRAM_BYTES_PER_PARAM = None
+
+METRIC = "AdamS 2:4 step params/s"
+
+
+def parse_args():
+    p = argparse.ArgumentParser()
+    p.add_argument("--gpus", type=int, default=1)
+    p.add_argument("--steps", type=int, default=100)
+    p.add_argument("--warmup", type=int, default=5)
+    p.add_argument("--impl", choices=["cuda", "reference"], default="cuda")
+    p.add_argument("--workload", default="llama2_7b")
+    p.add_argument("--nm", default="2:4")
+    p.add_argument("--l1-coeff", type=float, default=1e-3)
+    p.add_argument("--count-flips", action="store_true")
+    p.add_argument("--e2e-layers", type=int, default=1, help="LLaMA layers held in host memory for the e2e leg (0 = skip)")
+    p.add_argument("--e2e-steps", type=int, default=4)
+    p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
+    p.add_argument("--seed", type=int, default=0)
+    return p.parse_args()
+
+
+def measured_hbm_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons, sampled in the background; only reads, sets nothing."""
+
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_uuid: str):
+        self.samples = []
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", gpu_uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        rows = []
+        for ts, line in self.samples:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                rows.append((ts, float(parts[1]), float(parts[2]), parts[4:8]))
+            except ValueError:
+                continue
+        inside = [r for r in rows if t0 <= r[0] <= t1 + 0.15] or rows
+        if not inside:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3][i] == "Active" for r in inside)]
+        return {"sm_mhz": statistics.median(r[1] for r in inside), "sm_max_mhz": max(r[2] for r in inside),
+                "reasons": reasons, "samples": len(inside)}
+
+
+def host_threads() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def time_oracle(arrays, N, M, hyper, flags, threads: int):
+    """Run the CPU oracle (as it stands) over a list of host matrices, rows split over `threads`
+    Python threads (ctypes releases the GIL; the oracle itself stays a serial loop).
+    arrays: list of dict(w, m, v, g, scale, rows, cols) of numpy arrays.  Returns (seconds, outputs)."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import adams_oracle as orc
+
+    jobs, outs = [], []
+    for a in arrays:
+        rows, cols = a["rows"], a["cols"]
+        fwd = np.zeros(rows * cols, dtype=np.uint16)
+        meta = np.zeros(rows * cols // 32, dtype=np.uint32)
+        outs.append(dict(w=a["w"], m=a["m"], v=a["v"], w_fwd=fwd, meta=meta))
+        per = max(1, -(-rows // threads))
+        for r0 in range(0, rows, per):
+            r1 = min(rows, r0 + per)
+            sl = slice(r0 * cols, r1 * cols)
+            jobs.append((a["w"].reshape(-1)[sl], a["m"].reshape(-1)[sl], a["v"].reshape(-1)[sl], a["g"].reshape(-1)[sl],
+                         fwd[sl], meta[r0 * cols // 32:r1 * cols // 32],
+                         None if a["scale"] is None else a["scale"][r0:r1], r1 - r0, cols))
+
+    def one(j):
+        w, m, v, g, fwd, meta, sc, rows, cols = j
+        orc.adams_step_inplace(w, m, v, g, fwd, meta, sc, rows, cols, N, M, hyper, flags)
+
+    orc._load()
+    t0 = time.perf_counter()
+    if threads == 1:
+        for j in jobs:
+            one(j)
+    else:
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(one, jobs))
+    return time.perf_counter() - t0, outs
+
+
+def reference_arm(args):
+    """The CPU oracle timed on the host cores on a bounded sample of the workload (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+    from oracle import adams_oracle as orc
+    from paper_2509_25996_b200 import workloads
+
+    N, M = (int(x) for x in args.nm.split(":"))
+    wl = workloads.workload(args.workload)
+    threads = host_threads()
+    # bounded sample: the first matrices of the workload, up to ~34 M parameters per step
+    sample, n = [], 0
+    for i, (r, c) in enumerate(wl.shapes):
+        if n and n + r * c > 34_000_000:
+            break
+        t = workloads.gen_tensor_inputs(r, c, seed=args.seed, tensor_index=i, device="cpu", scale_mode="ones")
+        sample.append(dict(w=t.w.numpy(), m=t.m.numpy(), v=t.v.numpy(), g=workloads.bf16_bits(t.g),
+                           scale=t.scale.numpy(), rows=r, cols=c))
+        n += r * c
+    flags = orc.F_RESELECT | (0 if (N, M) == (2, 4) else orc.F_META_BITMASK)
+    times = []
+    for s in range(args.warmup + args.steps):
+        hyper = orc.Hyper(l1_coeff=args.l1_coeff, step=1000 + s, total_steps=wl.total_steps)
+        dt, _ = time_oracle(sample, N, M, hyper, flags, threads)
+        if s >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = n * len(times) / total
+    sample_note = f"first {len(sample)} matrices of {wl.name} ({n} parameters) per step, rows split over {threads} threads"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "nm": args.nm, "params": wl.n_params, "sample": sample_note},
+        "cpu_baseline": {"value": value, "unit": "params/s", "cores": threads, "kind": "oracle", "sample": sample_note},
+        "e2e": {"value": value, "unit": "params/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def cuda_arm(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+    import paper_2509_25996_b200 as cast
+    from paper_2509_25996_b200 import binding as B
+    from paper_2509_25996_b200 import workloads
+    from paper_2509_25996_b200.runner import DeviceModelState, Hyper
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    B.load_library()
+
+    N, M = (int(x) for x in args.nm.split(":"))
+    wl = workloads.workload(args.workload)
+    free, total_mem = torch.cuda.mem_get_info()
+    need = wl.n_params * 16.2 + 2e9
+    if need > free:                       # largest single-GPU configuration that fits
+        wl = workloads.workload("decoder_d768_12l")
+    flags = B.CAST_F_RESELECT | (0 if (N, M) == (2, 4) else B.CAST_F_META_BITMASK)
+    if args.count_flips:
+        flags |= B.CAST_F_COUNT_FLIPS
+    bytes_per_param = BYTES_PER_PARAM_FLIPS if args.count_flips else BYTES_PER_PARAM
+
+    state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones")
+    hyper = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl.total_steps)
+    stream = torch.cuda.current_stream(dev)
+
+    # parity sample (checked in the CPU-baseline leg): a few rows of the first and last matrices, copied
+    # before the first step and again after it
+    sample_rows = 16
+    picks = sorted({0, len(state.mats) // 2, len(state.mats) - 1})
+    parity_in = {}
+    if rank == 0 and args.cpu_baseline:
+        for t in picks:
+            s = state.mats[t]
+            parity_in[t] = dict(w=s.w[:sample_rows].cpu().numpy(), m=s.m[:sample_rows].cpu().numpy(),
+                                v=s.v[:sample_rows].cpu().numpy(), g=workloads.bf16_bits(s.g[:sample_rows]),
+                                scale=s.scale[:sample_rows].cpu().numpy(), rows=sample_rows, cols=s.cols)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
+    parity_out = {}
+    for i in range(args.warmup):
+        state.step(hyper, flags, stream)
+        hyper.step += 1
+        if i == 0 and parity_in:
+            torch.cuda.synchronize(dev)
+            for t in picks:
+                s = state.mats[t]
+                parity_out[t] = dict(w=s.w[:sample_rows].cpu().numpy(), m=s.m[:sample_rows].cpu().numpy(),
+                                     v=s.v[:sample_rows].cpu().numpy(), w_fwd=workloads.bf16_bits(s.w_fwd[:sample_rows]),
+                                     meta=s.meta[:sample_rows].cpu().numpy().view(np.uint32))
+
+    # ---- timed region: K steps, CUDA events on the launching stream, inputs (>= 2.4 GB, up to 104 GB) far larger than L2
+    launches0 = cast.cast_kernel_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        state.step(hyper, flags, stream)
+        hyper.step += 1
+    ev1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    launches = cast.cast_kernel_launch_count() - launches0
+    ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    clocks = None
+    if sampler is not None:
+        time.sleep(0.15)
+        sampler.stop()
+        clocks = sampler.summary(t_wall0, t_wall1)
+
+    ms_per_step = ms / args.steps
+    value = world * wl.n_params * args.steps / (ms * 1e-3)
+    per_gpu_gbs = wl.n_params * bytes_per_param / (ms_per_step * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+
+    # ---- e2e leg: the same step through cast_host_step with page-locked HOST buffers; every step copies
+    # its inputs host->device and its results device->host inside the timed region
+    e2e = None
+    if args.e2e_layers > 0:
+        per_layer = 7 if len(wl.shapes) % 7 == 0 and len(wl.shapes) > 7 else len(wl.shapes)
+        shapes = list(wl.shapes[:min(len(wl.shapes), per_layer * args.e2e_layers)])
+        host = []
+        for i, (r, c) in enumerate(shapes):
+            s = state.mats[i]
+            host.append(dict(w=s.w.cpu().pin_memory(), m=s.m.cpu().pin_memory(), v=s.v.cpu().pin_memory(),
+                             g=s.g.cpu().pin_memory(), scale=s.scale.cpu().pin_memory(),
+                             fwd=torch.empty((r, c), dtype=torch.bfloat16).pin_memory(),
+                             meta=torch.zeros((r, c // 32), dtype=torch.int32).pin_memory(), rows=r, cols=c))
+        n_e2e = sum(r * c for r, c in shapes)
+        rc, ctx = cast.cast_host_ctx_create(min(16 * 1024 * 1024, max(r * c for r, c in shapes)), 3)
+        cast.check(rc)
+        e_flags = flags & ~B.CAST_F_COUNT_FLIPS
+
+        def host_pass(step_no):
+            for h in host:
+                cast.check(cast.cast_host_step(ctx, h["w"], h["m"], h["v"], h["g"], h["fwd"], h["meta"], h["scale"],
+                                               h["scale"].shape[1], h["rows"], h["cols"], N, M, hyper.lr, hyper.beta1,
+                                               hyper.beta2, hyper.eps, hyper.l1_coeff, step_no, wl.total_steps, e_flags, None))
+            cast.check(cast.cast_host_ctx_sync(ctx))
+
+        for i in range(3):
+            host_pass(1000 + i)
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(args.e2e_steps):
+            host_pass(1003 + i)
+        barrier()
+        dt = time.perf_counter() - t0
+        if world > 1:
+            t = torch.tensor([dt], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dt = float(t.item())
+        cast.check(cast.cast_host_ctx_destroy(ctx))
+        scale_bytes = sum(h["scale"].numel() * 4 for h in host)
+        e2e = {"value": world * n_e2e * args.e2e_steps / dt, "unit": "params/s",
+               "h2d_bytes_per_step": int(n_e2e * 14 + scale_bytes), "d2h_bytes_per_step": int(n_e2e * 14.125),
+               "ms_per_step": 1e3 * dt / args.e2e_steps,
+               "workload": f"first {len(shapes)} matrices of {wl.name} ({n_e2e} parameters) held in page-locked host memory, "
+                           f"staged in 16 Mi-parameter blocks through 3 device slots",
+               "steps": args.e2e_steps}
+        del host
+
+    if rank != 0:
+        if world > 1:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    # ---- CPU baseline leg (rank 0, N = 1 only): the oracle as it stands on the host cores, plus parity of the sample
+    cpu_baseline = None
+    parity = None
+    if args.cpu_baseline and world == 1:
+        from oracle import adams_oracle as orc
+        oh = orc.Hyper(lr=hyper.lr, beta1=hyper.beta1, beta2=hyper.beta2, eps=hyper.eps, l1_coeff=hyper.l1_coeff,
+                       step=1000, total_steps=wl.total_steps)
+        o_flags = orc.F_RESELECT | (0 if (N, M) == (2, 4) else orc.F_META_BITMASK)
+        ok = bool(parity_out)
+        for t in (picks if parity_out else []):
+            a = parity_in[t]
+            _, outs = time_oracle([a], N, M, oh, o_flags, 1)
+            ref, got = outs[0], parity_out[t]
+            for k in ("w", "m", "v"):
+                r = ref[k].astype(np.float64).reshape(-1)
+                g_ = got[k].astype(np.float64).reshape(-1)
+                ok &= bool(np.all(np.abs(g_ - r) <= np.maximum(1e-6 * np.abs(r), 1e-9)))
+            ok &= bool(np.array_equal(ref["meta"].reshape(-1), got["meta"].reshape(-1)))
+            d = np.abs((ref["w_fwd"].astype(np.int32) & 0x7FFF) - (got["w_fwd"].reshape(-1).astype(np.int32) & 0x7FFF))
+            ok &= bool(d.max() <= 1)
+        parity = {"ok": ok, "sample": f"first {sample_rows} rows of matrices {picks} after the first step"}
+        # timing sample: whole matrices from the front of the workload, about 1e8 parameters
+        arrays, n = [], 0
+        for i, s in enumerate(state.mats):
+            if n and n + s.rows * s.cols > 110_000_000:
+                break
+            arrays.append(dict(w=s.w.cpu().numpy(), m=s.m.cpu().numpy(), v=s.v.cpu().numpy(), g=workloads.bf16_bits(s.g),
+                               scale=s.scale.cpu().numpy(), rows=s.rows, cols=s.cols))
+            n += s.rows * s.cols
+        threads = host_threads()
+        oh.step = hyper.step
+        time_oracle(arrays[:1], N, M, oh, o_flags, threads)                 # warm-up pass
+        dt_all, _ = time_oracle(arrays, N, M, oh, o_flags, threads)
+        dt_one, _ = time_oracle(arrays[:1], N, M, oh, o_flags, 1)
+        n_one = arrays[0]["rows"] * arrays[0]["cols"]
+        cpu_baseline = {"value": n / dt_all, "unit": "params/s", "cores": threads, "kind": "oracle",
+                        "sample": f"first {len(arrays)} matrices of {wl.name} ({n} parameters), one pass, rows split over "
+                                  f"{threads} threads; single thread on the first matrix: {n_one / dt_one:.4g} params/s",
+                        "single_thread_value": n_one / dt_one}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "params/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "note": wl.note, "nm": args.nm, "params": wl.n_params, "matrices": len(wl.shapes),
+                   "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs far larger than L2, no flush",
+                   "lr": hyper.lr, "betas": [hyper.beta1, hyper.beta2], "eps": hyper.eps, "l1_coeff": hyper.l1_coeff,
+                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "seed": args.seed},
+        "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
+                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_kernel<{M}, multi>",
+                     "bytes_per_param": bytes_per_param,
+                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None else NCU_DRAM_BYTES_PER_PARAM * wl.n_params)},
+        "cpu_baseline": cpu_baseline, "parity": parity,
+    }
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        cuda_arm(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -129,7 +129,10 @@ def test_single_matrix_3072x768_full():
     ties = U.near_tie_groups(inp.w.numpy(), 2, 4)
     print(f"near-tie groups: {ties} of {rows * cols // 4}; mask mismatches: 0; "
           f"v pure relative error {U.v_pure_relative_error(got, ref):.3g}")
-    assert U.v_pure_relative_error(got, ref) < 1e-6
+    # The 1e-9 floor is loose for v (~1e-6), so its pure relative error is reported too.  It is not
+    # ~1e-7 everywhere: where beta1 m and (1-beta1) g nearly cancel, mu carries a large relative (tiny
+    # absolute) error in any fp32 evaluation, and mu^2 dominates v when the old v is tiny.
+    assert U.v_pure_relative_error(got, ref) < 1e-4
 
 
 def test_two_runs_are_bit_identical():
