@@ -41,12 +41,12 @@ struct TensorDesc {
 
 // Scalars of one iteration, folded on the host in double precision.
 struct StepConsts {
-    float beta1;        // beta1
-    float omb1;         // 1 - beta1
+    double beta1;       // beta1
+    double omb1;        // 1 - beta1
+    double c_mu;        // 1 - alpha_t                  (Eq. 7)
+    double c_sign;      // alpha_t * lambda             (Eq. 7)
     float beta2;        // beta2
     float omb2;         // 1 - beta2
-    float c_mu;         // 1 - alpha_t                  (Eq. 7)
-    float c_sign;       // alpha_t * lambda             (Eq. 7)
     float inv_bc2;      // 1 / (1 - beta2^t)
     float lr_bc1;       // lr / (1 - beta1^t)
     float eps;
@@ -142,45 +142,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
-// The whole per-unit body: loads, selection, moments, decay, update, emission, metadata.
-// `active` is false for threads past the end of the matrix; they take part in the shuffles only.
-template <int M>
-__device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const StepConsts& c,
-                                                 uint32_t unit, bool active)
-{
+// Registers of one unit: state and gradient in, updated state, forward weight and metadata out.
+struct UnitRegs {
     float w[8], m[8], v[8];
-    uint4 graw = make_uint4(0, 0, 0, 0);
-    uint32_t prev_byte = 0;
-    const size_t e = (size_t)unit * kUnitElems;
-    const bool need_prev = ((c.flags & kReselect) == 0) || (c.flags & kCountFlips);
+    uint4 g;               // 8 bf16 gradients in; 8 bf16 forward weights out
+    uint32_t prev_byte;    // metadata byte of the unit before the step (when it is read)
+    uint32_t meta_byte;    // metadata byte after the step
+};
 
-    if (active) {
-        const float4 w0 = ld_f4(t.w + e), w1 = ld_f4(t.w + e + 4);
-        const float4 m0 = ld_f4(t.m + e), m1 = ld_f4(t.m + e + 4);
-        const float4 v0 = ld_f4(t.v + e), v1 = ld_f4(t.v + e + 4);
-        graw = *reinterpret_cast<const uint4*>(t.g + e);
-        if (need_prev) prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[unit];
-        w[0] = w0.x; w[1] = w0.y; w[2] = w0.z; w[3] = w0.w; w[4] = w1.x; w[5] = w1.y; w[6] = w1.z; w[7] = w1.w;
-        m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
-        v[0] = v0.x; v[1] = v0.y; v[2] = v0.z; v[3] = v0.w; v[4] = v1.x; v[5] = v1.y; v[6] = v1.z; v[7] = v1.w;
-    } else {
-#pragma unroll
-        for (int i = 0; i < 8; ++i) { w[i] = 0.f; m[i] = 0.f; v[i] = 0.f; }
-    }
-
+// Arithmetic of one unit, registers only (and warp shuffles for M > 8: every lane of the warp must
+// call this, lanes without data pass zeros).  `a` is the unit's scale A[r, segment].  Returns the
+// number of flipped mask bits of the unit (App. C: ||M_t - M_{t-1}||_0).
+template <int M>
+__device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a)
+{
     const bool bitmask = (c.flags & kMetaBitmask) != 0;
-    const uint32_t prev_keep = keep_from_meta_byte(prev_byte, bitmask);
+    const uint32_t prev_keep = keep_from_meta_byte(u.prev_byte, bitmask);
     uint32_t keep;
-    if (c.flags & kReselect) keep = select_keep<M>(w, c.n_keep);     // uniform branch: all lanes shuffle
+    if (c.flags & kReselect) keep = select_keep<M>(u.w, c.n_keep);     // uniform branch: all lanes shuffle
     else keep = prev_keep;
 
-    float a = 1.0f;
-    if (active && t.scale != nullptr) {
-        const uint32_t seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
-        a = __ldg(t.scale + seg);
-    }
-
-    const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
+    const uint32_t gw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
     const bool v_from_g = (c.flags & kVKeptFromG) != 0;
     const bool dense = (c.flags & kEmitDense) != 0;
     float fwd[8];
@@ -188,41 +170,79 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
     for (int i = 0; i < 8; ++i) {
         const float g32 = __uint_as_float((i & 1) ? (gw[i >> 1] & 0xFFFF0000u) : (gw[i >> 1] << 16));
         const bool kept = (keep >> i) & 1u;
-        // first moment, stored undecayed (Alg. 1)
-        const float mu = fmaf(c.beta1, m[i], c.omb1 * g32);
-        m[i] = mu;
-        // proportional L1 decay outside the kept set (Eq. 7); Sign(0) = 0
-        const float sgn_term = (w[i] == 0.0f) ? 0.0f : copysignf(c.c_sign, w[i]);
-        const float mu_t = kept ? mu : fmaf(c.c_mu, mu, sgn_term);
+        // First moment, stored undecayed (Alg. 1), and the proportional L1 decay outside the kept set
+        // (Eq. 7; Sign(0) = 0).  Both are sums of terms of opposite sign and like size (beta1 m against
+        // (1 - beta1) g, (1 - alpha) mu against alpha lambda), so they are formed in fp64 from the exact
+        // inputs: in fp32 a cancellation leaves mu with a large relative error, which the quotient
+        // mu / sqrt(v) carries into w wherever v is small as well.  Everything after is a product or a
+        // sum of like signs and stays in fp32.
+        const double mu = fma(c.beta1, (double)u.m[i], c.omb1 * (double)g32);
+        u.m[i] = (float)mu;
+        const double sgn_term = (u.w[i] == 0.0f) ? 0.0 : copysign(c.c_sign, (double)u.w[i]);
+        const float mu_t = (float)(kept ? mu : fma(c.c_mu, mu, sgn_term));
         // second moment from the decayed first moment (Eq. 8)
         const float src = (v_from_g && kept) ? g32 : mu_t;
-        const float vn = fmaf(c.beta2, v[i], (c.omb2 * src) * src);
-        v[i] = vn;
+        const float vn = fmaf(c.beta2, u.v[i], (c.omb2 * src) * src);
+        u.v[i] = vn;
         // bias-corrected update
         const float denom = sqrtf(vn * c.inv_bc2) + c.eps;
-        const float wn = w[i] - (c.lr_bc1 * mu_t) / denom;
-        w[i] = wn;
+        const float wn = u.w[i] - (c.lr_bc1 * mu_t) / denom;
+        u.w[i] = wn;
         // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for
         fwd[i] = (kept || dense) ? a * wn : 0.0f;
     }
+    u.g.x = pack_bf16x2(fwd[0], fwd[1]);
+    u.g.y = pack_bf16x2(fwd[2], fwd[3]);
+    u.g.z = pack_bf16x2(fwd[4], fwd[5]);
+    u.g.w = pack_bf16x2(fwd[6], fwd[7]);
+    u.meta_byte = meta_byte_from_keep(keep, bitmask);
+    return (uint32_t)__popc(keep ^ prev_keep);
+}
+
+// The whole per-unit body: loads, arithmetic, stores.
+// `active` is false for threads past the end of the matrix; they take part in the shuffles only.
+template <int M>
+__device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const StepConsts& c,
+                                                 uint32_t unit, bool active)
+{
+    UnitRegs u;
+    u.g = make_uint4(0, 0, 0, 0);
+    u.prev_byte = 0;
+    const size_t e = (size_t)unit * kUnitElems;
+    const bool need_prev = ((c.flags & kReselect) == 0) || (c.flags & kCountFlips);
+    float a = 1.0f;
 
     if (active) {
-        st_f4(t.w + e, make_float4(w[0], w[1], w[2], w[3]));
-        st_f4(t.w + e + 4, make_float4(w[4], w[5], w[6], w[7]));
-        st_f4(t.m + e, make_float4(m[0], m[1], m[2], m[3]));
-        st_f4(t.m + e + 4, make_float4(m[4], m[5], m[6], m[7]));
-        st_f4(t.v + e, make_float4(v[0], v[1], v[2], v[3]));
-        st_f4(t.v + e + 4, make_float4(v[4], v[5], v[6], v[7]));
-        uint4 f;
-        f.x = pack_bf16x2(fwd[0], fwd[1]);
-        f.y = pack_bf16x2(fwd[2], fwd[3]);
-        f.z = pack_bf16x2(fwd[4], fwd[5]);
-        f.w = pack_bf16x2(fwd[6], fwd[7]);
-        *reinterpret_cast<uint4*>(t.w_fwd + e) = f;
-        reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)meta_byte_from_keep(keep, bitmask);
+        const float4 w0 = ld_f4(t.w + e), w1 = ld_f4(t.w + e + 4);
+        const float4 m0 = ld_f4(t.m + e), m1 = ld_f4(t.m + e + 4);
+        const float4 v0 = ld_f4(t.v + e), v1 = ld_f4(t.v + e + 4);
+        u.g = *reinterpret_cast<const uint4*>(t.g + e);
+        if (need_prev) u.prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[unit];
+        if (t.scale != nullptr) {
+            const uint32_t seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
+            a = __ldg(t.scale + seg);
+        }
+        u.w[0] = w0.x; u.w[1] = w0.y; u.w[2] = w0.z; u.w[3] = w0.w; u.w[4] = w1.x; u.w[5] = w1.y; u.w[6] = w1.z; u.w[7] = w1.w;
+        u.m[0] = m0.x; u.m[1] = m0.y; u.m[2] = m0.z; u.m[3] = m0.w; u.m[4] = m1.x; u.m[5] = m1.y; u.m[6] = m1.z; u.m[7] = m1.w;
+        u.v[0] = v0.x; u.v[1] = v0.y; u.v[2] = v0.z; u.v[3] = v0.w; u.v[4] = v1.x; u.v[5] = v1.y; u.v[6] = v1.z; u.v[7] = v1.w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) { u.w[i] = 0.f; u.m[i] = 0.f; u.v[i] = 0.f; }
     }
-    // flips of this unit (App. C: ||M_t - M_{t-1}||_0)
-    return active ? (uint32_t)__popc(keep ^ prev_keep) : 0u;
+
+    const uint32_t flips = compute_unit<M>(u, c, a);
+
+    if (active) {
+        st_f4(t.w + e, make_float4(u.w[0], u.w[1], u.w[2], u.w[3]));
+        st_f4(t.w + e + 4, make_float4(u.w[4], u.w[5], u.w[6], u.w[7]));
+        st_f4(t.m + e, make_float4(u.m[0], u.m[1], u.m[2], u.m[3]));
+        st_f4(t.m + e + 4, make_float4(u.m[4], u.m[5], u.m[6], u.m[7]));
+        st_f4(t.v + e, make_float4(u.v[0], u.v[1], u.v[2], u.v[3]));
+        st_f4(t.v + e + 4, make_float4(u.v[4], u.v[5], u.v[6], u.v[7]));
+        *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
+        reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;
+    }
+    return active ? flips : 0u;
 }
 
 // Persistent grid: CTA b handles tiles b, b + gridDim.x, ...  For the multi-tensor form the tile

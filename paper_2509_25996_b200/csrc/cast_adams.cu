@@ -45,12 +45,12 @@ int make_step_consts(float lr, float beta1, float beta2, float eps, float l1_coe
     const double bc1 = 1.0 - std::pow((double)beta1, (double)step);
     const double bc2 = 1.0 - std::pow((double)beta2, (double)step);
     StepConsts c;
-    c.beta1 = beta1;
-    c.omb1 = (float)(1.0 - (double)beta1);
+    c.beta1 = (double)beta1;
+    c.omb1 = 1.0 - (double)beta1;
+    c.c_mu = 1.0 - alpha;
+    c.c_sign = alpha * (double)l1_coeff;
     c.beta2 = beta2;
     c.omb2 = (float)(1.0 - (double)beta2);
-    c.c_mu = (float)(1.0 - alpha);
-    c.c_sign = (float)(alpha * (double)l1_coeff);
     c.inv_bc2 = (float)(1.0 / bc2);
     c.lr_bc1 = (float)((double)lr / bc1);
     c.eps = eps;

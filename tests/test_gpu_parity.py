@@ -146,19 +146,22 @@ def test_two_runs_are_bit_identical():
 def test_three_steps_with_refresh_schedule():
     """Steps t = 9, 10, 11 with the paper's refresh every T1 = 10 iterations: step 10 reselects and counts
     flips, the others reuse the stored mask.  Each step starts from the CUDA path's own previous state,
-    copied to the host for the oracle, so every step is compared from identical inputs."""
+    copied to the host for the oracle, so every step is compared from identical inputs.  The learning
+    rate keeps the update below ~1e-3 per step: the 1e-9 absolute floor of the tolerance is a few fp32
+    ulps of an update of that size, so a larger rate puts any fp32 evaluation (the fp32 oracle too)
+    outside it wherever w_new is close to zero."""
     rows, cols = 16, 2048
     inp = inputs(rows, cols, seed=9)
     meta = U.run_oracle(inp, 2, 4, Hyper(lr=0.0), RS)["meta"]       # mask of step 0
     for t in (9, 10, 11):
         flags = (RS | B.CAST_F_COUNT_FLIPS) if t % 10 == 0 else 0
-        h = Hyper(lr=5e-3, l1_coeff=1e-3, step=t, total_steps=12)
+        h = Hyper(lr=2e-4, l1_coeff=1e-3, step=t, total_steps=12)
         inp.g = workloads.gen_gradient(rows, cols, 9, 0, t)
         got = U.run_cuda_single(inp, 2, 4, h, flags, meta_in=meta)
         ref = U.run_oracle(inp, 2, 4, h, flags, meta_in=meta)
         U.assert_parity(got, ref, f"step {t}")
         if t == 10:
-            assert got["flips"] == ref["flips"]
+            assert got["flips"] == ref["flips"] > 0
         inp.w, inp.m, inp.v = (torch.from_numpy(got[k].copy()) for k in ("w", "m", "v"))
         meta = got["meta"]
 
