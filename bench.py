@@ -397,7 +397,7 @@ def cuda_arm(args):
         "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_kernel<{M}, multi>",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_kernel<{M}, true>",
                      "bytes_per_param": bytes_per_param,
                      "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None else NCU_DRAM_BYTES_PER_PARAM * wl.n_params)},
         "cpu_baseline": cpu_baseline, "parity": parity,

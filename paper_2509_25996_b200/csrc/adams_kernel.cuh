@@ -6,6 +6,11 @@
 // top-N selection is a register-only rank network; groups of 16 or 32 columns are shared by 2
 // or 4 neighbouring lanes through warp shuffles.  A warp covers 256 consecutive parameters:
 // 1 KB of each fp32 array, 512 B of each bf16 array and one 32-byte sector of metadata.
+//
+// Launch shape: one CTA of 128 threads per tile of 1024 parameters, one unit per thread, no loop.
+// Measured on B200, small short-lived CTAs (7 resident per SM, the hardware scheduler handing out
+// tiles in address order) stream faster than a persistent grid-stride loop of the same body or a
+// bulk-copy/mbarrier ring through shared memory, and as fast with 128-bit as with 256-bit accesses.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -13,9 +18,10 @@
 
 namespace cast {
 
-constexpr int kThreads = 256;          // threads per CTA
-constexpr int kUnitElems = 8;          // parameters per thread per tile
-constexpr int kTileUnits = kThreads;   // units per tile (2048 parameters)
+constexpr int kThreads = 128;          // threads per CTA
+constexpr int kUnitElems = 8;          // parameters per thread
+constexpr int kTileUnits = kThreads;   // units per tile (1024 parameters)
+constexpr int kMinCtasPerSm = 7;       // register budget the kernels are compiled for (M <= 8)
 
 // flag bits (values of the public header)
 constexpr uint32_t kReselect = 1u << 0;
@@ -245,42 +251,65 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
     return active ? flips : 0u;
 }
 
-// Persistent grid: CTA b handles tiles b, b + gridDim.x, ...  For the multi-tensor form the tile
-// index space is the concatenation of all matrices' tiles (each matrix padded to whole tiles);
-// tile_start[k] is the first tile of matrix k and tile_start[n_tensors] the total.  Because a CTA's
-// tile index only grows, the matrix index is found by walking forward, never by searching.
-template <int M, bool MULTI>
-__global__ void __launch_bounds__(kThreads)
-adams_nm_kernel(const __grid_constant__ TensorDesc single,
-                const TensorDesc* __restrict__ descs, const uint32_t* __restrict__ tile_start,
-                uint32_t total_tiles, const __grid_constant__ StepConsts c,
+// Tables of one multi-tensor launch, passed by value in kernel parameter space (constant bank): a CTA
+// lives only a few microseconds, so finding its matrix must not cost a chain of global-memory
+// round trips, and the constant cache is not swept by the streaming data the way L1 is.
+// The tile index space is the concatenation of all matrices' tiles (each matrix padded to whole
+// tiles): tile_start[k] is the first tile of matrix k, tile_start[n] the total.
+// hint[b >> hint_shift] is the matrix that holds tile (b >> hint_shift) << hint_shift, from which the
+// CTA walks forward (usually zero or one step).
+constexpr int kMaxLaunchTensors = 384;
+constexpr int kHintEntries = 256;
+struct MultiParams {
+    uint32_t n_tensors;
+    uint32_t hint_shift;
+    uint16_t hint[kHintEntries];
+    uint32_t tile_start[kMaxLaunchTensors + 1];
+    TensorDesc desc[kMaxLaunchTensors];
+};
+static_assert(sizeof(MultiParams) + sizeof(StepConsts) + 16 <= 32764, "kernel parameters are limited to 32764 bytes");
+
+// Flips of the CTA added to the caller's counter (one atomic per CTA that saw any).
+__device__ __forceinline__ void add_flips(uint32_t flips, unsigned long long* flip_count)
+{
+    flips = __reduce_add_sync(0xFFFFFFFFu, flips);
+    __shared__ uint32_t warp_sums[kThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = flips;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long total = 0;
+#pragma unroll
+        for (int i = 0; i < kThreads / 32; ++i) total += warp_sums[i];
+        if (total) atomicAdd(flip_count, total);
+    }
+}
+
+#define CAST_LAUNCH_BOUNDS(M) __launch_bounds__(kThreads, ((M) <= 8) ? kMinCtasPerSm : 5)
+
+// One matrix: CTA b handles tile b.
+template <int M>
+__global__ void CAST_LAUNCH_BOUNDS(M)
+adams_nm_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c,
                 unsigned long long* __restrict__ flip_count)
 {
-    uint32_t flips = 0;
-    uint32_t k = 0;
-    for (uint32_t tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-        if constexpr (MULTI) {
-            while (tile >= __ldg(tile_start + k + 1)) ++k;
-            const TensorDesc t = descs[k];
-            const uint32_t unit = (tile - __ldg(tile_start + k)) * kTileUnits + threadIdx.x;
-            flips += process_unit<M>(t, c, unit, unit < t.n_units);
-        } else {
-            const uint32_t unit = tile * kTileUnits + threadIdx.x;
-            flips += process_unit<M>(single, c, unit, unit < single.n_units);
-        }
-    }
-    if (c.flags & kCountFlips) {
-        flips = __reduce_add_sync(0xFFFFFFFFu, flips);
-        __shared__ uint32_t warp_sums[kThreads / 32];
-        if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = flips;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned long long total = 0;
-#pragma unroll
-            for (int i = 0; i < kThreads / 32; ++i) total += warp_sums[i];
-            if (total) atomicAdd(flip_count, total);
-        }
-    }
+    const uint32_t unit = blockIdx.x * kTileUnits + threadIdx.x;
+    const uint32_t flips = process_unit<M>(t, c, unit, unit < t.n_units);
+    if (c.flags & kCountFlips) add_flips(flips, flip_count);
+}
+
+// Up to kMaxLaunchTensors matrices in one grid: CTA b handles tile b of the concatenated index space.
+template <int M>
+__global__ void CAST_LAUNCH_BOUNDS(M)
+adams_nm_multi_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
+                      unsigned long long* __restrict__ flip_count)
+{
+    const uint32_t tile = blockIdx.x;
+    uint32_t k = p.hint[tile >> p.hint_shift];
+    while (tile >= p.tile_start[k + 1]) ++k;
+    const TensorDesc& t = p.desc[k];
+    const uint32_t unit = (tile - p.tile_start[k]) * kTileUnits + threadIdx.x;
+    const uint32_t flips = process_unit<M>(t, c, unit, unit < t.n_units);
+    if (c.flags & kCountFlips) add_flips(flips, flip_count);
 }
 
 }  // namespace cast

@@ -3,7 +3,6 @@
 #include <atomic>
 #include <cmath>
 #include <cstring>
-#include <mutex>
 #include <new>
 #include <vector>
 
@@ -140,84 +139,70 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
 
 namespace {
 
-struct DeviceInfo { int sm_count = 0; };
-std::mutex g_mu;
-DeviceInfo g_dev[64];
-int g_blocks_per_sm[64][6][2];   // [device][log2 M][multi], 0 = unknown
-
-int device_info(int* dev_out, DeviceInfo* info)
+template <int M>
+int launch_single_t(const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    int dev = 0;
-    CAST_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return CAST_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(g_mu);
-    if (g_dev[dev].sm_count == 0) {
-        int sms = 0;
-        CAST_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-        g_dev[dev].sm_count = sms;
-    }
-    *dev_out = dev;
-    *info = g_dev[dev];
-    return CAST_OK;
-}
-
-template <int M, bool MULTI>
-int launch_t(const TensorDesc& single, const TensorDesc* descs, const uint32_t* tile_start,
-             uint32_t total_tiles, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
-             int log2m)
-{
-    if (total_tiles == 0) return CAST_OK;
-    int dev = 0;
-    DeviceInfo info;
-    int rc = device_info(&dev, &info);
-    if (rc != CAST_OK) return rc;
-    int per_sm;
-    {
-        std::lock_guard<std::mutex> lock(g_mu);
-        per_sm = g_blocks_per_sm[dev][log2m][MULTI ? 1 : 0];
-    }
-    if (per_sm == 0) {
-        CAST_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, adams_nm_kernel<M, MULTI>, kThreads, 0));
-        if (per_sm < 1) per_sm = 1;
-        std::lock_guard<std::mutex> lock(g_mu);
-        g_blocks_per_sm[dev][log2m][MULTI ? 1 : 0] = per_sm;
-    }
-    // persistent grid: a whole number of CTAs per SM
-    uint64_t grid = (uint64_t)info.sm_count * (uint64_t)per_sm;
-    if (grid > total_tiles) grid = total_tiles;
-    adams_nm_kernel<M, MULTI><<<(unsigned)grid, kThreads, 0, stream>>>(single, descs, tile_start, total_tiles, c, flip_count);
+    const uint32_t tiles = tiles_of(d);
+    if (tiles == 0) return CAST_OK;
+    if (tiles > kMaxTiles) return CAST_ERR_SHAPE;
+    adams_nm_kernel<M><<<tiles, kThreads, 0, stream>>>(d, c, flip_count);
     CAST_CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CAST_OK;
 }
 
-template <bool MULTI>
-int launch_m(int M, const TensorDesc& single, const TensorDesc* descs, const uint32_t* tile_start,
-             uint32_t total_tiles, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+template <int M>
+int launch_multi_t(const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    switch (M) {
-        case 2:  return launch_t<2, MULTI>(single, descs, tile_start, total_tiles, c, flip_count, stream, 1);
-        case 4:  return launch_t<4, MULTI>(single, descs, tile_start, total_tiles, c, flip_count, stream, 2);
-        case 8:  return launch_t<8, MULTI>(single, descs, tile_start, total_tiles, c, flip_count, stream, 3);
-        case 16: return launch_t<16, MULTI>(single, descs, tile_start, total_tiles, c, flip_count, stream, 4);
-        case 32: return launch_t<32, MULTI>(single, descs, tile_start, total_tiles, c, flip_count, stream, 5);
-    }
-    return CAST_ERR_NM;
+    const uint32_t tiles = p.tile_start[p.n_tensors];
+    if (tiles == 0) return CAST_OK;
+    adams_nm_multi_kernel<M><<<tiles, kThreads, 0, stream>>>(p, c, flip_count);
+    CAST_CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CAST_OK;
 }
 
 }  // namespace
 
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    return launch_m<false>(M, d, nullptr, nullptr, tiles_of(d), c, flip_count, stream);
+    switch (M) {
+        case 2:  return launch_single_t<2>(d, c, flip_count, stream);
+        case 4:  return launch_single_t<4>(d, c, flip_count, stream);
+        case 8:  return launch_single_t<8>(d, c, flip_count, stream);
+        case 16: return launch_single_t<16>(d, c, flip_count, stream);
+        case 32: return launch_single_t<32>(d, c, flip_count, stream);
+    }
+    return CAST_ERR_NM;
 }
 
-int launch_multi(const TensorDesc* d_descs, const uint32_t* d_tile_start, uint32_t total_tiles, int M,
-                 const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    TensorDesc none;
-    std::memset(&none, 0, sizeof none);
-    return launch_m<true>(M, none, d_descs, d_tile_start, total_tiles, c, flip_count, stream);
+    switch (M) {
+        case 2:  return launch_multi_t<2>(p, c, flip_count, stream);
+        case 4:  return launch_multi_t<4>(p, c, flip_count, stream);
+        case 8:  return launch_multi_t<8>(p, c, flip_count, stream);
+        case 16: return launch_multi_t<16>(p, c, flip_count, stream);
+        case 32: return launch_multi_t<32>(p, c, flip_count, stream);
+    }
+    return CAST_ERR_NM;
+}
+
+void fill_hints(MultiParams* p)
+{
+    const uint64_t tiles = p->tile_start[p->n_tensors];
+    uint32_t shift = 0;
+    while (((tiles + (1ull << shift) - 1) >> shift) > (uint64_t)kHintEntries) ++shift;
+    p->hint_shift = shift;
+    const size_t n_hints = (size_t)((tiles + (1ull << shift) - 1) >> shift);
+    size_t k = 0;
+    for (size_t b = 0; b < (size_t)kHintEntries; ++b) {
+        if (b < n_hints) {
+            const uint64_t first = (uint64_t)b << shift;
+            while (first >= p->tile_start[k + 1]) ++k;
+        }
+        p->hint[b] = (uint16_t)k;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -230,10 +215,7 @@ struct Plan {
     int device;
     int N, M;
     int n_tensors;
-    uint32_t total_tiles;
-    void* d_table;                // [n_tensors] TensorDesc, then [n_tensors + 1] uint32 tile starts
-    const TensorDesc* d_descs;
-    const uint32_t* d_tile_start;
+    std::vector<MultiParams> launches;   // one table per launch of up to kMaxLaunchTensors matrices
 };
 }  // namespace
 
@@ -273,20 +255,12 @@ extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int
     // the encoding flag is a per-step choice; here only N:M itself is checked
     if ((rc = check_nm_flags(N, M, CAST_F_META_BITMASK, nullptr)) != CAST_OK) return rc;
 
-    std::vector<TensorDesc> descs((size_t)n_tensors);
-    std::vector<uint32_t> tile_start((size_t)n_tensors + 1);
-    uint64_t tiles = 0;
     for (int i = 0; i < n_tensors; ++i) {
         const cast_tensor_t& t = tensors[i];
         if (!t.w || !t.m || !t.v || !t.g || !t.w_fwd || !t.meta) return CAST_ERR_NULL;
         if ((rc = check_shape(t.rows, t.cols, M, t.scale != nullptr, t.scale_groups)) != CAST_OK) return rc;
         if ((rc = check_pointers(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols)) != CAST_OK) return rc;
-        descs[(size_t)i] = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols);
-        tile_start[(size_t)i] = (uint32_t)tiles;
-        tiles += tiles_of(descs[(size_t)i]);
-        if (tiles >= 0xFFFFFFFFull) return CAST_ERR_SHAPE;
     }
-    tile_start[(size_t)n_tensors] = (uint32_t)tiles;
     for (int i = 0; i < n_tensors; ++i) {
         const cast_tensor_t& t = tensors[i];
         const void* ptrs[7] = {t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale};
@@ -295,22 +269,36 @@ extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int
 
     Plan* p = new (std::nothrow) Plan;
     if (!p) return CAST_ERR_PLAN;
-    std::memset(p, 0, sizeof *p);
+    p->magic = 0;
     cudaError_t e = cudaGetDevice(&p->device);
     if (e != cudaSuccess) { delete p; return cuda_failed(e); }
-    const size_t desc_bytes = sizeof(TensorDesc) * (size_t)n_tensors;
-    const size_t start_bytes = sizeof(uint32_t) * ((size_t)n_tensors + 1);
-    e = cudaMalloc(&p->d_table, desc_bytes + start_bytes);
-    if (e != cudaSuccess) { delete p; return cuda_failed(e); }
-    e = cudaMemcpy(p->d_table, descs.data(), desc_bytes, cudaMemcpyHostToDevice);
-    if (e == cudaSuccess)
-        e = cudaMemcpy((char*)p->d_table + desc_bytes, tile_start.data(), start_bytes, cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) { cudaFree(p->d_table); delete p; return cuda_failed(e); }
+    // cut the list into launches: at most kMaxLaunchTensors matrices and kMaxTiles tiles each
+    try {
+        int i = 0;
+        while (i < n_tensors) {
+            p->launches.emplace_back();
+            MultiParams& mp = p->launches.back();
+            std::memset(&mp, 0, sizeof mp);
+            uint64_t tiles = 0;
+            while (i < n_tensors && mp.n_tensors < (uint32_t)kMaxLaunchTensors) {
+                const cast_tensor_t& t = tensors[i];
+                const TensorDesc d = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols);
+                if (tiles + tiles_of(d) > kMaxTiles) break;      // a single matrix always fits (rows*cols < 2^31)
+                mp.desc[mp.n_tensors] = d;
+                mp.tile_start[mp.n_tensors] = (uint32_t)tiles;
+                tiles += tiles_of(d);
+                ++mp.n_tensors;
+                ++i;
+            }
+            mp.tile_start[mp.n_tensors] = (uint32_t)tiles;
+            fill_hints(&mp);
+        }
+    } catch (const std::bad_alloc&) {
+        delete p;
+        return CAST_ERR_PLAN;
+    }
     p->magic = kPlanMagic;
     p->N = N; p->M = M; p->n_tensors = n_tensors;
-    p->total_tiles = (uint32_t)tiles;
-    p->d_descs = (const TensorDesc*)p->d_table;
-    p->d_tile_start = (const uint32_t*)((char*)p->d_table + desc_bytes);
     *plan_out = p;
     return CAST_OK;
 }
@@ -332,7 +320,9 @@ extern "C" int cast_plan_step(void* plan, const cast_hyper_t* h, unsigned long l
         const void* fp[1] = {flip_count};
         if ((rc = check_device_memory(fp, 1)) != CAST_OK) return rc;
     }
-    return launch_multi(p->d_descs, p->d_tile_start, p->total_tiles, p->M, c, flip_count, (cudaStream_t)stream);
+    for (const MultiParams& mp : p->launches)
+        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream)) != CAST_OK) return rc;
+    return CAST_OK;
 }
 
 extern "C" int cast_plan_destroy(void* plan)
@@ -340,9 +330,7 @@ extern "C" int cast_plan_destroy(void* plan)
     Plan* p = (Plan*)plan;
     if (!p || p->magic != kPlanMagic) return CAST_ERR_PLAN;
     p->magic = 0;
-    cudaError_t e = cudaFree(p->d_table);
     delete p;
-    if (e != cudaSuccess) return cuda_failed(e);
     return CAST_OK;
 }
 

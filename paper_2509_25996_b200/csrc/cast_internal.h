@@ -41,10 +41,15 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
 
 inline uint32_t tiles_of(const TensorDesc& d) { return (d.n_units + kTileUnits - 1) / kTileUnits; }
 
-// Launch over one matrix (descriptor passed by value) or over a device table of matrices.
+// Launch over one matrix or over a table of matrices (both passed by value as kernel parameters).
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count,
                   cudaStream_t stream);
-int launch_multi(const TensorDesc* d_descs, const uint32_t* d_tile_start, uint32_t total_tiles, int M,
-                 const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
+int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
+
+// Fill hint_shift and hint[] of a table whose n_tensors and tile_start[] are set.
+void fill_hints(MultiParams* p);
+
+// A grid holds at most this many tiles (one CTA per tile, gridDim.x < 2^31).
+constexpr uint64_t kMaxTiles = 0x7FFFFFFFull;
 
 }  // namespace cast

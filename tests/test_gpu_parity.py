@@ -33,7 +33,7 @@ def inputs(rows, cols, seed=0, idx=0, scale_mode="jitter"):
 @pytest.mark.parametrize("N,M", NM_ALL)
 @pytest.mark.parametrize("rows,cols", [(1, 32), (3, 64), (5, 96), (7, 2080)])
 def test_small_shapes_every_nm(N, M, rows, cols):
-    """1 x 32 up to 7 x 2080 (7.1 tiles of 2048 parameters: several tiles and a ragged tail)."""
+    """1 x 32 up to 7 x 2080 (14.2 tiles of 1024 parameters: several tiles and a ragged tail)."""
     inp = inputs(rows, cols, seed=1, idx=N * 100 + M)
     if inp.scale is not None and (cols // 2) % max(M, 8) != 0:
         inp.scale = None
@@ -116,7 +116,7 @@ def test_general_nm_flip_count():
 
 
 def test_single_matrix_3072x768_full():
-    """The one-matrix workload in full (2,359,296 parameters, 1152 tiles)."""
+    """The one-matrix workload in full (2,359,296 parameters, 2304 tiles)."""
     w = workloads.workload("opt125m_fc2")
     rows, cols = w.shapes[0]
     inp = workloads.gen_tensor_inputs(rows, cols, seed=0, tensor_index=0, device=DEV, scale_mode="jitter")

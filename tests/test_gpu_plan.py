@@ -15,7 +15,7 @@ DEV = "cuda:0"
 RS, BM = B.CAST_F_RESELECT, B.CAST_F_META_BITMASK
 
 
-def run_plan(inputs_list, N, M, hyper: Hyper, flags, metas=None):
+def run_plan(inputs_list, N, M, hyper: Hyper, flags, metas=None, launches=1):
     states = [U.to_device(inp, DEV, None if metas is None else metas[i]) for i, inp in enumerate(inputs_list)]
     tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale,
                              1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in states]
@@ -27,14 +27,14 @@ def run_plan(inputs_list, N, M, hyper: Hyper, flags, metas=None):
     cast.check(cast.cast_plan_step(plan, B.make_hyper(lr, b1, b2, eps, lam, hyper.step, hyper.total_steps, flags),
                                    flips, torch.cuda.current_stream()))
     torch.cuda.synchronize()
-    assert cast.cast_kernel_launch_count() == before + 1          # one grid covers every matrix
+    assert cast.cast_kernel_launch_count() == before + launches   # one grid covers up to 384 matrices
     cast.check(cast.cast_plan_destroy(plan))
     assert all(s.all_intact() for s in states)
     return [U.device_outputs(s) for s in states], (None if flips is None else int(flips.item()))
 
 
 def test_plan_mixed_shapes_ragged_tiles():
-    """Matrices of 0.02 to 33 tiles, most with a ragged last tile, some without a scale tensor."""
+    """Matrices of 0.03 to 66 tiles, most with a ragged last tile, some without a scale tensor."""
     shapes = [(1, 32), (3, 96), (64, 1056), (7, 2080), (1, 2048), (33, 2048), (5, 416), (2, 64), (40, 800)]
     ins = [workloads.gen_tensor_inputs(r, c, seed=20, tensor_index=i, device="cpu",
                                        scale_mode=("none" if i % 3 == 0 else "jitter")) for i, (r, c) in enumerate(shapes)]
@@ -46,6 +46,31 @@ def test_plan_mixed_shapes_ragged_tiles():
     total = 0
     for i, inp in enumerate(ins):
         ref = U.run_oracle(inp, 2, 4, h, fl, meta_in=prev[i])
+        U.assert_parity(got[i], ref, f"tensor {i} {shapes[i]}")
+        total += ref["flips"]
+    assert flips == total
+
+
+def test_plan_many_small_matrices_around_a_large_one():
+    """More than 256 tiles in total, so one entry of the tile-to-matrix hint table covers several tiles,
+    and dozens of one-tile matrices share an entry: the forward walk from the hint takes many steps."""
+    shapes = [(1, 32)] * 37 + [(4096, 2304)] + [(1, 64)] * 5 + [(2, 1024)] + [(1, 32)] * 3
+    ins = [workloads.gen_tensor_inputs(r, c, seed=24, tensor_index=i, scale_mode=("none" if c < 64 else "jitter"))
+           for i, (r, c) in enumerate(shapes)]
+    got, _ = run_plan(ins, 2, 4, Hyper(), RS)
+    for i, inp in enumerate(ins):
+        U.assert_parity(got[i], U.run_oracle(inp, 2, 4, Hyper(), RS), f"tensor {i} {shapes[i]}")
+
+
+def test_plan_more_matrices_than_one_launch_holds():
+    """A launch carries the descriptors of at most 384 matrices: 400 small matrices take two launches."""
+    shapes = [(1 + i % 3, 32 * (1 + i % 5)) for i in range(400)]
+    ins = [workloads.gen_tensor_inputs(r, c, seed=25, tensor_index=i, scale_mode="none") for i, (r, c) in enumerate(shapes)]
+    fl = RS | B.CAST_F_COUNT_FLIPS
+    got, flips = run_plan(ins, 2, 4, Hyper(), fl, launches=2)
+    total = 0
+    for i, inp in enumerate(ins):
+        ref = U.run_oracle(inp, 2, 4, Hyper(), fl)
         U.assert_parity(got[i], ref, f"tensor {i} {shapes[i]}")
         total += ref["flips"]
     assert flips == total
