@@ -132,16 +132,18 @@ typedef struct cast_hyper {
 
 /*
  * Multi-tensor plan: the AdamS iteration of Alg. 1 over "each parameter theta in Theta", i.e. over
- * every prunable matrix of the model, in ONE kernel launch.
+ * every prunable matrix of the model, in ONE kernel launch per 384 matrices.
  *
- * cast_plan_create  validates `n_tensors` descriptors (host array, copied), uploads a descriptor table
- *                   to the current device (one allocation, one blocking copy) and returns an opaque
- *                   handle in *plan_out.  All matrices share N:M.  The buffers named by the descriptors
- *                   stay owned by the caller and must outlive the plan's use.
- * cast_plan_step    launches one grid over all matrices on `stream`; arguments as cast_adams_step.
- *                   The plan may be stepped any number of times, on any stream of its device; two
- *                   steps of one plan must not overlap in time (they update the same state).
- * cast_plan_destroy frees the table.  The caller makes sure no step is still running.
+ * cast_plan_create  validates `n_tensors` descriptors (host array, copied) and returns an opaque handle
+ *                   in *plan_out.  The plan is host memory only: it holds the launch tables, which travel
+ *                   to the device as kernel parameters at every step, and allocates nothing on the
+ *                   device.  All matrices share N:M.  The buffers named by the descriptors stay owned by
+ *                   the caller and must outlive the plan's use.
+ * cast_plan_step    launches one grid over all matrices on `stream` (ceil(n_tensors / 384) grids for
+ *                   larger lists); arguments as cast_adams_step.  The plan may be stepped any number of
+ *                   times, on any stream of its device; two steps of one plan must not overlap in time
+ *                   (they update the same state).
+ * cast_plan_destroy frees the handle (no device work).
  */
 CAST_API int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out);
 CAST_API int cast_plan_step(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,

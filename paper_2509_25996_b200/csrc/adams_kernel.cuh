@@ -3,14 +3,20 @@
 // Streaming kernel, HBM-bound: 14 B read and 14.125 B written per parameter.  One thread owns
 // a "unit" of 8 consecutive columns (32 B of each fp32 array, 16 B of each bf16 array, one
 // metadata byte), so every group of M <= 8 columns lives in one thread's registers and the
-// top-N selection is a register-only rank network; groups of 16 or 32 columns are shared by 2
-// or 4 neighbouring lanes through warp shuffles.  A warp covers 256 consecutive parameters:
+// top-N selection is a register-only comparison network; groups of 16 or 32 columns are shared
+// by 2 or 4 neighbouring lanes through warp shuffles.  A warp covers 256 consecutive parameters:
 // 1 KB of each fp32 array, 512 B of each bf16 array and one 32-byte sector of metadata.
 //
 // Launch shape: one CTA of 128 threads per tile of 1024 parameters, one unit per thread, no loop.
 // Measured on B200, small short-lived CTAs (7 resident per SM, the hardware scheduler handing out
 // tiles in address order) stream faster than a persistent grid-stride loop of the same body or a
 // bulk-copy/mbarrier ring through shared memory, and as fast with 128-bit as with 256-bit accesses.
+//
+// Instruction budget: at ~6.8 TB/s an SM retires ~0.85 parameters per clock, so the body has to stay
+// well under ~100 thread instructions per parameter or instruction issue (and, under the board's
+// power cap, the SM clock) becomes the limit.  Hence: flags are compile-time constants in the two
+// common modes, the 2:4 selection is six comparisons and four 3-input predicate functions per group,
+// and the update uses the approximate reciprocal and square root units (error analysis below).
 #pragma once
 
 #include <cuda_runtime.h>
@@ -29,6 +35,11 @@ constexpr uint32_t kCountFlips = 1u << 1;
 constexpr uint32_t kMetaBitmask = 1u << 2;
 constexpr uint32_t kVKeptFromG = 1u << 3;
 constexpr uint32_t kEmitDense = 1u << 4;
+
+// Kernel modes: the flag word is a compile-time constant in the two common cases.
+constexpr int kModeGeneric = 0;        // any flags, read from StepConsts at run time
+constexpr int kModeSelectIdx = 1;      // flags == kReselect, 2:4, index-form metadata
+constexpr int kModeSelectMask = 2;     // flags == kReselect | kMetaBitmask, any N:M
 
 // One matrix as the kernel sees it.
 struct TensorDesc {
@@ -63,30 +74,46 @@ struct StepConsts {
 __device__ __forceinline__ float4 ld_f4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 __device__ __forceinline__ void st_f4(float* p, float4 x) { *reinterpret_cast<float4*>(p) = x; }
 
-// Keep mask (bit j = column j of the unit is kept) of the groups held by this thread.
-// Order inside a group: larger |w| first, lower column first among equal magnitudes (Eq. 6 with
-// exactly N kept, Eq. 4).  Magnitudes are compared as integers: for non-NaN floats the bit
-// pattern without the sign orders exactly like the absolute value, and -0 equals +0.
-template <int M>
-__device__ __forceinline__ uint32_t select_keep(const float (&w)[8], int n_keep)
-{
-    uint32_t a[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) a[i] = __float_as_uint(w[i]) & 0x7FFFFFFFu;
+// Approximate units: sqrt.approx.f32 has a maximum relative error of 2^-23 over the positive finite
+// range, rcp.approx.f32 of 1 ulp (PTX ISA).  Neither flushes subnormals in this (non-ftz) form.
+__device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
 
+// |w| as an integer: for non-NaN floats the bit pattern without the sign orders exactly like the
+// absolute value, and -0 equals +0.
+__device__ __forceinline__ uint32_t abs_bits(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
+
+// Order inside a group (Eq. 6 with exactly N kept, Eq. 4): larger |w| first, lower column first
+// among equal magnitudes.  Column j (< k) comes before column k iff a[j] >= a[k].
+
+// 2:4: a column is kept iff at least two of the other three do not come before it.
+__device__ __forceinline__ bool at_least_two(bool x, bool y, bool z) { return (x && y) || (x && z) || (y && z); }
+__device__ __forceinline__ void select_2of4(const uint32_t* a, bool* kept)
+{
+    const bool c01 = a[0] >= a[1], c02 = a[0] >= a[2], c03 = a[0] >= a[3];
+    const bool c12 = a[1] >= a[2], c13 = a[1] >= a[3], c23 = a[2] >= a[3];
+    kept[0] = at_least_two(c01, c02, c03);
+    kept[1] = at_least_two(!c01, c12, c13);
+    kept[2] = at_least_two(!c02, !c12, c23);
+    kept[3] = at_least_two(!c03, !c13, !c23);
+}
+
+// General N:M: rank of a column = how many columns of its group come before it; kept iff rank < N.
+// Returns the keep mask of the unit (bit j = column j of the unit is kept).
+template <int M>
+__device__ __forceinline__ uint32_t select_by_rank(const uint32_t (&a)[8], int n_keep)
+{
     constexpr int G = (M <= 8) ? M : 8;      // columns of one group held by this thread
     int rank[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) rank[i] = 0;
-
-    // pairs inside the thread
 #pragma unroll
     for (int base = 0; base < 8; base += G) {
 #pragma unroll
         for (int j = 0; j < G; ++j) {
 #pragma unroll
             for (int k = j + 1; k < G; ++k) {
-                const bool j_first = a[base + j] >= a[base + k];   // equal: the lower column wins
+                const bool j_first = a[base + j] >= a[base + k];
                 rank[base + k] += j_first ? 1 : 0;
                 rank[base + j] += j_first ? 0 : 1;
             }
@@ -116,24 +143,16 @@ __device__ __forceinline__ uint32_t select_keep(const float (&w)[8], int n_keep)
     return keep;
 }
 
-// 2:4 index form <-> keep bits, one nibble per group.  Table entry k (a 4-bit keep mask with two
-// bits set) holds lo | hi << 2; entries of other masks are unused.
-__device__ __forceinline__ uint32_t idx2_from_keep_nibble(uint32_t k)
+// 2:4 index form: one nibble per group, lo | hi << 2 with lo < hi the positions of the kept pair.
+__device__ __forceinline__ uint32_t idx2_from_kept(const bool* k)
 {
-    // k: 0011->lo0 hi1 = 0x4, 0101->0,2 = 0x8, 0110->1,2 = 0x9, 1001->0,3 = 0xC, 1010->1,3 = 0xD, 1100->2,3 = 0xE
-    constexpr unsigned long long table =
-        (0x4ull << (4 * 0x3)) | (0x8ull << (4 * 0x5)) | (0x9ull << (4 * 0x6)) |
-        (0xCull << (4 * 0x9)) | (0xDull << (4 * 0xA)) | (0xEull << (4 * 0xC));
-    return (uint32_t)(table >> (4 * k)) & 0xFu;
+    const uint32_t lo = k[0] ? 0u : (k[1] ? 1u : 2u);
+    const uint32_t hi = k[3] ? 3u : (k[2] ? 2u : 1u);
+    return lo | (hi << 2);
 }
 __device__ __forceinline__ uint32_t keep_nibble_from_idx2(uint32_t f)
 {
     return (1u << (f & 3u)) | (1u << ((f >> 2) & 3u));
-}
-__device__ __forceinline__ uint32_t meta_byte_from_keep(uint32_t keep, bool bitmask)
-{
-    if (bitmask) return keep;
-    return idx2_from_keep_nibble(keep & 0xFu) | (idx2_from_keep_nibble(keep >> 4) << 4);
 }
 __device__ __forceinline__ uint32_t keep_from_meta_byte(uint32_t b, bool bitmask)
 {
@@ -156,58 +175,92 @@ struct UnitRegs {
     uint32_t meta_byte;    // metadata byte after the step
 };
 
+template <int MODE>
+__device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
+{
+    if constexpr (MODE == kModeSelectIdx) return kReselect;
+    else if constexpr (MODE == kModeSelectMask) return kReselect | kMetaBitmask;
+    else return c.flags;
+}
+
 // Arithmetic of one unit, registers only (and warp shuffles for M > 8: every lane of the warp must
 // call this, lanes without data pass zeros).  `a` is the unit's scale A[r, segment].  Returns the
-// number of flipped mask bits of the unit (App. C: ||M_t - M_{t-1}||_0).
-template <int M>
+// number of flipped mask bits of the unit (App. C: ||M_t - M_{t-1}||_0; 0 unless flips are counted).
+//
+// Precision.  The first moment and the decayed first moment are sums of terms of opposite sign and
+// like size (beta1 m against (1 - beta1) g, (1 - alpha) mu against alpha lambda), so they are formed
+// in fp64 from the exact inputs: in fp32 a cancellation leaves mu with a large relative error, which
+// the quotient mu / sqrt(v) carries into w wherever v is small as well.  Everything after is a
+// product or a sum of like signs and stays in fp32.  The update lr mu^ / (sqrt(v^) + eps) uses the
+// approximate square root and reciprocal: its relative error is below ~5e-7 (2^-23 each, plus five
+// roundings of 2^-24), i.e. below 2.5e-10 absolute for updates up to 5e-4, which is under both the
+// fp32 spacing of typical weights (1.9e-9 at 0.02) and the 1e-9 floor of the accepted error.
+template <int M, int MODE>
 __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a)
 {
-    const bool bitmask = (c.flags & kMetaBitmask) != 0;
-    const uint32_t prev_keep = keep_from_meta_byte(u.prev_byte, bitmask);
-    uint32_t keep;
-    if (c.flags & kReselect) keep = select_keep<M>(u.w, c.n_keep);     // uniform branch: all lanes shuffle
-    else keep = prev_keep;
+    static_assert(MODE != kModeSelectIdx || M == 4, "index-form metadata is 2:4 only");
+    const uint32_t flags = mode_flags<MODE>(c);
+    const bool bitmask = (flags & kMetaBitmask) != 0;
+    uint32_t ab[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) ab[i] = abs_bits(u.w[i]);
+
+    bool kept[8];
+    uint32_t flips = 0;
+    if constexpr (MODE == kModeSelectIdx) {
+        select_2of4(ab, kept);
+        select_2of4(ab + 4, kept + 4);
+        u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+    } else {
+        uint32_t keep;
+        uint32_t prev_keep = 0;
+        if constexpr (MODE == kModeGeneric) prev_keep = keep_from_meta_byte(u.prev_byte, bitmask);
+        if (flags & kReselect) keep = select_by_rank<M>(ab, c.n_keep);     // uniform branch: all lanes shuffle
+        else keep = prev_keep;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+        if (bitmask) u.meta_byte = keep;
+        else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+        if constexpr (MODE == kModeGeneric) flips = (uint32_t)__popc(keep ^ prev_keep);
+    }
 
     const uint32_t gw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
-    const bool v_from_g = (c.flags & kVKeptFromG) != 0;
-    const bool dense = (c.flags & kEmitDense) != 0;
+    const bool v_from_g = (flags & kVKeptFromG) != 0;
+    const bool dense = (flags & kEmitDense) != 0;
+    const int sign_hi = __double2hiint(c.c_sign), sign_lo = __double2loint(c.c_sign);
     float fwd[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const float g32 = __uint_as_float((i & 1) ? (gw[i >> 1] & 0xFFFF0000u) : (gw[i >> 1] << 16));
-        const bool kept = (keep >> i) & 1u;
-        // First moment, stored undecayed (Alg. 1), and the proportional L1 decay outside the kept set
-        // (Eq. 7; Sign(0) = 0).  Both are sums of terms of opposite sign and like size (beta1 m against
-        // (1 - beta1) g, (1 - alpha) mu against alpha lambda), so they are formed in fp64 from the exact
-        // inputs: in fp32 a cancellation leaves mu with a large relative error, which the quotient
-        // mu / sqrt(v) carries into w wherever v is small as well.  Everything after is a product or a
-        // sum of like signs and stays in fp32.
+        // first moment, stored undecayed (Alg. 1)
         const double mu = fma(c.beta1, (double)u.m[i], c.omb1 * (double)g32);
-        u.m[i] = (float)mu;
-        const double sgn_term = (u.w[i] == 0.0f) ? 0.0 : copysign(c.c_sign, (double)u.w[i]);
-        const float mu_t = (float)(kept ? mu : fma(c.c_mu, mu, sgn_term));
+        const float mu_f = (float)mu;
+        u.m[i] = mu_f;
+        // proportional L1 decay outside the kept set (Eq. 7): alpha lambda Sign(w), Sign(+-0) = 0
+        const bool w_zero = ab[i] == 0u;
+        const double sgn_term = __hiloint2double(w_zero ? 0 : (sign_hi | (int)(__float_as_uint(u.w[i]) & 0x80000000u)),
+                                                 w_zero ? 0 : sign_lo);
+        const float mu_t = kept[i] ? mu_f : (float)fma(c.c_mu, mu, sgn_term);
         // second moment from the decayed first moment (Eq. 8)
-        const float src = (v_from_g && kept) ? g32 : mu_t;
+        const float src = (v_from_g && kept[i]) ? g32 : mu_t;
         const float vn = fmaf(c.beta2, u.v[i], (c.omb2 * src) * src);
         u.v[i] = vn;
-        // bias-corrected update
-        const float denom = sqrtf(vn * c.inv_bc2) + c.eps;
-        const float wn = u.w[i] - (c.lr_bc1 * mu_t) / denom;
+        // bias-corrected update (Alg. 1): w - (lr / bc1) mu~ / (sqrt(v / bc2) + eps)
+        const float wn = fmaf(-(c.lr_bc1 * mu_t), rcp_approx(sqrt_approx(vn * c.inv_bc2) + c.eps), u.w[i]);
         u.w[i] = wn;
         // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for
-        fwd[i] = (kept || dense) ? a * wn : 0.0f;
+        fwd[i] = (kept[i] || dense) ? a * wn : 0.0f;
     }
     u.g.x = pack_bf16x2(fwd[0], fwd[1]);
     u.g.y = pack_bf16x2(fwd[2], fwd[3]);
     u.g.z = pack_bf16x2(fwd[4], fwd[5]);
     u.g.w = pack_bf16x2(fwd[6], fwd[7]);
-    u.meta_byte = meta_byte_from_keep(keep, bitmask);
-    return (uint32_t)__popc(keep ^ prev_keep);
+    return flips;
 }
 
 // The whole per-unit body: loads, arithmetic, stores.
 // `active` is false for threads past the end of the matrix; they take part in the shuffles only.
-template <int M>
+template <int M, int MODE>
 __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const StepConsts& c,
                                                  uint32_t unit, bool active)
 {
@@ -215,7 +268,8 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
     u.g = make_uint4(0, 0, 0, 0);
     u.prev_byte = 0;
     const size_t e = (size_t)unit * kUnitElems;
-    const bool need_prev = ((c.flags & kReselect) == 0) || (c.flags & kCountFlips);
+    const uint32_t flags = mode_flags<MODE>(c);
+    const bool need_prev = ((flags & kReselect) == 0) || (flags & kCountFlips);
     float a = 1.0f;
 
     if (active) {
@@ -236,7 +290,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         for (int i = 0; i < 8; ++i) { u.w[i] = 0.f; u.m[i] = 0.f; u.v[i] = 0.f; }
     }
 
-    const uint32_t flips = compute_unit<M>(u, c, a);
+    const uint32_t flips = compute_unit<M, MODE>(u, c, a);
 
     if (active) {
         st_f4(t.w + e, make_float4(u.w[0], u.w[1], u.w[2], u.w[3]));
@@ -287,18 +341,19 @@ __device__ __forceinline__ void add_flips(uint32_t flips, unsigned long long* fl
 #define CAST_LAUNCH_BOUNDS(M) __launch_bounds__(kThreads, ((M) <= 8) ? kMinCtasPerSm : 5)
 
 // One matrix: CTA b handles tile b.
-template <int M>
+template <int M, int MODE>
 __global__ void CAST_LAUNCH_BOUNDS(M)
 adams_nm_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c,
                 unsigned long long* __restrict__ flip_count)
 {
     const uint32_t unit = blockIdx.x * kTileUnits + threadIdx.x;
-    const uint32_t flips = process_unit<M>(t, c, unit, unit < t.n_units);
-    if (c.flags & kCountFlips) add_flips(flips, flip_count);
+    const uint32_t flips = process_unit<M, MODE>(t, c, unit, unit < t.n_units);
+    if constexpr (MODE == kModeGeneric)
+        if (c.flags & kCountFlips) add_flips(flips, flip_count);
 }
 
 // Up to kMaxLaunchTensors matrices in one grid: CTA b handles tile b of the concatenated index space.
-template <int M>
+template <int M, int MODE>
 __global__ void CAST_LAUNCH_BOUNDS(M)
 adams_nm_multi_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
                       unsigned long long* __restrict__ flip_count)
@@ -308,8 +363,9 @@ adams_nm_multi_kernel(const __grid_constant__ MultiParams p, const __grid_consta
     while (tile >= p.tile_start[k + 1]) ++k;
     const TensorDesc& t = p.desc[k];
     const uint32_t unit = (tile - p.tile_start[k]) * kTileUnits + threadIdx.x;
-    const uint32_t flips = process_unit<M>(t, c, unit, unit < t.n_units);
-    if (c.flags & kCountFlips) add_flips(flips, flip_count);
+    const uint32_t flips = process_unit<M, MODE>(t, c, unit, unit < t.n_units);
+    if constexpr (MODE == kModeGeneric)
+        if (c.flags & kCountFlips) add_flips(flips, flip_count);
 }
 
 }  // namespace cast

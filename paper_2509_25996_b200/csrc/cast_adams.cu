@@ -139,27 +139,60 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
 
 namespace {
 
-template <int M>
+// The flag word is a compile-time constant of the kernel in the two common cases.
+int mode_of(const StepConsts& c, int M)
+{
+    if (c.flags == kReselect && M == 4 && c.n_keep == 2) return kModeSelectIdx;
+    if (c.flags == (kReselect | kMetaBitmask)) return kModeSelectMask;
+    return kModeGeneric;
+}
+
+template <int M, int MODE>
 int launch_single_t(const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
     const uint32_t tiles = tiles_of(d);
     if (tiles == 0) return CAST_OK;
     if (tiles > kMaxTiles) return CAST_ERR_SHAPE;
-    adams_nm_kernel<M><<<tiles, kThreads, 0, stream>>>(d, c, flip_count);
+    // one CTA per tile: the hardware scheduler hands tiles out in address order
+    adams_nm_kernel<M, MODE><<<tiles, kThreads, 0, stream>>>(d, c, flip_count);
+    CAST_CUDA_TRY(cudaGetLastError());
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return CAST_OK;
+}
+
+template <int M, int MODE>
+int launch_multi_t(const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+{
+    const uint32_t tiles = p.tile_start[p.n_tensors];
+    if (tiles == 0) return CAST_OK;
+    adams_nm_multi_kernel<M, MODE><<<tiles, kThreads, 0, stream>>>(p, c, flip_count);
     CAST_CUDA_TRY(cudaGetLastError());
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return CAST_OK;
 }
 
 template <int M>
-int launch_multi_t(const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+int launch_single_m(const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    const uint32_t tiles = p.tile_start[p.n_tensors];
-    if (tiles == 0) return CAST_OK;
-    adams_nm_multi_kernel<M><<<tiles, kThreads, 0, stream>>>(p, c, flip_count);
-    CAST_CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return CAST_OK;
+    switch (mode_of(c, M)) {
+        case kModeSelectIdx:
+            if constexpr (M == 4) return launch_single_t<4, kModeSelectIdx>(d, c, flip_count, stream);
+            break;
+        case kModeSelectMask: return launch_single_t<M, kModeSelectMask>(d, c, flip_count, stream);
+    }
+    return launch_single_t<M, kModeGeneric>(d, c, flip_count, stream);
+}
+
+template <int M>
+int launch_multi_m(const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+{
+    switch (mode_of(c, M)) {
+        case kModeSelectIdx:
+            if constexpr (M == 4) return launch_multi_t<4, kModeSelectIdx>(p, c, flip_count, stream);
+            break;
+        case kModeSelectMask: return launch_multi_t<M, kModeSelectMask>(p, c, flip_count, stream);
+    }
+    return launch_multi_t<M, kModeGeneric>(p, c, flip_count, stream);
 }
 
 }  // namespace
@@ -167,11 +200,11 @@ int launch_multi_t(const MultiParams& p, const StepConsts& c, unsigned long long
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
     switch (M) {
-        case 2:  return launch_single_t<2>(d, c, flip_count, stream);
-        case 4:  return launch_single_t<4>(d, c, flip_count, stream);
-        case 8:  return launch_single_t<8>(d, c, flip_count, stream);
-        case 16: return launch_single_t<16>(d, c, flip_count, stream);
-        case 32: return launch_single_t<32>(d, c, flip_count, stream);
+        case 2:  return launch_single_m<2>(d, c, flip_count, stream);
+        case 4:  return launch_single_m<4>(d, c, flip_count, stream);
+        case 8:  return launch_single_m<8>(d, c, flip_count, stream);
+        case 16: return launch_single_m<16>(d, c, flip_count, stream);
+        case 32: return launch_single_m<32>(d, c, flip_count, stream);
     }
     return CAST_ERR_NM;
 }
@@ -179,11 +212,11 @@ int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
     switch (M) {
-        case 2:  return launch_multi_t<2>(p, c, flip_count, stream);
-        case 4:  return launch_multi_t<4>(p, c, flip_count, stream);
-        case 8:  return launch_multi_t<8>(p, c, flip_count, stream);
-        case 16: return launch_multi_t<16>(p, c, flip_count, stream);
-        case 32: return launch_multi_t<32>(p, c, flip_count, stream);
+        case 2:  return launch_multi_m<2>(p, c, flip_count, stream);
+        case 4:  return launch_multi_m<4>(p, c, flip_count, stream);
+        case 8:  return launch_multi_m<8>(p, c, flip_count, stream);
+        case 16: return launch_multi_m<16>(p, c, flip_count, stream);
+        case 32: return launch_multi_m<32>(p, c, flip_count, stream);
     }
     return CAST_ERR_NM;
 }
