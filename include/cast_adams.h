@@ -179,6 +179,40 @@ CAST_API int cast_host_step(void* ctx,
 CAST_API int cast_host_ctx_sync(void* ctx);
 CAST_API int cast_host_ctx_destroy(void* ctx);
 
+/*
+ * cast_host_step_static -- cast_host_step for callers that must not allocate device memory.
+ * (The paper has no counterpart to this entry point: it is a packaging variant of the call above.)
+ *
+ * cast_host_ctx_create reserves its staging slots with cudaMalloc.  A caller whose framework allocator
+ * already owns all device memory, that cannot afford the device-wide synchronisation an allocation or a
+ * free implies, or that may not grow its device footprint after start-up, uses this call instead: the
+ * staging area is a fixed array inside the library image (about 16.6 MiB, held by every GPU on which the
+ * process uses the library, until the process exits), and the call allocates and frees nothing, on the
+ * device or through any other library.
+ *
+ *   Arguments as cast_host_step (every data pointer is a HOST pointer; flip_count is a host counter that
+ *   is added to), plus `stream`, on which the copies and the kernel are queued.
+ *   Limit: rows * cols <= CAST_STATIC_MAX_PARAMS; a larger matrix is refused with CAST_ERR_PLAN (the
+ *   staging area is too small) and nothing is queued.  Cut larger matrices into blocks of whole rows.
+ *   The call is synchronous: it returns after `stream` has finished the step, with the results in the
+ *   host buffers.
+ *   The first call on each device looks up the device address of the staging area (with that device
+ *   current); make that first call outside any stream capture.
+ *   All calls of a process on one device share the one staging area, which keeps the contents the
+ *   previous call left (the call clears the only part that must start at zero, its flip counter).
+ *   Two calls that overlap in time on the same device -- from two host threads, on the same or different
+ *   streams -- race on it and corrupt each other's results: serialise them.
+ */
+#define CAST_STATIC_MAX_PARAMS 1048576
+CAST_API int cast_host_step_static(float* w, float* m, float* v, const cast_bf16* g,
+                   cast_bf16* w_fwd_bf16, uint32_t* meta,
+                   const float* scale, int scale_groups,
+                   int64_t rows, int64_t cols, int N, int M,
+                   float lr, float beta1, float beta2, float eps, float l1_coeff,
+                   int64_t step, int64_t total_steps,
+                   uint32_t flags, unsigned long long* flip_count,
+                   cast_stream_t stream);
+
 /* Static description of a status code (never NULL). */
 CAST_API const char* cast_strerror(int status);
 

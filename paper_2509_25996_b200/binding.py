@@ -36,6 +36,7 @@ CAST_F_EMIT_DENSE = 1 << 4
 EXPORTS = (
     "cast_adams_step", "cast_plan_create", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
+    "cast_host_step_static",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
 )
 
@@ -99,6 +100,8 @@ def load_library() -> ctypes.CDLL:
     lib.cast_host_ctx_create.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.POINTER(ctypes.c_void_p)]
     lib.cast_host_step.restype = ctypes.c_int
     lib.cast_host_step.argtypes = [ctypes.c_void_p] + _STEP_ARGS
+    lib.cast_host_step_static.restype = ctypes.c_int
+    lib.cast_host_step_static.argtypes = _STEP_ARGS + [ctypes.c_void_p]
     lib.cast_host_ctx_sync.restype = ctypes.c_int
     lib.cast_host_ctx_sync.argtypes = [ctypes.c_void_p]
     lib.cast_host_ctx_destroy.restype = ctypes.c_int
@@ -201,6 +204,19 @@ def cast_host_step(ctx, w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows,
         ctx, _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
         int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
         int(flags), _ptr(flip_count))
+
+
+CAST_STATIC_MAX_PARAMS = 1048576
+
+
+def cast_host_step_static(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols, N, M,
+                          lr, beta1, beta2, eps, l1_coeff, step, total_steps, flags, flip_count=None, stream=None) -> int:
+    """cast_host_step through the staging area built into the library: host pointers in and out, no device
+    allocation by the call, at most CAST_STATIC_MAX_PARAMS parameters, synchronous on `stream`."""
+    return load_library().cast_host_step_static(
+        _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
+        int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
+        int(flags), _ptr(flip_count), _stream(stream))
 
 
 def cast_host_ctx_sync(ctx) -> int:
