@@ -208,7 +208,7 @@ def cuda_arm(args):
     import paper_2509_25996_b200 as cast
     from paper_2509_25996_b200 import binding as B
     from paper_2509_25996_b200 import workloads
-    from paper_2509_25996_b200.runner import DeviceModelState, Hyper
+    from paper_2509_25996_b200.runner import DeviceModelState, StreamedModelState, Hyper
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -224,26 +224,36 @@ def cuda_arm(args):
     N, M = (int(x) for x in args.nm.split(":"))
     wl = workloads.workload(args.workload)
     free, total_mem = torch.cuda.mem_get_info()
-    need = wl.n_params * 16.2 + 2e9
-    if need > free:                       # largest single-GPU configuration that fits
+    resident = wl.n_params if not wl.resident_layers else \
+        wl.resident_layers * sum(r * c for r, c in wl.shapes[:wl.layer_matrices])
+    if resident * 16.2 + 2e9 > free:      # largest single-GPU configuration that fits
         wl = workloads.workload("decoder_d768_12l")
     flags = B.CAST_F_RESELECT | (0 if (N, M) == (2, 4) else B.CAST_F_META_BITMASK)
     if args.count_flips:
         flags |= B.CAST_F_COUNT_FLIPS
     bytes_per_param = BYTES_PER_PARAM_FLIPS if args.count_flips else BYTES_PER_PARAM
 
-    state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones")
+    if wl.resident_layers:
+        # per-layer calls alternating on 2 streams over the resident layer slots (no host traffic)
+        state = StreamedModelState(wl.shapes[:wl.layer_matrices], len(wl.shapes) // wl.layer_matrices, wl.resident_layers, 2,
+                                   N, M, seed=args.seed, device=dev, scale_mode="ones")
+        mats = state.slots[0].mats
+        oracle_repeats = len(wl.shapes) // wl.layer_matrices // wl.resident_layers   # steps a slot takes per pass
+    else:
+        state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones")
+        mats = state.mats
+        oracle_repeats = 1
     hyper = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl.total_steps)
     stream = torch.cuda.current_stream(dev)
 
     # parity sample (checked in the CPU-baseline leg): a few rows of the first and last matrices, copied
     # before the first step and again after it
     sample_rows = 16
-    picks = sorted({0, len(state.mats) // 2, len(state.mats) - 1})
+    picks = sorted({0, len(mats) // 2, len(mats) - 1})
     parity_in = {}
     if rank == 0 and args.cpu_baseline:
         for t in picks:
-            s = state.mats[t]
+            s = mats[t]
             parity_in[t] = dict(w=s.w[:sample_rows].cpu().numpy(), m=s.m[:sample_rows].cpu().numpy(),
                                 v=s.v[:sample_rows].cpu().numpy(), g=workloads.bf16_bits(s.g[:sample_rows]),
                                 scale=s.scale[:sample_rows].cpu().numpy(), rows=sample_rows, cols=s.cols)
@@ -261,7 +271,7 @@ def cuda_arm(args):
         if i == 0 and parity_in:
             torch.cuda.synchronize(dev)
             for t in picks:
-                s = state.mats[t]
+                s = mats[t]
                 parity_out[t] = dict(w=s.w[:sample_rows].cpu().numpy(), m=s.m[:sample_rows].cpu().numpy(),
                                      v=s.v[:sample_rows].cpu().numpy(), w_fwd=workloads.bf16_bits(s.w_fwd[:sample_rows]),
                                      meta=s.meta[:sample_rows].cpu().numpy().view(np.uint32))
@@ -304,7 +314,7 @@ def cuda_arm(args):
         shapes = list(wl.shapes[:min(len(wl.shapes), per_layer * args.e2e_layers)])
         host = []
         for i, (r, c) in enumerate(shapes):
-            s = state.mats[i]
+            s = mats[i]
             host.append(dict(w=s.w.cpu().pin_memory(), m=s.m.cpu().pin_memory(), v=s.v.cpu().pin_memory(),
                              g=s.g.cpu().pin_memory(), scale=s.scale.cpu().pin_memory(),
                              fwd=torch.empty((r, c), dtype=torch.bfloat16).pin_memory(),
@@ -361,7 +371,8 @@ def cuda_arm(args):
         ok = bool(parity_out)
         for t in (picks if parity_out else []):
             a = parity_in[t]
-            _, outs = time_oracle([a], N, M, oh, o_flags, 1)
+            for _ in range(oracle_repeats):
+                _, outs = time_oracle([a], N, M, oh, o_flags, 1)
             ref, got = outs[0], parity_out[t]
             for k in ("w", "m", "v"):
                 r = ref[k].astype(np.float64).reshape(-1)
@@ -373,7 +384,7 @@ def cuda_arm(args):
         parity = {"ok": ok, "sample": f"first {sample_rows} rows of matrices {picks} after the first step"}
         # timing sample: whole matrices from the front of the workload, about 2e8 parameters (one LLaMA2-7B layer)
         arrays, n = [], 0
-        for i, s in enumerate(state.mats):
+        for i, s in enumerate(mats):
             if n and n + s.rows * s.cols > 210_000_000:
                 break
             arrays.append(dict(w=s.w.cpu().numpy(), m=s.m.cpu().numpy(), v=s.v.cpu().numpy(), g=workloads.bf16_bits(s.g),
@@ -402,6 +413,7 @@ def cuda_arm(args):
         "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "note": wl.note, "nm": args.nm, "params": wl.n_params, "matrices": len(wl.shapes),
                    "parallelism": "replicas only" if world > 1 else "1 gpu", "l2": "inputs far larger than L2, no flush",
+                   "resident_layers": wl.resident_layers, "streams": 2 if wl.resident_layers else 1,
                    "lr": hyper.lr, "betas": [hyper.beta1, hyper.beta2], "eps": hyper.eps, "l1_coeff": hyper.l1_coeff,
                    "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "seed": args.seed},
         "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
@@ -409,7 +421,10 @@ def cuda_arm(args):
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
                      "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}>",
                      "bytes_per_param": bytes_per_param,
-                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None else NCU_DRAM_BYTES_PER_PARAM * wl.n_params)},
+                     "launches_per_step": launches // args.steps,
+                     "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params * args.steps / max(launches, 1),
+                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None
+                                 else NCU_DRAM_BYTES_PER_PARAM * wl.n_params * args.steps / max(launches, 1))},
         "cpu_baseline": cpu_baseline, "parity": parity,
     }
     if world > 1:

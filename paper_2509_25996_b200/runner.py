@@ -78,3 +78,48 @@ class DeviceModelState:
             self.close()
         except Exception:
             pass
+
+
+class StreamedModelState:
+    """A model too large to keep resident: `n_slots` layers of state stay on the GPU and the `n_layers`
+    layers are stepped one plan call per layer, layer L in slot L mod n_slots, the calls alternating over
+    `n_streams` CUDA streams so that the tail of one layer's grid overlaps the head of the next.
+
+    Two calls on one slot must not overlap (they update the same state): n_slots must be a multiple of
+    n_streams, so that a slot is always stepped on the same stream and its calls are ordered by it."""
+
+    def __init__(self, layer_shapes: Sequence[Tuple[int, int]], n_layers: int, n_slots: int, n_streams: int = 2,
+                 N: int = 2, M: int = 4, seed: int = 0, device="cuda:0", scale_mode: str = "ones"):
+        if n_slots % n_streams != 0:
+            raise ValueError("n_slots must be a multiple of n_streams")
+        self.device = torch.device(device)
+        self.n_layers = n_layers
+        per_layer = len(layer_shapes)
+        self.slots = [DeviceModelState(layer_shapes, N, M, seed=seed, device=device, scale_mode=scale_mode,
+                                       first_tensor_index=i * per_layer) for i in range(min(n_slots, n_layers))]
+        self.streams = [torch.cuda.Stream(device=self.device) for _ in range(n_streams)]
+        self.n_params = n_layers * self.slots[0].n_params
+        self._done = [torch.cuda.Event() for _ in range(n_streams)]
+
+    def step(self, hyper: Hyper, flags: int, stream=None) -> None:
+        """One AdamS iteration over all layers.  Work is ordered after what `stream` (default: the current
+        stream) has queued so far, and `stream` waits for it at the end, so the caller can bracket steps with
+        events on that one stream."""
+        cur = stream if stream is not None else torch.cuda.current_stream(self.device)
+        start = torch.cuda.Event()
+        start.record(cur)
+        for s in self.streams:
+            s.wait_event(start)
+        for layer in range(self.n_layers):
+            self.slots[layer % len(self.slots)].step(hyper, flags, self.streams[layer % len(self.streams)])
+        for s, ev in zip(self.streams, self._done):
+            ev.record(s)
+            cur.wait_event(ev)
+
+    @property
+    def flips(self) -> torch.Tensor:
+        return sum(s.flips for s in self.slots)
+
+    def close(self) -> None:
+        for s in self.slots:
+            s.close()

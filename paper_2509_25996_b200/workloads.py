@@ -43,6 +43,9 @@ class Workload:
     shapes: Tuple[Shape, ...]
     total_steps: int              # T of alpha_t = t/T (Table 11 step counts)
     note: str = ""
+    layer_matrices: int = 0       # matrices per decoder layer (0: not a layered workload)
+    resident_layers: int = 0      # > 0: only this many layers of state are resident; the layers are stepped
+                                  # one call per layer, layer L in slot L mod resident_layers
 
     @property
     def n_params(self) -> int:
@@ -66,7 +69,8 @@ def workload(name: str) -> Workload:
                         "1 layer of LLaMA2-13B, 7 matrices")
     if name == "llama2_13b":
         return Workload(name, tuple(decoder_linear_shapes(40, 5120, 13824, gated=True)), 7500,
-                        "40 layers, d=5120, ffn=13824, 280 matrices")
+                        "40 layers, d=5120, ffn=13824, 280 matrices; per-layer calls on 2 streams over 10 resident layer slots",
+                        layer_matrices=7, resident_layers=10)
     raise KeyError(name)
 
 

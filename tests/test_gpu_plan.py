@@ -101,6 +101,34 @@ def test_plan_decoder_d768_12_layers_full():
     print(f"near-tie groups: {ties} of {wl.n_params // 4}; mask mismatches: 0")
 
 
+def test_streamed_layers_on_two_streams_match_oracle():
+    """Per-layer plan calls alternating on two streams over fewer resident slots than layers: 6 layers in 4
+    slots, so slots 0 and 1 are stepped twice (layers 0, 4 and 1, 5) and slots 2 and 3 once."""
+    from paper_2509_25996_b200.runner import StreamedModelState, Hyper as RunHyper
+    layer_shapes = [(64, 256), (64, 256), (96, 256), (64, 384)]
+    st = StreamedModelState(layer_shapes, n_layers=6, n_slots=4, n_streams=2, N=2, M=4, seed=3, device=DEV,
+                            scale_mode="jitter")
+    before = [[workloads.TensorInputs(m.w.cpu(), m.g.cpu(), m.m.cpu(), m.v.cpu(), m.scale.cpu()) for m in slot.mats]
+              for slot in st.slots]
+    h = RunHyper()
+    launches = cast.cast_kernel_launch_count()
+    st.step(h, RS)
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == launches + 6
+    oh = Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
+    for si, slot in enumerate(st.slots):
+        for mi, mat in enumerate(slot.mats):
+            inp = before[si][mi]
+            for _ in range(2 if si < 2 else 1):
+                ref = U.run_oracle(inp, 2, 4, oh, RS)
+                inp = workloads.TensorInputs(torch.from_numpy(ref["w"]), inp.g, torch.from_numpy(ref["m"]),
+                                             torch.from_numpy(ref["v"]), inp.scale)
+            got = dict(w=mat.w.cpu().numpy(), m=mat.m.cpu().numpy(), v=mat.v.cpu().numpy(),
+                       w_fwd=workloads.bf16_bits(mat.w_fwd), meta=mat.meta.cpu().numpy().view(np.uint32))
+            U.assert_parity(got, ref, f"slot {si} matrix {mi}")
+    st.close()
+
+
 def test_plan_rejects_wrong_device_memory_and_survives():
     inp = workloads.gen_tensor_inputs(4, 64, seed=23)
     s = U.to_device(inp, DEV)
