@@ -39,6 +39,9 @@ def _load():
                 ctypes.c_int64, ctypes.c_int64,                                       # step total_steps
                 ctypes.c_uint32, ctypes.c_void_p,                                     # flags flip_count
             ]
+        lib.oracle_mask_stats.restype = ctypes.c_int
+        lib.oracle_mask_stats.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                          ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -109,3 +112,26 @@ def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELE
     flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision)
     return dict(w=w2.reshape(rows, cols), m=m2.reshape(rows, cols), v=v2.reshape(rows, cols),
                 w_fwd=fwd.reshape(rows, cols), meta=meta.reshape(rows, cols // 32), flips=flips)
+
+
+def mask_stats(w, meta, meta_ref, M: int, bitmask: bool):
+    """Mask statistics of App. C for one matrix: dict(flips = ||M - M_ref||_0 (0 without meta_ref),
+    kept_abs = ||W (.) M||_1, total_abs = ||W||_1), sums in fp64.  w: float32 [rows, cols]; meta, meta_ref:
+    uint32 [rows, cols/32]."""
+    lib = _load()
+    rows, cols = w.shape
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    meta = np.ascontiguousarray(meta, dtype=np.uint32)
+    assert meta.size == rows * cols // 32
+    ref_ptr = None
+    if meta_ref is not None:
+        meta_ref = np.ascontiguousarray(meta_ref, dtype=np.uint32)
+        assert meta_ref.size == meta.size
+        ref_ptr = meta_ref.ctypes.data
+    flips = ctypes.c_uint64(0)
+    sums = (ctypes.c_double * 2)(0.0, 0.0)
+    rc = lib.oracle_mask_stats(w.ctypes.data, meta.ctypes.data, ref_ptr, rows, cols, M, 1 if bitmask else 0,
+                               ctypes.addressof(flips), ctypes.addressof(sums))
+    if rc != 0:
+        raise ValueError("oracle_mask_stats rejected its arguments")
+    return dict(flips=int(flips.value), kept_abs=float(sums[0]), total_abs=float(sums[1]))

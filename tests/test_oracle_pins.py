@@ -432,3 +432,68 @@ def test_masked_weights_shrink_as_alpha_ramps():
         keep = keep_mask_from_meta(meta, cols, 4, True)
         ratios.append(np.abs(w[keep]).sum() / np.abs(w).sum())
     assert ratios[-1] > 0.97 and ratios[-1] > ratios[0] + 0.1
+
+
+# --------------------------------------------------------------------------- mask statistics (App. C)
+
+@pytest.mark.parametrize("N,M,bitmask", [(2, 4, False), (2, 4, True), (4, 8, True), (1, 4, True), (5, 16, True)])
+def test_mask_statistics_match_numpy_on_an_independently_decoded_mask(N, M, bitmask):
+    rng = np.random.default_rng(50 + M)
+    rows, cols = 7, 192
+    enc = orc.F_META_BITMASK if bitmask else 0
+    w = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    w_ref = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    meta = run(w, N=N, M=M, flags=orc.F_RESELECT | enc)["meta"]
+    meta_ref = run(w_ref, N=N, M=M, flags=orc.F_RESELECT | enc)["meta"]
+    w_now = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)     # statistics take any W with any mask
+    got = orc.mask_stats(w_now, meta, meta_ref, M, bitmask)
+    keep = keep_mask_from_meta(meta, cols, M, bitmask)
+    keep_ref = keep_mask_from_meta(meta_ref, cols, M, bitmask)
+    a = np.abs(w_now.astype(np.float64))
+    assert got["flips"] == int(np.sum(keep != keep_ref)) > 0
+    assert got["kept_abs"] == pytest.approx(float(a[keep].sum()), rel=1e-13)
+    assert got["total_abs"] == pytest.approx(float(a.sum()), rel=1e-13)
+    assert orc.mask_stats(w_now, meta, None, M, bitmask)["flips"] == 0
+
+
+def test_mask_statistics_closed_forms():
+    rng = np.random.default_rng(60)
+    rows, cols = 3, 64
+    w = rng.normal(0, 1, size=(rows, cols)).astype(np.float32)
+    # full density: every entry kept, S_t = 1; a mask against itself: no flips
+    full = run(w, N=4, M=4)["meta"]
+    s = orc.mask_stats(w, full, full, 4, True)
+    assert s["flips"] == 0 and s["kept_abs"] == s["total_abs"] > 0
+    # complementary 2:4 masks (keep {0, 1} against keep {2, 3}) differ in every entry
+    lo = np.full((rows, cols // 32), 0x33333333, dtype=np.uint32)
+    hi = np.full((rows, cols // 32), 0xCCCCCCCC, dtype=np.uint32)
+    assert orc.mask_stats(w, lo, hi, 4, True)["flips"] == rows * cols
+    # the same two masks in index form: nibble 0x4 = positions (0, 1), nibble 0xE = positions (2, 3)
+    lo_i = np.full((rows, cols // 32), 0x44444444, dtype=np.uint32)
+    hi_i = np.full((rows, cols // 32), 0xEEEEEEEE, dtype=np.uint32)
+    si = orc.mask_stats(w, lo_i, hi_i, 4, False)
+    assert si["flips"] == rows * cols
+    assert si["kept_abs"] == pytest.approx(float(np.abs(w.astype(np.float64)).reshape(-1, 4)[:, :2].sum()), rel=1e-13)
+    # a hand-sized case: one row of 32 columns, keep columns 0 and 3 of every group; |w| = 1, 2, 3, 4 repeating
+    w1 = np.tile(np.array([1, -2, 3, -4], dtype=np.float32), 8)[None, :]
+    m1 = np.full((1, 1), 0x99999999, dtype=np.uint32)
+    s1 = orc.mask_stats(w1, m1, None, 4, True)
+    assert s1["kept_abs"] == 8 * (1 + 4) and s1["total_abs"] == 8 * 10
+
+
+def test_sparse_weight_ratio_rises_as_alpha_ramps():
+    """App. C: with the decay ramping up, masked magnitudes shrink and S_t moves toward 1 (smoke test)."""
+    rng = np.random.default_rng(61)
+    rows, cols = 8, 128
+    w = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    m = np.zeros_like(w)
+    v = np.full_like(w, 1e-6)
+    g = np.zeros((rows, cols), dtype=np.uint16)
+    ratios = []
+    T = 60
+    for t in range(1, T + 1):
+        out = run(w, m, v, g, N=2, M=4, hyper=Hyper(lr=1e-3, l1_coeff=1e-3, step=t, total_steps=T))
+        w, m, v = out["w"], out["m"], out["v"]
+        s = orc.mask_stats(w, out["meta"], None, 4, True)
+        ratios.append(s["kept_abs"] / s["total_abs"])
+    assert ratios[-1] > ratios[0] and ratios[-1] > 0.9
