@@ -52,6 +52,8 @@ def parse_args():
     p.add_argument("--e2e-steps", type=int, default=4)
     p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
     p.add_argument("--seed", type=int, default=0)
+    p.add_argument("--op", choices=["step", "mask_stats"], default="step",
+                   help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass")
     return p.parse_args()
 
 
@@ -444,8 +446,82 @@ def cuda_arm(args):
     print(json.dumps(line), flush=True)
 
 
+def stats_arm(args):
+    """The App. C statistics pass (cast_plan_mask_stats, one launch over all matrices) over the workload: 4 B of weight and
+    2/8 B of metadata read per parameter, nothing written but three counters."""
+    import ctypes
+    import numpy as np
+    import torch
+    import paper_2509_25996_b200 as cast
+    from paper_2509_25996_b200 import binding as B
+    from paper_2509_25996_b200 import workloads
+    from paper_2509_25996_b200.runner import DeviceModelState, Hyper
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    N, M = (int(x) for x in args.nm.split(":"))
+    wl = workloads.workload(args.workload)
+    enc = 0 if (N, M) == (2, 4) else B.CAST_F_META_BITMASK
+    state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones")
+    hyper = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl.total_steps)
+    refs = []
+    state.step(hyper, B.CAST_F_RESELECT | enc)                 # mask of the initial weights
+    for mat in state.mats:
+        refs.append(mat.meta.clone())
+    hyper.step += 1
+    state.step(hyper, B.CAST_F_RESELECT | enc)                 # mask one step later
+    stats = torch.zeros(ctypes.sizeof(B.cast_mask_stats_t), dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def one_pass():
+        cast.check(cast.cast_plan_mask_stats(state.plan, refs, enc, stats, stream))
+
+    for _ in range(args.warmup):
+        one_pass()
+    torch.cuda.synchronize(dev)
+    stats.zero_()
+    launches0 = cast.cast_kernel_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        one_pass()
+    ev1.record(stream)
+    torch.cuda.synchronize(dev)
+    torch.cuda.profiler.stop()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    launches = cast.cast_kernel_launch_count() - launches0
+    got = B.cast_mask_stats_t.from_buffer_copy(stats.cpu().numpy().tobytes())
+    # parity on the first matrix against the oracle (host copies)
+    from oracle import adams_oracle as orc
+    m0 = state.mats[0]
+    single = torch.zeros_like(stats)
+    cast.check(cast.cast_mask_stats(m0.w, m0.meta, refs[0], m0.rows, m0.cols, M, enc, single, stream))
+    torch.cuda.synchronize(dev)
+    g0 = B.cast_mask_stats_t.from_buffer_copy(single.cpu().numpy().tobytes())
+    r0 = orc.mask_stats(m0.w.cpu().numpy(), m0.meta.cpu().numpy().view(np.uint32), refs[0].cpu().numpy().view(np.uint32),
+                        M, bool(enc))
+    ok = (g0.mask_diff == r0["flips"] and abs(g0.kept_abs_sum - r0["kept_abs"]) <= 1e-12 * r0["kept_abs"]
+          and abs(g0.total_abs_sum - r0["total_abs"]) <= 1e-12 * r0["total_abs"])
+    gbs = wl.n_params * 4.25 / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    print(json.dumps({
+        "metric": "mask statistics (App. C) params/s", "value": wl.n_params / (ms * 1e-3), "unit": "params/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "nm": args.nm, "params": wl.n_params, "matrices": len(wl.shapes),
+                   "l2": "inputs far larger than L2, no flush"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
+                     "kernel": "mask_stats_kernel", "bytes_per_param": 4.25, "launches_per_step": launches // args.steps, "traffic": None},
+        "stats": {"flip_rate_vs_initial": got.mask_diff / args.steps / wl.n_params,
+                  "sparse_weight_ratio": got.kept_abs_sum / got.total_abs_sum},
+        "parity": {"ok": bool(ok), "sample": "first matrix against the CPU oracle"}}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.op == "mask_stats" and args.impl != "reference":
+        return stats_arm(args)
     if args.impl == "reference":
         reference_arm(args)
     else:

@@ -180,6 +180,44 @@ CAST_API int cast_host_ctx_sync(void* ctx);
 CAST_API int cast_host_ctx_destroy(void* ctx);
 
 /*
+ * cast_mask_stats -- the mask statistics the paper monitors during training (App. C), for one matrix:
+ *
+ *   mask_diff      += ||M - M_ref||_0   numerator of the flip rate r_t when M_ref is the previous mask, of the
+ *                                       initial flip rate i_t when it is the initial mask (0 when meta_ref is NULL)
+ *   kept_abs_sum   += ||W (.) M||_1     numerator of the sparse weight ratio S_t
+ *   total_abs_sum  += ||W||_1           its denominator
+ *
+ * The denominators of r_t and i_t are the parameter counts, which the caller knows.  Sums are formed in fp64
+ * (their last bits depend on the order in which CTAs add their parts).
+ *
+ *   w          device, fp32 [rows*cols]: the weights W.
+ *   meta       device, uint32 [rows*cols/32]: the mask M in the metadata layout described at the top.
+ *   meta_ref   device, same shape and form as meta, or NULL.
+ *   M          group size (2, 4, 8, 16, 32); flags: CAST_F_META_BITMASK or 0 (index form, M == 4 only).
+ *   stats      device, 8-byte aligned; the call ADDS to it (zero it before the first matrix of a model, then
+ *              call once per matrix to get the model-wide sums of App. C).
+ * Asynchronous on `stream`.  Errors as cast_adams_step; nothing is launched on an error.
+ */
+typedef struct cast_mask_stats {
+    unsigned long long mask_diff;
+    unsigned long long reserved_;     /* keeps the doubles 16-byte aligned; never written */
+    double kept_abs_sum;
+    double total_abs_sum;
+} cast_mask_stats_t;
+CAST_API int cast_mask_stats(const float* w, const uint32_t* meta, const uint32_t* meta_ref,
+                    int64_t rows, int64_t cols, int M, uint32_t flags,
+                    cast_mask_stats_t* stats, cast_stream_t stream);
+
+/*
+ * cast_plan_mask_stats -- cast_mask_stats over every matrix of a plan in one launch (per 384 matrices), with
+ * the weights and masks the plan's descriptors name.  `meta_ref` is a HOST array of n_tensors device pointers
+ * (the reference mask of each matrix, same shape and form as its mask), or NULL for no reference.  `flags`
+ * is CAST_F_META_BITMASK or 0 and must name the form the plan's steps write.  `stats` as in cast_mask_stats.
+ */
+CAST_API int cast_plan_mask_stats(void* plan, const uint32_t* const* meta_ref, uint32_t flags,
+                         cast_mask_stats_t* stats, cast_stream_t stream);
+
+/*
  * cast_host_step_static -- cast_host_step for callers that must not allocate device memory.
  * (The paper has no counterpart to this entry point: it is a packaging variant of the call above.)
  *

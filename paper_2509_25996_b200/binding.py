@@ -36,7 +36,7 @@ CAST_F_EMIT_DENSE = 1 << 4
 EXPORTS = (
     "cast_adams_step", "cast_plan_create", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
-    "cast_host_step_static",
+    "cast_host_step_static", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
 )
 
@@ -102,6 +102,12 @@ def load_library() -> ctypes.CDLL:
     lib.cast_host_step.argtypes = [ctypes.c_void_p] + _STEP_ARGS
     lib.cast_host_step_static.restype = ctypes.c_int
     lib.cast_host_step_static.argtypes = _STEP_ARGS + [ctypes.c_void_p]
+    lib.cast_mask_stats.restype = ctypes.c_int
+    lib.cast_mask_stats.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                    ctypes.c_int, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p]
+    lib.cast_plan_mask_stats.restype = ctypes.c_int
+    lib.cast_plan_mask_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_uint32, ctypes.c_void_p,
+                                         ctypes.c_void_p]
     lib.cast_host_ctx_sync.restype = ctypes.c_int
     lib.cast_host_ctx_sync.argtypes = [ctypes.c_void_p]
     lib.cast_host_ctx_destroy.restype = ctypes.c_int
@@ -217,6 +223,25 @@ def cast_host_step_static(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, row
         _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
         int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
         int(flags), _ptr(flip_count), _stream(stream))
+
+
+class cast_mask_stats_t(ctypes.Structure):
+    _fields_ = [("mask_diff", ctypes.c_ulonglong), ("reserved_", ctypes.c_ulonglong),
+                ("kept_abs_sum", ctypes.c_double), ("total_abs_sum", ctypes.c_double)]
+
+
+def cast_mask_stats(w, meta, meta_ref, rows, cols, M, flags, stats, stream=None) -> int:
+    """`stats`: device buffer of sizeof(cast_mask_stats_t) = 32 bytes that the call adds to."""
+    return load_library().cast_mask_stats(_ptr(w), _ptr(meta), _ptr(meta_ref), int(rows), int(cols), int(M), int(flags),
+                                          _ptr(stats), _stream(stream))
+
+
+def cast_plan_mask_stats(plan, meta_refs, flags, stats, stream=None) -> int:
+    """`meta_refs`: a sequence of one reference-mask buffer per matrix of the plan, or None."""
+    arr = None
+    if meta_refs is not None:
+        arr = (ctypes.c_void_p * len(meta_refs))(*[_ptr(r) for r in meta_refs])
+    return load_library().cast_plan_mask_stats(plan, arr, int(flags), _ptr(stats), _stream(stream))
 
 
 def cast_host_ctx_sync(ctx) -> int:

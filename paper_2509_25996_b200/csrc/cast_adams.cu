@@ -13,6 +13,8 @@ namespace cast {
 static thread_local int g_last_cuda_error = 0;
 static std::atomic<unsigned long long> g_launches{0};
 
+void count_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+
 int cuda_failed(cudaError_t e)
 {
     g_last_cuda_error = (int)e;
@@ -251,6 +253,30 @@ struct Plan {
     std::vector<MultiParams> launches;   // one table per launch of up to kMaxLaunchTensors matrices
 };
 }  // namespace
+
+int plan_tensor_count(const void* plan)
+{
+    const Plan* p = (const Plan*)plan;
+    if (!p || p->magic != kPlanMagic) return -1;
+    return p->n_tensors;
+}
+
+bool plan_tensor(const void* plan, int i, int* M, const float** w, const uint32_t** meta, uint32_t* n_units)
+{
+    const Plan* p = (const Plan*)plan;
+    if (!p || p->magic != kPlanMagic || i < 0 || i >= p->n_tensors) return false;
+    for (const MultiParams& mp : p->launches) {
+        if (i < (int)mp.n_tensors) {
+            *M = p->M;
+            *w = mp.desc[i].w;
+            *meta = mp.desc[i].meta;
+            *n_units = mp.desc[i].n_units;
+            return true;
+        }
+        i -= (int)mp.n_tensors;
+    }
+    return false;
+}
 
 }  // namespace cast
 

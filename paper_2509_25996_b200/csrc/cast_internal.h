@@ -18,6 +18,9 @@ int cuda_failed(cudaError_t e);
         if (cast_e_ != cudaSuccess) return ::cast::cuda_failed(cast_e_); \
     } while (0)
 
+// One more kernel launched (for cast_kernel_launch_count).
+void count_launch();
+
 // N:M, flags and the flip counter pointer.
 int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count);
 

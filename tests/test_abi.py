@@ -141,3 +141,21 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(B, "LIB_PATH", os.path.join(ROOT, "no_such_dir", "libcast_adams.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         B.load_library()
+
+
+def test_mask_stats_argument_checks():
+    ok = dict(w=W, meta=META, meta_ref=None, rows=4, cols=64, M=4, flags=0, stats=SC)
+    def call_stats(**over):
+        a = dict(ok); a.update(over)
+        return cast.cast_mask_stats(**a)
+    before = cast.cast_kernel_launch_count()
+    assert call_stats(w=None) == B.CAST_ERR_NULL
+    assert call_stats(stats=None) == B.CAST_ERR_NULL
+    assert call_stats(M=3) == B.CAST_ERR_NM
+    assert call_stats(M=8) == B.CAST_ERR_NM                       # index form is 2:4 only
+    assert call_stats(flags=B.CAST_F_RESELECT) == B.CAST_ERR_HYPER
+    assert call_stats(cols=48) == B.CAST_ERR_SHAPE
+    assert call_stats(meta=META + 4) == B.CAST_ERR_ALIGN
+    assert call_stats(stats=SC + 4) == B.CAST_ERR_ALIGN
+    assert call_stats() in (B.CAST_ERR_CUDA, B.CAST_ERR_MEMORY)   # fake addresses are not device memory
+    assert cast.cast_kernel_launch_count() == before
