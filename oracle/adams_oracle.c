@@ -44,6 +44,9 @@ typedef REAL real;
 #define ORACLE_F_META_BITMASK   4u   /* metadata = M-bit keep mask per group             */
 #define ORACLE_F_V_KEPT_FROM_G  8u   /* alternate reading: kept entries feed g^2 into v  */
 #define ORACLE_F_EMIT_DENSE    16u   /* forward weight is Diag(A) W without the mask     */
+#define ORACLE_F_EMIT_COMPRESSED 32u /* forward weight holds only the kept entries: rows x cols*N/M,
+                                        the N kept values of each group in column order (the pruned
+                                        matrix of Alg. 2's final loop without its zeros)               */
 
 enum { ORACLE_OK = 0, ORACLE_BAD_ARGS = -1 };
 
@@ -152,6 +155,7 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
     const int bitmask_encoding = (flags & ORACLE_F_META_BITMASK) != 0;
     if (!bitmask_encoding && !(N == 2 && M == 4)) return ORACLE_BAD_ARGS;
     if ((flags & ORACLE_F_COUNT_FLIPS) && !flip_count) return ORACLE_BAD_ARGS;
+    if ((flags & ORACLE_F_EMIT_COMPRESSED) && (flags & ORACLE_F_EMIT_DENSE)) return ORACLE_BAD_ARGS;
 
     /* scalars of the step, formed in double and rounded once to the working type */
     const real alpha = (real)((double)step / (double)total_steps);   /* alpha_t = t/T   (Alg. 1) */
@@ -191,6 +195,7 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
                 flips += (uint64_t)popcount32(keep ^ prev);       /* ||M_t - M_{t-1}||_0, App. C */
             }
 
+            int n_emitted = 0;      /* kept entries of this group written so far (compressed form) */
             for (int j = 0; j < M; ++j) {
                 const int64_t idx = base + j;
                 const int kept = (keep >> j) & 1u;
@@ -227,7 +232,13 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
                  * The scale multiplies the stored (rounded) master weight. */
                 const int64_t col = i * M + j;
                 const real a = scale ? (real)scale[r * n_seg + col / (cols / n_seg)] : one;
-                if (kept || (flags & ORACLE_F_EMIT_DENSE))
+                if (flags & ORACLE_F_EMIT_COMPRESSED) {
+                    /* group i of row r owns slots (r * cols/M + i) * N ... + N - 1 */
+                    if (kept && n_emitted < N) {
+                        w_fwd[(r * (cols / M) + i) * N + n_emitted] = real_to_bf16_rne(a * (real)w[idx]);
+                        ++n_emitted;
+                    }
+                } else if (kept || (flags & ORACLE_F_EMIT_DENSE))
                     w_fwd[idx] = real_to_bf16_rne(a * (real)w[idx]);
                 else
                     w_fwd[idx] = 0;                                             /* +0.0 */

@@ -19,6 +19,7 @@ F_COUNT_FLIPS = 2
 F_META_BITMASK = 4
 F_V_KEPT_FROM_G = 8
 F_EMIT_DENSE = 16
+F_EMIT_COMPRESSED = 32
 
 _lib = None
 
@@ -76,6 +77,7 @@ def adams_step_inplace(w, m, v, g_bits, w_fwd_bits, meta, scale, rows, cols, N, 
                   (w_fwd_bits, np.uint16), (meta, np.uint32)):
         assert a.dtype == dt and a.flags["C_CONTIGUOUS"], (a.dtype, dt)
     assert w.size == rows * cols and meta.size == rows * cols // 32
+    assert w_fwd_bits.size == (rows * cols * N // M if flags & F_EMIT_COMPRESSED else rows * cols)
     n_seg = 1
     scale_ptr = None
     if scale is not None:
@@ -97,13 +99,15 @@ def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELE
                meta_in=None, precision: str = "f64"):
     """Out-of-place convenience wrapper for 2-D inputs.
 
-    Returns dict(w, m, v, w_fwd (uint16 bf16 bits), meta (uint32 [rows, cols/32]), flips)."""
+    Returns dict(w, m, v, w_fwd (uint16 bf16 bits; [rows, cols*N/M] with F_EMIT_COMPRESSED), meta (uint32
+    [rows, cols/32]), flips)."""
     rows, cols = w.shape
     w2 = np.ascontiguousarray(w, dtype=np.float32).copy().reshape(-1)
     m2 = np.ascontiguousarray(m, dtype=np.float32).copy().reshape(-1)
     v2 = np.ascontiguousarray(v, dtype=np.float32).copy().reshape(-1)
     g2 = np.ascontiguousarray(g_bits, dtype=np.uint16).reshape(-1)
-    fwd = np.zeros(rows * cols, dtype=np.uint16)
+    fwd_cols = cols * N // M if flags & F_EMIT_COMPRESSED else cols
+    fwd = np.zeros(rows * fwd_cols, dtype=np.uint16)
     if meta_in is None:
         meta = np.zeros(rows * cols // 32, dtype=np.uint32)
     else:
@@ -111,7 +115,7 @@ def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELE
     sc = None if scale is None else np.ascontiguousarray(scale, dtype=np.float32)
     flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision)
     return dict(w=w2.reshape(rows, cols), m=m2.reshape(rows, cols), v=v2.reshape(rows, cols),
-                w_fwd=fwd.reshape(rows, cols), meta=meta.reshape(rows, cols // 32), flips=flips)
+                w_fwd=fwd.reshape(rows, fwd_cols), meta=meta.reshape(rows, cols // 32), flips=flips)
 
 
 def mask_stats(w, meta, meta_ref, M: int, bitmask: bool):

@@ -497,3 +497,37 @@ def test_sparse_weight_ratio_rises_as_alpha_ramps():
         s = orc.mask_stats(w, out["meta"], None, 4, True)
         ratios.append(s["kept_abs"] / s["total_abs"])
     assert ratios[-1] > ratios[0] and ratios[-1] > 0.9
+
+
+# --------------------------------------------------------------------------- compressed emission (Alg. 2, final loop)
+
+@pytest.mark.parametrize("N,M,bitmask", [(2, 4, False), (2, 4, True), (1, 4, True), (3, 4, True), (4, 8, True), (1, 2, True), (5, 16, True)])
+def test_compressed_emission_is_the_pruned_matrix_without_its_pruned_slots(N, M, bitmask):
+    """The compressed forward weight holds, group by group and in column order, exactly the entries the pruned
+    form keeps: gathering the pruned form through an independently decoded mask gives it, and scattering it
+    back through that mask gives the pruned form."""
+    rng = np.random.default_rng(70 + M + N)
+    rows, cols = 5, 160
+    w = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    g = bf16_exact(rng.normal(0, 1e-3, size=(rows, cols)))[1]
+    scale = (1.0 + 0.1 * rng.random((rows, 2))).astype(np.float32)
+    enc = orc.F_META_BITMASK if bitmask else 0
+    dense = run(w, g=g, scale=scale, N=N, M=M, flags=orc.F_RESELECT | enc)
+    comp = run(w, g=g, scale=scale, N=N, M=M, flags=orc.F_RESELECT | enc | orc.F_EMIT_COMPRESSED)
+    for k in ("w", "m", "v", "meta"):
+        assert np.array_equal(dense[k], comp[k])
+    assert comp["w_fwd"].shape == (rows, cols * N // M)
+    keep = keep_mask_from_meta(dense["meta"], cols, M, bitmask)
+    assert np.array_equal(comp["w_fwd"].reshape(-1), dense["w_fwd"][keep])        # row-major gather keeps column order
+    back = np.zeros((rows, cols), dtype=np.uint16)
+    back[keep] = comp["w_fwd"].reshape(-1)
+    assert np.array_equal(back, dense["w_fwd"])
+
+
+def test_compressed_emission_hand_example():
+    """One row, 2:4, weights that do not move (lr = 0), scale 2: the kept pair of every group, doubled."""
+    w = np.tile(np.array([0.5, -4.0, 3.0, 0.25, 1.0, 1.0, -1.0, 0.125], dtype=np.float32), 4)[None, :]
+    out = run(w, N=2, M=4, scale=np.full((1, 2), 2.0, dtype=np.float32), hyper=Hyper(lr=0.0),
+              flags=orc.F_RESELECT | orc.F_EMIT_COMPRESSED)
+    want = np.tile(np.array([-8.0, 6.0, 2.0, 2.0], dtype=np.float32), 4)            # ties: the lower columns (1.0, 1.0)
+    assert np.array_equal(bf16_bits_to_f32(out["w_fwd"]).reshape(-1), want)
