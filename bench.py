@@ -48,6 +48,8 @@ def parse_args():
     p.add_argument("--nm", default="2:4")
     p.add_argument("--l1-coeff", type=float, default=1e-3)
     p.add_argument("--count-flips", action="store_true")
+    p.add_argument("--emit", choices=["pruned", "dense", "compressed"], default="pruned",
+                   help="forward weight: pruned product in the dense layout (default), dense product, or kept entries only")
     p.add_argument("--e2e-layers", type=int, default=1, help="LLaMA layers held in host memory for the e2e leg (0 = skip)")
     p.add_argument("--e2e-steps", type=int, default=4)
     p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
@@ -134,7 +136,8 @@ def time_oracle(arrays, N, M, hyper, flags, threads: int):
     jobs, outs = [], []
     for a in arrays:
         rows, cols = a["rows"], a["cols"]
-        fwd = np.zeros(rows * cols, dtype=np.uint16)
+        fcols = cols * N // M if flags & orc.F_EMIT_COMPRESSED else cols      # forward-weight columns per row
+        fwd = np.zeros(rows * fcols, dtype=np.uint16)
         meta = np.zeros(rows * cols // 32, dtype=np.uint32)
         outs.append(dict(w=a["w"], m=a["m"], v=a["v"], w_fwd=fwd, meta=meta))
         per = max(1, -(-rows // threads))
@@ -142,7 +145,7 @@ def time_oracle(arrays, N, M, hyper, flags, threads: int):
             r1 = min(rows, r0 + per)
             sl = slice(r0 * cols, r1 * cols)
             jobs.append((a["w"].reshape(-1)[sl], a["m"].reshape(-1)[sl], a["v"].reshape(-1)[sl], a["g"].reshape(-1)[sl],
-                         fwd[sl], meta[r0 * cols // 32:r1 * cols // 32],
+                         fwd[r0 * fcols:r1 * fcols], meta[r0 * cols // 32:r1 * cols // 32],
                          None if a["scale"] is None else a["scale"][r0:r1], r1 - r0, cols))
 
     def one(j):
@@ -234,6 +237,13 @@ def cuda_arm(args):
     if args.count_flips:
         flags |= B.CAST_F_COUNT_FLIPS
     bytes_per_param = BYTES_PER_PARAM_FLIPS if args.count_flips else BYTES_PER_PARAM
+    if args.emit == "dense":
+        flags |= B.CAST_F_EMIT_DENSE
+    compressed = args.emit == "compressed"
+    if compressed:
+        if wl.resident_layers:
+            raise SystemExit("--emit compressed is not wired for the streamed workload")
+        bytes_per_param -= 2.0 * (1.0 - N / M)            # only N of every M forward weights are written
 
     if wl.resident_layers:
         # per-layer calls alternating on 2 streams over the resident layer slots (no host traffic)
@@ -242,7 +252,7 @@ def cuda_arm(args):
         mats = state.slots[0].mats
         oracle_repeats = len(wl.shapes) // wl.layer_matrices // wl.resident_layers   # steps a slot takes per pass
     else:
-        state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones")
+        state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones", compressed=compressed)
         mats = state.mats
         oracle_repeats = 1
     hyper = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl.total_steps)
@@ -380,6 +390,7 @@ def cuda_arm(args):
         oh = orc.Hyper(lr=hyper.lr, beta1=hyper.beta1, beta2=hyper.beta2, eps=hyper.eps, l1_coeff=hyper.l1_coeff,
                        step=1000, total_steps=wl.total_steps)
         o_flags = orc.F_RESELECT | (0 if (N, M) == (2, 4) else orc.F_META_BITMASK)
+        o_flags |= {"pruned": 0, "dense": orc.F_EMIT_DENSE, "compressed": orc.F_EMIT_COMPRESSED}[args.emit]
         ok = bool(parity_out)
         for t in (picks if parity_out else []):
             a = parity_in[t]
@@ -428,7 +439,7 @@ def cuda_arm(args):
                                                                                   else "L2 flushed by a 512 MB write before every step, steps timed one by one"),
                    "resident_layers": wl.resident_layers, "streams": 2 if wl.resident_layers else 1,
                    "lr": hyper.lr, "betas": [hyper.beta1, hyper.beta2], "eps": hyper.eps, "l1_coeff": hyper.l1_coeff,
-                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "seed": args.seed},
+                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "seed": args.seed},
         "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,

@@ -74,8 +74,13 @@ enum cast_flags {
     CAST_F_META_BITMASK  = 1u << 2, /* bitmask-form metadata (required unless N:M == 2:4)              */
     CAST_F_V_KEPT_FROM_G = 1u << 3, /* alternate reading of Eq. 8: kept entries feed g^2 (textbook Adam)
                                        into v; entries outside the kept set still feed mu~^2           */
-    CAST_F_EMIT_DENSE    = 1u << 4  /* emit Diag(A~) W~ for all entries (the dense training-time forward
+    CAST_F_EMIT_DENSE    = 1u << 4, /* emit Diag(A~) W~ for all entries (the dense training-time forward
                                        weight of Alg. 2) instead of the pruned product                  */
+    CAST_F_EMIT_COMPRESSED = 1u << 5 /* emit only the kept entries of the pruned product (Alg. 2, final loop):
+                                       w_fwd_bf16 is then [rows][cols*N/M], the N kept values of each group in
+                                       column order; with the metadata it is the whole pruned matrix, and a
+                                       step writes 2 N/M instead of 2 bytes per parameter.  M <= 8 only; not
+                                       together with CAST_F_EMIT_DENSE                                   */
 };
 
 /*
@@ -85,7 +90,7 @@ enum cast_flags {
  *   w, m, v      device, fp32 [rows*cols], in/out: master weight, first moment (stored undecayed),
  *                second moment.
  *   g            device, bf16 [rows*cols], in: gradient of this iteration.
- *   w_fwd_bf16   device, bf16 [rows*cols], out: bf16(A[r, c / (cols/scale_groups)] * w_new[r, c]) where
+ *   w_fwd_bf16   device, bf16 [rows*cols] ([rows*cols*N/M] with CAST_F_EMIT_COMPRESSED), out: bf16(A[r, c / (cols/scale_groups)] * w_new[r, c]) where
  *                kept, +0.0 (0x0000) elsewhere (all entries with CAST_F_EMIT_DENSE).  Rounding is to
  *                nearest even of the fp32 product.
  *   meta         device, uint32 [rows*cols/32], in/out (layout above).  Read when CAST_F_RESELECT is
@@ -146,6 +151,11 @@ typedef struct cast_hyper {
  * cast_plan_destroy frees the handle (no device work).
  */
 CAST_API int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out);
+/* As cast_plan_create, for matrices whose w_fwd buffers have the compressed size: plan_flags is
+ * CAST_F_EMIT_COMPRESSED (or 0 = cast_plan_create).  Every step of such a plan must carry that flag, and a step
+ * of an ordinary plan must not (CAST_ERR_PLAN otherwise): the buffer sizes are fixed when the plan is made. */
+CAST_API int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, int N, int M, uint32_t plan_flags,
+                        void** plan_out);
 CAST_API int cast_plan_step(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
                    cast_stream_t stream);
 CAST_API int cast_plan_destroy(void* plan);

@@ -32,9 +32,10 @@ CAST_F_COUNT_FLIPS = 1 << 1
 CAST_F_META_BITMASK = 1 << 2
 CAST_F_V_KEPT_FROM_G = 1 << 3
 CAST_F_EMIT_DENSE = 1 << 4
+CAST_F_EMIT_COMPRESSED = 1 << 5
 
 EXPORTS = (
-    "cast_adams_step", "cast_plan_create", "cast_plan_step", "cast_plan_destroy",
+    "cast_adams_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
@@ -92,6 +93,9 @@ def load_library() -> ctypes.CDLL:
     lib.cast_plan_create.restype = ctypes.c_int
     lib.cast_plan_create.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                      ctypes.POINTER(ctypes.c_void_p)]
+    lib.cast_plan_create_ex.restype = ctypes.c_int
+    lib.cast_plan_create_ex.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_uint32,
+                                        ctypes.POINTER(ctypes.c_void_p)]
     lib.cast_plan_step.restype = ctypes.c_int
     lib.cast_plan_step.argtypes = [ctypes.c_void_p, ctypes.POINTER(cast_hyper_t), ctypes.c_void_p, ctypes.c_void_p]
     lib.cast_plan_destroy.restype = ctypes.c_int
@@ -181,6 +185,15 @@ def cast_plan_create(tensors: Sequence[cast_tensor_t], N: int, M: int):
     arr = (cast_tensor_t * max(n, 1))(*tensors)
     out = ctypes.c_void_p(None)
     rc = load_library().cast_plan_create(arr if n else None, n, int(N), int(M), ctypes.byref(out))
+    return rc, (out.value if rc == CAST_OK else None)
+
+
+def cast_plan_create_ex(tensors: Sequence[cast_tensor_t], N: int, M: int, plan_flags: int):
+    """Returns (status, plan handle or None); plan_flags: CAST_F_EMIT_COMPRESSED or 0."""
+    n = len(tensors)
+    arr = (cast_tensor_t * max(n, 1))(*tensors)
+    out = ctypes.c_void_p(None)
+    rc = load_library().cast_plan_create_ex(arr if n else None, n, int(N), int(M), int(plan_flags), ctypes.byref(out))
     return rc, (out.value if rc == CAST_OK else None)
 
 

@@ -35,6 +35,7 @@ constexpr uint32_t kCountFlips = 1u << 1;
 constexpr uint32_t kMetaBitmask = 1u << 2;
 constexpr uint32_t kVKeptFromG = 1u << 3;
 constexpr uint32_t kEmitDense = 1u << 4;
+constexpr uint32_t kEmitCompressed = 1u << 5;
 
 // Kernel modes: the flag word is a compile-time constant in the two common cases.
 constexpr int kModeGeneric = 0;        // any flags, read from StepConsts at run time
@@ -173,6 +174,7 @@ struct UnitRegs {
     uint4 g;               // 8 bf16 gradients in; 8 bf16 forward weights out
     uint32_t prev_byte;    // metadata byte of the unit before the step (when it is read)
     uint32_t meta_byte;    // metadata byte after the step
+    uint32_t keep;         // keep mask of the unit (bit j = column j kept); not set in the 2:4 index mode
 };
 
 template <int MODE>
@@ -219,6 +221,7 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
         else keep = prev_keep;
 #pragma unroll
         for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+        u.keep = keep;
         if (bitmask) u.meta_byte = keep;
         else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
         if constexpr (MODE == kModeGeneric) flips = (uint32_t)__popc(keep ^ prev_keep);
@@ -299,7 +302,29 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         st_f4(t.m + e + 4, make_float4(u.m[4], u.m[5], u.m[6], u.m[7]));
         st_f4(t.v + e, make_float4(u.v[0], u.v[1], u.v[2], u.v[3]));
         st_f4(t.v + e + 4, make_float4(u.v[4], u.v[5], u.v[6], u.v[7]));
-        *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
+        bool compressed = false;
+        if constexpr (MODE == kModeGeneric && M <= 8) compressed = (flags & kEmitCompressed) != 0;
+        if (!compressed) {
+            *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
+        } else {
+            // Compressed form: only the kept entries, in column order, 8 N / M per unit.  Every group keeps
+            // exactly N, so the slot of a kept column is the number of kept columns before it in the unit.
+            // The values are scattered into a private 16-byte row of shared memory and read back as a vector.
+            __shared__ __align__(16) uint16_t s_comp[kThreads * 8];
+            uint16_t* mine = s_comp + threadIdx.x * 8;
+            const uint32_t hw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                if ((u.keep >> i) & 1u)
+                    mine[__popc(u.keep & ((1u << i) - 1u))] = (uint16_t)(hw[i >> 1] >> (16 * (i & 1)));
+            const uint32_t cnt = (uint32_t)(8 * c.n_keep) / (uint32_t)M;
+            uint16_t* dst = t.w_fwd + (size_t)unit * cnt;
+            if (cnt == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(mine);
+            else if (cnt == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(mine);
+            else if (cnt == 2) *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(mine);
+            else
+                for (uint32_t k = 0; k < cnt; ++k) dst[k] = mine[k];
+        }
         reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;
     }
     return active ? flips : 0u;

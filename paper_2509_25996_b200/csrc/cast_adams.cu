@@ -28,8 +28,10 @@ int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count)
     if (N < 1 || N > M) return CAST_ERR_NM;
     if (!(flags & CAST_F_META_BITMASK) && !(N == 2 && M == 4)) return CAST_ERR_NM;
     const uint32_t known = CAST_F_RESELECT | CAST_F_COUNT_FLIPS | CAST_F_META_BITMASK |
-                           CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE;
+                           CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE | CAST_F_EMIT_COMPRESSED;
     if (flags & ~known) return CAST_ERR_HYPER;
+    if ((flags & CAST_F_EMIT_COMPRESSED) && (flags & CAST_F_EMIT_DENSE)) return CAST_ERR_HYPER;
+    if ((flags & CAST_F_EMIT_COMPRESSED) && M > kUnitElems) return CAST_ERR_NM;
     if ((flags & CAST_F_COUNT_FLIPS) && flip_count == nullptr) return CAST_ERR_NULL;
     return CAST_OK;
 }
@@ -81,7 +83,8 @@ inline bool overlap(const Range& a, const Range& b) { return a.lo < b.hi && b.lo
 }  // namespace
 
 int check_pointers(const void* w, const void* m, const void* v, const void* g, const void* w_fwd,
-                   const void* meta, const void* scale, int scale_groups, int64_t rows, int64_t cols)
+                   const void* meta, const void* scale, int scale_groups, int64_t rows, int64_t cols,
+                   uint64_t fwd_elems)
 {
     if (!w || !m || !v || !g || !w_fwd || !meta) return CAST_ERR_NULL;
     const void* all[7] = {w, m, v, g, w_fwd, meta, scale};
@@ -91,7 +94,7 @@ int check_pointers(const void* w, const void* m, const void* v, const void* g, c
     Range r[7] = {
         {(uintptr_t)w, (uintptr_t)w + 4 * P},         {(uintptr_t)m, (uintptr_t)m + 4 * P},
         {(uintptr_t)v, (uintptr_t)v + 4 * P},         {(uintptr_t)g, (uintptr_t)g + 2 * P},
-        {(uintptr_t)w_fwd, (uintptr_t)w_fwd + 2 * P}, {(uintptr_t)meta, (uintptr_t)meta + P / 8},
+        {(uintptr_t)w_fwd, (uintptr_t)w_fwd + 2 * fwd_elems}, {(uintptr_t)meta, (uintptr_t)meta + P / 8},
         {(uintptr_t)scale, (uintptr_t)scale + (scale ? 4ull * (uint64_t)rows * (uint64_t)scale_groups : 0)}};
     const int n = scale ? 7 : 6;
     for (int i = 0; i < n; ++i)
@@ -250,6 +253,7 @@ struct Plan {
     int device;
     int N, M;
     int n_tensors;
+    uint32_t plan_flags;                 // CAST_F_EMIT_COMPRESSED or 0: fixes the size of the w_fwd buffers
     std::vector<MultiParams> launches;   // one table per launch of up to kMaxLaunchTensors matrices
 };
 }  // namespace
@@ -297,7 +301,8 @@ extern "C" int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
     if ((rc = make_step_consts(lr, beta1, beta2, eps, l1_coeff, step, total_steps, N, flags, &c)) != CAST_OK) return rc;
     if (!w || !m || !v || !g || !w_fwd_bf16 || !meta) return CAST_ERR_NULL;
     if ((rc = check_shape(rows, cols, M, scale != nullptr, scale_groups)) != CAST_OK) return rc;
-    if ((rc = check_pointers(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols)) != CAST_OK) return rc;
+    if ((rc = check_pointers(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols,
+                             fwd_elems_of(rows, cols, N, M, flags))) != CAST_OK) return rc;
     const void* ptrs[8] = {w, m, v, g, w_fwd_bf16, meta, scale, (flags & CAST_F_COUNT_FLIPS) ? flip_count : nullptr};
     if ((rc = check_device_memory(ptrs, 8)) != CAST_OK) return rc;
     const TensorDesc d = make_desc(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols);
@@ -306,19 +311,27 @@ extern "C" int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
 
 extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out)
 {
+    return cast_plan_create_ex(tensors, n_tensors, N, M, 0u, plan_out);
+}
+
+extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, int N, int M, uint32_t plan_flags,
+                                   void** plan_out)
+{
     if (!plan_out) return CAST_ERR_NULL;
     *plan_out = nullptr;
     if (!tensors) return CAST_ERR_NULL;
     if (n_tensors < 1) return CAST_ERR_SHAPE;
     int rc;
-    // the encoding flag is a per-step choice; here only N:M itself is checked
-    if ((rc = check_nm_flags(N, M, CAST_F_META_BITMASK, nullptr)) != CAST_OK) return rc;
+    if (plan_flags & ~(uint32_t)CAST_F_EMIT_COMPRESSED) return CAST_ERR_HYPER;
+    // the encoding flag is a per-step choice; here only N:M itself (and the compressed form's M <= 8) is checked
+    if ((rc = check_nm_flags(N, M, CAST_F_META_BITMASK | plan_flags, nullptr)) != CAST_OK) return rc;
 
     for (int i = 0; i < n_tensors; ++i) {
         const cast_tensor_t& t = tensors[i];
         if (!t.w || !t.m || !t.v || !t.g || !t.w_fwd || !t.meta) return CAST_ERR_NULL;
         if ((rc = check_shape(t.rows, t.cols, M, t.scale != nullptr, t.scale_groups)) != CAST_OK) return rc;
-        if ((rc = check_pointers(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols)) != CAST_OK) return rc;
+        if ((rc = check_pointers(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols,
+                                 fwd_elems_of(t.rows, t.cols, N, M, plan_flags))) != CAST_OK) return rc;
     }
     for (int i = 0; i < n_tensors; ++i) {
         const cast_tensor_t& t = tensors[i];
@@ -358,6 +371,7 @@ extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int
     }
     p->magic = kPlanMagic;
     p->N = N; p->M = M; p->n_tensors = n_tensors;
+    p->plan_flags = plan_flags;
     *plan_out = p;
     return CAST_OK;
 }
@@ -369,6 +383,7 @@ extern "C" int cast_plan_step(void* plan, const cast_hyper_t* h, unsigned long l
     if (!h) return CAST_ERR_NULL;
     int rc;
     if ((rc = check_nm_flags(p->N, p->M, h->flags, flip_count)) != CAST_OK) return rc;
+    if ((h->flags & CAST_F_EMIT_COMPRESSED) != p->plan_flags) return CAST_ERR_PLAN;
     StepConsts c;
     if ((rc = make_step_consts(h->lr, h->beta1, h->beta2, h->eps, h->l1_coeff, h->step, h->total_steps,
                                p->N, h->flags, &c)) != CAST_OK) return rc;

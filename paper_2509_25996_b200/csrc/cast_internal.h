@@ -32,8 +32,17 @@ int make_step_consts(float lr, float beta1, float beta2, float eps, float l1_coe
 int check_shape(int64_t rows, int64_t cols, int M, bool has_scale, int scale_groups);
 
 // Null / alignment / overlap rules of one matrix's pointers (addresses only, never dereferenced).
+// `fwd_elems` is the number of bf16 elements of w_fwd (rows*cols, or rows*cols*N/M in compressed form).
 int check_pointers(const void* w, const void* m, const void* v, const void* g, const void* w_fwd,
-                   const void* meta, const void* scale, int scale_groups, int64_t rows, int64_t cols);
+                   const void* meta, const void* scale, int scale_groups, int64_t rows, int64_t cols,
+                   uint64_t fwd_elems);
+
+// Elements of the forward-weight buffer of one matrix under `flags`.
+inline uint64_t fwd_elems_of(int64_t rows, int64_t cols, int N, int M, uint32_t flags)
+{
+    const uint64_t P = (uint64_t)rows * (uint64_t)cols;
+    return (flags & CAST_F_EMIT_COMPRESSED) ? P / (uint64_t)M * (uint64_t)N : P;
+}
 
 // Every given pointer must be device-accessible memory on the current device.
 int check_device_memory(const void* const* ptrs, int n);

@@ -140,7 +140,8 @@ extern "C" int cast_host_step(void* ctx,
     if ((rc = make_step_consts(lr, beta1, beta2, eps, l1_coeff, step, total_steps, N, flags, &k)) != CAST_OK) return rc;
     if (!w || !m || !v || !g || !w_fwd_bf16 || !meta) return CAST_ERR_NULL;
     if ((rc = check_shape(rows, cols, M, scale != nullptr, scale_groups)) != CAST_OK) return rc;
-    if ((rc = check_pointers(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols)) != CAST_OK) return rc;
+    const uint64_t fwd_total = fwd_elems_of(rows, cols, N, M, flags);
+    if ((rc = check_pointers(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols, fwd_total)) != CAST_OK) return rc;
     if (cols > c->max_block) return CAST_ERR_PLAN;
     int dev = -1;
     CAST_CUDA_TRY(cudaGetDevice(&dev));
@@ -175,7 +176,9 @@ extern "C" int cast_host_step(void* ctx,
         CAST_CUDA_TRY(cudaMemcpyAsync(w + off, s.w, 4 * P, cudaMemcpyDeviceToHost, s.stream));
         CAST_CUDA_TRY(cudaMemcpyAsync(m + off, s.m, 4 * P, cudaMemcpyDeviceToHost, s.stream));
         CAST_CUDA_TRY(cudaMemcpyAsync(v + off, s.v, 4 * P, cudaMemcpyDeviceToHost, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16 + off, s.fwd, 2 * P, cudaMemcpyDeviceToHost, s.stream));
+        const size_t fwd_scale_n = (flags & CAST_F_EMIT_COMPRESSED) ? (size_t)N : 1, fwd_scale_m = (flags & CAST_F_EMIT_COMPRESSED) ? (size_t)M : 1;
+        CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16 + off / fwd_scale_m * fwd_scale_n, s.fwd, 2 * (P / fwd_scale_m * fwd_scale_n),
+                                      cudaMemcpyDeviceToHost, s.stream));
         CAST_CUDA_TRY(cudaMemcpyAsync(meta + off / 32, s.meta, P / 8, cudaMemcpyDeviceToHost, s.stream));
     }
     return CAST_OK;

@@ -77,7 +77,8 @@ extern "C" int cast_host_step_static(float* w, float* m, float* v, const cast_bf
     if (!w || !m || !v || !g || !w_fwd_bf16 || !meta) return CAST_ERR_NULL;
     if ((rc = check_shape(rows, cols, M, scale != nullptr, scale_groups)) != CAST_OK) return rc;
     if (rows * cols > kStaticMaxParams) return CAST_ERR_PLAN;          // larger than the built-in staging area
-    if ((rc = check_pointers(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols)) != CAST_OK) return rc;
+    const uint64_t fwd_total = fwd_elems_of(rows, cols, N, M, flags);
+    if ((rc = check_pointers(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, cols, fwd_total)) != CAST_OK) return rc;
     const void* host_ptrs[7] = {w, m, v, g, w_fwd_bf16, meta, scale};
     for (const void* p : host_ptrs) {
         if (!p) continue;
@@ -115,7 +116,7 @@ extern "C" int cast_host_step_static(float* w, float* m, float* v, const cast_bf
     CAST_CUDA_TRY(cudaMemcpyAsync(w, d_w, 4 * P, cudaMemcpyDeviceToHost, s));
     CAST_CUDA_TRY(cudaMemcpyAsync(m, d_m, 4 * P, cudaMemcpyDeviceToHost, s));
     CAST_CUDA_TRY(cudaMemcpyAsync(v, d_v, 4 * P, cudaMemcpyDeviceToHost, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16, d_fwd, 2 * P, cudaMemcpyDeviceToHost, s));
+    CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16, d_fwd, 2 * (size_t)fwd_total, cudaMemcpyDeviceToHost, s));
     CAST_CUDA_TRY(cudaMemcpyAsync(meta, d_meta, P / 8, cudaMemcpyDeviceToHost, s));
     unsigned long long flips = 0;
     if (count) CAST_CUDA_TRY(cudaMemcpyAsync(&flips, d_flips, sizeof flips, cudaMemcpyDeviceToHost, s));

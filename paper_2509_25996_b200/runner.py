@@ -42,27 +42,32 @@ class DeviceModelState:
     """All prunable matrices of a model on one GPU plus the plan that steps them in one launch."""
 
     def __init__(self, shapes: Sequence[Tuple[int, int]], N: int = 2, M: int = 4, seed: int = 0,
-                 device="cuda:0", scale_mode: str = "ones", first_tensor_index: int = 0):
+                 device="cuda:0", scale_mode: str = "ones", first_tensor_index: int = 0, compressed: bool = False):
+        """compressed: the forward-weight buffers hold only the kept entries ([rows, cols*N/M]); every step of
+        this state then carries CAST_F_EMIT_COMPRESSED."""
         self.device = torch.device(device)
         self.N, self.M = N, M
+        self.compressed = compressed
         self.mats: List[MatrixState] = []
         for i, (rows, cols) in enumerate(shapes):
             inp = workloads.gen_tensor_inputs(rows, cols, seed=seed, tensor_index=first_tensor_index + i,
                                               device=self.device, scale_mode=scale_mode)
             self.mats.append(MatrixState(
                 rows, cols, inp.w, inp.m, inp.v, inp.g,
-                torch.empty((rows, cols), dtype=torch.bfloat16, device=self.device),
+                torch.empty((rows, cols * N // M if compressed else cols), dtype=torch.bfloat16, device=self.device),
                 torch.zeros((rows, cols // 32), dtype=torch.int32, device=self.device),
                 inp.scale))
         self.n_params = sum(s.rows * s.cols for s in self.mats)
         self.flips = torch.zeros(1, dtype=torch.int64, device=self.device)
         tensors = [B.make_tensor(s.w, s.m, s.v, s.g, s.w_fwd, s.meta, s.scale,
                                  1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in self.mats]
-        rc, self.plan = B.cast_plan_create(tensors, N, M)
+        rc, self.plan = B.cast_plan_create_ex(tensors, N, M, B.CAST_F_EMIT_COMPRESSED if compressed else 0)
         B.check(rc)
 
     def step(self, hyper: Hyper, flags: int, stream=None) -> None:
         """One AdamS iteration over every matrix (asynchronous on `stream` or the current stream)."""
+        if self.compressed:
+            flags |= B.CAST_F_EMIT_COMPRESSED
         h = B.make_hyper(hyper.lr, hyper.beta1, hyper.beta2, hyper.eps, hyper.l1_coeff,
                          hyper.step, hyper.total_steps, flags)
         s = stream if stream is not None else torch.cuda.current_stream(self.device)

@@ -51,7 +51,7 @@ class DeviceState:
         return all(b.intact() for b in (self.w, self.m, self.v, self.g, self.w_fwd, self.meta))
 
 
-def to_device(inp: workloads.TensorInputs, device, meta_in: Optional[np.ndarray] = None) -> DeviceState:
+def to_device(inp: workloads.TensorInputs, device, meta_in: Optional[np.ndarray] = None, fwd_elems: Optional[int] = None) -> DeviceState:
     rows, cols = inp.w.shape
     n = rows * cols
     meta = Guarded(n // 32, torch.int32, device)
@@ -59,7 +59,7 @@ def to_device(inp: workloads.TensorInputs, device, meta_in: Optional[np.ndarray]
         meta.view.copy_(torch.from_numpy(np.ascontiguousarray(meta_in).view(np.int32).reshape(-1)))
     else:
         meta.view.zero_()
-    fwd = Guarded(n, torch.bfloat16, device)
+    fwd = Guarded(n if fwd_elems is None else fwd_elems, torch.bfloat16, device)
     return DeviceState(rows, cols,
                        Guarded(n, torch.float32, device, inp.w.to(device)),
                        Guarded(n, torch.float32, device, inp.m.to(device)),
@@ -79,7 +79,7 @@ def oracle_flags(flags: int) -> int:
     out = 0
     for lib_bit, orc_bit in ((B.CAST_F_RESELECT, orc.F_RESELECT), (B.CAST_F_COUNT_FLIPS, orc.F_COUNT_FLIPS),
                              (B.CAST_F_META_BITMASK, orc.F_META_BITMASK), (B.CAST_F_V_KEPT_FROM_G, orc.F_V_KEPT_FROM_G),
-                             (B.CAST_F_EMIT_DENSE, orc.F_EMIT_DENSE)):
+                             (B.CAST_F_EMIT_DENSE, orc.F_EMIT_DENSE), (B.CAST_F_EMIT_COMPRESSED, orc.F_EMIT_COMPRESSED)):
         if flags & lib_bit:
             out |= orc_bit
     return out
@@ -96,7 +96,7 @@ def device_outputs(st: DeviceState, flips=None):
         w=st.w.view.cpu().numpy().reshape(rows, cols),
         m=st.m.view.cpu().numpy().reshape(rows, cols),
         v=st.v.view.cpu().numpy().reshape(rows, cols),
-        w_fwd=workloads.bf16_bits(st.w_fwd.view).reshape(rows, cols),
+        w_fwd=workloads.bf16_bits(st.w_fwd.view).reshape(rows, -1),
         meta=st.meta.view.cpu().numpy().view(np.uint32).reshape(rows, cols // 32),
     )
     if flips is not None:
@@ -105,7 +105,8 @@ def device_outputs(st: DeviceState, flips=None):
 
 
 def run_cuda_single(inp: workloads.TensorInputs, N, M, hyper: orc.Hyper, flags, meta_in=None, device="cuda:0"):
-    st = to_device(inp, device, meta_in)
+    rows_, cols_ = inp.w.shape
+    st = to_device(inp, device, meta_in, rows_ * cols_ * N // M if flags & B.CAST_F_EMIT_COMPRESSED else None)
     flips = torch.zeros(1, dtype=torch.int64, device=device) if flags & B.CAST_F_COUNT_FLIPS else None
     lr, b1, b2, eps, lam = hyper.as_f32()
     n_seg = 1 if st.scale is None else st.scale.shape[1]

@@ -88,6 +88,43 @@ def test_flags_and_scale_segments(extra, scale_mode, n_seg):
     U.assert_parity(got, U.run_oracle(inp, 2, 4, h, RS | extra), f"flags {extra} scale {scale_mode}/{n_seg}")
 
 
+@pytest.mark.parametrize("N,M", [(2, 4), (1, 4), (3, 4), (4, 4), (1, 2), (2, 2), (4, 8), (1, 8), (3, 8), (8, 8)])
+@pytest.mark.parametrize("extra", [0, BM, BM | B.CAST_F_COUNT_FLIPS | B.CAST_F_V_KEPT_FROM_G])
+def test_compressed_emission(N, M, extra):
+    """Only the kept entries are written, 8 N / M per thread: every store width (2 to 16 bytes) and the
+    odd counts, over several tiles with a ragged tail; the guard bands catch a write past the shorter buffer."""
+    if extra == 0 and (N, M) != (2, 4):
+        pytest.skip("index-form metadata is 2:4 only")
+    rows, cols = 7, 2080
+    inp = inputs(rows, cols, seed=12, idx=N * 10 + M)
+    if (cols // 2) % max(M, 8) != 0:
+        inp.scale = None
+    flags = RS | extra | B.CAST_F_EMIT_COMPRESSED
+    prev = U.run_oracle(inputs(rows, cols, seed=13), N, M, Hyper(), RS | (extra & BM))["meta"]
+    got = U.run_cuda_single(inp, N, M, Hyper(), flags, meta_in=prev)
+    ref = U.run_oracle(inp, N, M, Hyper(), flags, meta_in=prev)
+    assert got["w_fwd"].shape == (rows, cols * N // M)
+    U.assert_parity(got, ref, f"compressed {N}:{M} flags {extra}")
+
+
+def test_compressed_emission_with_a_reused_mask_and_rejections():
+    rows, cols = 6, 1056
+    inp = inputs(rows, cols, seed=14)
+    stored = U.run_oracle(inputs(rows, cols, seed=15), 2, 4, Hyper(), RS)["meta"]
+    flags = B.CAST_F_EMIT_COMPRESSED                       # no reselection: kept set decoded from the stored metadata
+    got = U.run_cuda_single(inp, 2, 4, Hyper(), flags, meta_in=stored)
+    U.assert_parity(got, U.run_oracle(inp, 2, 4, Hyper(), flags, meta_in=stored), "compressed, reused mask")
+    st = U.to_device(inp, DEV)
+    lr, b1, b2, eps, lam = Hyper().as_f32()
+    def call(N, M, fl):
+        return cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, None, 1,
+                                    rows, cols, N, M, lr, b1, b2, eps, lam, 10, 100, fl, None, None)
+    before = cast.cast_kernel_launch_count()
+    assert call(8, 16, RS | BM | B.CAST_F_EMIT_COMPRESSED) == B.CAST_ERR_NM                      # groups wider than a thread's unit
+    assert call(2, 4, RS | B.CAST_F_EMIT_COMPRESSED | B.CAST_F_EMIT_DENSE) == B.CAST_ERR_HYPER
+    assert cast.cast_kernel_launch_count() == before
+
+
 @pytest.mark.parametrize("bitmask", [False, True])
 def test_mask_reuse_and_flip_count(bitmask):
     """Kept set decoded from the stored metadata (no reselection), and flips against a previous mask."""

@@ -15,6 +15,10 @@ DEV = "cuda:0"
 RS, BM = B.CAST_F_RESELECT, B.CAST_F_META_BITMASK
 
 
+def pinned(t: torch.Tensor) -> torch.Tensor:
+    return t.contiguous().pin_memory()
+
+
 def run_plan(inputs_list, N, M, hyper: Hyper, flags, metas=None, launches=1):
     states = [U.to_device(inp, DEV, None if metas is None else metas[i]) for i, inp in enumerate(inputs_list)]
     tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale,
@@ -101,6 +105,61 @@ def test_plan_decoder_d768_12_layers_full():
     print(f"near-tie groups: {ties} of {wl.n_params // 4}; mask mismatches: 0")
 
 
+def test_compressed_plan_and_host_step():
+    """Plans made for compressed forward-weight buffers, and the host-staged step with the compressed form."""
+    shapes = [(3, 96), (64, 1056), (7, 2080), (1, 32)]
+    C = B.CAST_F_EMIT_COMPRESSED
+    ins = [workloads.gen_tensor_inputs(r, c, seed=26, tensor_index=i, scale_mode="jitter" if c % 64 == 0 else "none")
+           for i, (r, c) in enumerate(shapes)]
+    for N, M, enc in ((2, 4, 0), (4, 8, BM)):
+        states = [U.to_device(inp, DEV, None, inp.w.numel() * N // M) for inp in ins]
+        tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale,
+                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in states]
+        rc, plan = cast.cast_plan_create_ex(tensors, N, M, C)
+        cast.check(rc)
+        h = Hyper()
+        lr, b1, b2, eps, lam = h.as_f32()
+        before = cast.cast_kernel_launch_count()
+        # a step without the flag is refused: the buffers are too short for the full form
+        assert cast.cast_plan_step(plan, B.make_hyper(lr, b1, b2, eps, lam, h.step, h.total_steps, RS | enc), None, None) == B.CAST_ERR_PLAN
+        assert cast.cast_kernel_launch_count() == before
+        cast.check(cast.cast_plan_step(plan, B.make_hyper(lr, b1, b2, eps, lam, h.step, h.total_steps, RS | enc | C), None,
+                                       torch.cuda.current_stream()))
+        torch.cuda.synchronize()
+        cast.check(cast.cast_plan_destroy(plan))
+        for i, (s, inp) in enumerate(zip(states, ins)):
+            assert s.all_intact()
+            U.assert_parity(U.device_outputs(s), U.run_oracle(inp, N, M, h, RS | enc | C), f"compressed plan {N}:{M} tensor {i}")
+    # an ordinary plan refuses the flag
+    states = [U.to_device(inp, DEV) for inp in ins]
+    tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, None, 1, s.rows, s.cols) for s in states]
+    rc, plan = cast.cast_plan_create(tensors, 2, 4)
+    cast.check(rc)
+    assert cast.cast_plan_step(plan, B.make_hyper(1e-4, 0.9, 0.95, 1e-8, 1e-3, 1, 10, RS | C), None, None) == B.CAST_ERR_PLAN
+    cast.check(cast.cast_plan_destroy(plan))
+    # host-resident state, blocks of 4 rows
+    rows, cols = 37, 1024
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=33, scale_mode="jitter")
+    ref = U.run_oracle(inp, 2, 4, Hyper(), RS | C)
+    w, m, v, g, sc = pinned(inp.w), pinned(inp.m), pinned(inp.v), pinned(inp.g), pinned(inp.scale)
+    fwd = pinned(torch.zeros((rows, cols // 2), dtype=torch.bfloat16))
+    meta = pinned(torch.zeros((rows, cols // 32), dtype=torch.int32))
+    rc, ctx = cast.cast_host_ctx_create(4096, 2)
+    cast.check(rc)
+    lr, b1, b2, eps, lam = Hyper().as_f32()
+    cast.check(cast.cast_host_step(ctx, w, m, v, g, fwd, meta, sc, 2, rows, cols, 2, 4, lr, b1, b2, eps, lam, 1000, 30000, RS | C, None))
+    cast.check(cast.cast_host_ctx_destroy(ctx))
+    got = dict(w=w.numpy(), m=m.numpy(), v=v.numpy(), w_fwd=workloads.bf16_bits(fwd), meta=meta.numpy().view(np.uint32))
+    U.assert_parity(got, ref, "host blocks, compressed")
+    fwd2 = torch.zeros((rows, cols // 2), dtype=torch.bfloat16)
+    st2 = [inp.w.clone(), inp.m.clone(), inp.v.clone()]
+    meta2 = torch.zeros((rows, cols // 32), dtype=torch.int32)
+    cast.check(cast.cast_host_step_static(st2[0], st2[1], st2[2], inp.g, fwd2, meta2, inp.scale, 2, rows, cols, 2, 4,
+                                          lr, b1, b2, eps, lam, 1000, 30000, RS | C, None, None))
+    got = dict(w=st2[0].numpy(), m=st2[1].numpy(), v=st2[2].numpy(), w_fwd=workloads.bf16_bits(fwd2), meta=meta2.numpy().view(np.uint32))
+    U.assert_parity(got, ref, "static staging, compressed")
+
+
 def test_streamed_layers_on_two_streams_match_oracle():
     """Per-layer plan calls alternating on two streams over fewer resident slots than layers: 6 layers in 4
     slots, so slots 0 and 1 are stepped twice (layers 0, 4 and 1, 5) and slots 2 and 3 once."""
@@ -139,9 +198,6 @@ def test_plan_rejects_wrong_device_memory_and_survives():
 
 
 # ------------------------------------------------------------------------------- host-resident state
-
-def pinned(t: torch.Tensor) -> torch.Tensor:
-    return t.contiguous().pin_memory()
 
 
 @pytest.mark.parametrize("block,slots", [(4096, 2), (8192 * 3, 3)])
