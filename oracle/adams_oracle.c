@@ -44,6 +44,9 @@ typedef REAL real;
 #define ORACLE_F_META_BITMASK   4u   /* metadata = M-bit keep mask per group             */
 #define ORACLE_F_V_KEPT_FROM_G  8u   /* alternate reading: kept entries feed g^2 into v  */
 #define ORACLE_F_EMIT_DENSE    16u   /* forward weight is Diag(A) W without the mask     */
+#define ORACLE_F_GRAD_OF_SCALED 64u  /* g is the gradient with respect to the scaled weight Diag(A~) W~ of
+                                        Eq. 12; the chain rule gives dL/dW = A (.) g, and
+                                        dL/dA[r, s] = sum over segment s of g[r, c] W_{t-1}[r, c]         */
 #define ORACLE_F_EMIT_COMPRESSED 32u /* forward weight holds only the kept entries: rows x cols*N/M,
                                         the N kept values of each group in column order (the pruned
                                         matrix of Alg. 2's final loop without its zeros)               */
@@ -145,7 +148,8 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
           int64_t rows, int64_t cols, int N, int M,
           double lr_d, double beta1_d, double beta2_d, double eps_d, double l1_coeff_d,
           int64_t step, int64_t total_steps,
-          uint32_t flags, uint64_t *flip_count)
+          uint32_t flags, uint64_t *flip_count,
+          double *scale_grad)   /* [rows][n_seg], added to; may be NULL; used with ORACLE_F_GRAD_OF_SCALED */
 {
     if (!w || !m || !v || !g || !w_fwd || !meta) return ORACLE_BAD_ARGS;
     if (rows < 0 || cols < 0 || M < 1 || M > 32 || N < 1 || N > M) return ORACLE_BAD_ARGS;
@@ -156,6 +160,7 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
     if (!bitmask_encoding && !(N == 2 && M == 4)) return ORACLE_BAD_ARGS;
     if ((flags & ORACLE_F_COUNT_FLIPS) && !flip_count) return ORACLE_BAD_ARGS;
     if ((flags & ORACLE_F_EMIT_COMPRESSED) && (flags & ORACLE_F_EMIT_DENSE)) return ORACLE_BAD_ARGS;
+    if (scale_grad && !(flags & ORACLE_F_GRAD_OF_SCALED)) return ORACLE_BAD_ARGS;
 
     /* scalars of the step, formed in double and rounded once to the working type */
     const real alpha = (real)((double)step / (double)total_steps);   /* alpha_t = t/T   (Alg. 1) */
@@ -200,7 +205,14 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
                 const int64_t idx = base + j;
                 const int kept = (keep >> j) & 1u;
                 const real theta_prev = (real)w[idx];
-                const real grad = bf16_to_real(g[idx]);
+                real grad = bf16_to_real(g[idx]);
+                if (flags & ORACLE_F_GRAD_OF_SCALED) {
+                    /* W_scale[r, c] = A[r, s(c)] W[r, c]  (Eq. 12)  =>  dL/dA[r, s] += g W,  dL/dW = A g */
+                    const int64_t col_g = i * M + j;
+                    const int64_t seg = scale ? col_g / (cols / n_seg) : 0;
+                    if (scale_grad) scale_grad[r * (scale ? n_seg : 1) + seg] += (double)grad * (double)w[idx];
+                    if (scale) grad = (real)scale[r * n_seg + seg] * grad;
+                }
 
                 /* first moment (Alg. 1: mu_t = beta1 mu_{t-1} + (1 - beta1) g_t); stored undecayed */
                 const real mu = beta1 * (real)m[idx] + (one - beta1) * grad;

@@ -20,6 +20,7 @@ F_META_BITMASK = 4
 F_V_KEPT_FROM_G = 8
 F_EMIT_DENSE = 16
 F_EMIT_COMPRESSED = 32
+F_GRAD_OF_SCALED = 64
 
 _lib = None
 
@@ -39,7 +40,11 @@ def _load():
                 ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double,
                 ctypes.c_int64, ctypes.c_int64,                                       # step total_steps
                 ctypes.c_uint32, ctypes.c_void_p,                                     # flags flip_count
+                ctypes.c_void_p,                                                      # scale_grad
             ]
+        lib.oracle_plain_adam.restype = ctypes.c_int
+        lib.oracle_plain_adam.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                          ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int64]
         lib.oracle_mask_stats.restype = ctypes.c_int
         lib.oracle_mask_stats.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                           ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p]
@@ -65,7 +70,7 @@ class Hyper:
 
 
 def adams_step_inplace(w, m, v, g_bits, w_fwd_bits, meta, scale, rows, cols, N, M, hyper: Hyper,
-                       flags: int, precision: str = "f64") -> int:
+                       flags: int, precision: str = "f64", scale_grad=None) -> int:
     """Run the oracle in place on C-contiguous numpy arrays.
 
     w, m, v: float32 [rows*cols]; g_bits, w_fwd_bits: uint16 (raw bf16);
@@ -84,12 +89,14 @@ def adams_step_inplace(w, m, v, g_bits, w_fwd_bits, meta, scale, rows, cols, N, 
         assert scale.dtype == np.float32 and scale.flags["C_CONTIGUOUS"] and scale.shape[0] == rows
         n_seg = scale.shape[1]
         scale_ptr = scale.ctypes.data
+    if scale_grad is not None:
+        assert scale_grad.dtype == np.float64 and scale_grad.flags["C_CONTIGUOUS"] and scale_grad.size == rows * n_seg
     flips = ctypes.c_uint64(0)
     lr, b1, b2, eps, lam = hyper.as_f32()
     rc = fn(w.ctypes.data, m.ctypes.data, v.ctypes.data, g_bits.ctypes.data,
             w_fwd_bits.ctypes.data, meta.ctypes.data, scale_ptr, n_seg,
             rows, cols, N, M, lr, b1, b2, eps, lam, hyper.step, hyper.total_steps,
-            flags, ctypes.addressof(flips))
+            flags, ctypes.addressof(flips), None if scale_grad is None else scale_grad.ctypes.data)
     if rc != 0:
         raise ValueError(f"oracle rejected its arguments (status {rc})")
     return int(flips.value)
@@ -113,8 +120,11 @@ def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELE
     else:
         meta = np.ascontiguousarray(meta_in, dtype=np.uint32).copy().reshape(-1)
     sc = None if scale is None else np.ascontiguousarray(scale, dtype=np.float32)
-    flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision)
-    return dict(w=w2.reshape(rows, cols), m=m2.reshape(rows, cols), v=v2.reshape(rows, cols),
+    scale_grad = None
+    if flags & F_GRAD_OF_SCALED:
+        scale_grad = np.zeros((rows, 1 if sc is None else sc.shape[1]), dtype=np.float64)
+    flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision, scale_grad)
+    return dict(scale_grad=scale_grad, w=w2.reshape(rows, cols), m=m2.reshape(rows, cols), v=v2.reshape(rows, cols),
                 w_fwd=fwd.reshape(rows, fwd_cols), meta=meta.reshape(rows, cols // 32), flips=flips)
 
 
@@ -139,3 +149,16 @@ def mask_stats(w, meta, meta_ref, M: int, bitmask: bool):
     if rc != 0:
         raise ValueError("oracle_mask_stats rejected its arguments")
     return dict(flips=int(flips.value), kept_abs=float(sums[0]), total_abs=float(sums[1]))
+
+
+def plain_adam(theta, m, v, grad, lr, beta1, beta2, eps, step):
+    """Textbook Adam with bias correction on float32 arrays (copies returned): the optimizer of the scale matrix."""
+    lib = _load()
+    t2, m2, v2 = (np.ascontiguousarray(a, dtype=np.float32).copy() for a in (theta, m, v))
+    g2 = np.ascontiguousarray(grad, dtype=np.float32)
+    f = lambda x: float(np.float32(x))
+    rc = lib.oracle_plain_adam(t2.ctypes.data, m2.ctypes.data, v2.ctypes.data, g2.ctypes.data, t2.size,
+                               f(lr), f(beta1), f(beta2), f(eps), int(step))
+    if rc != 0:
+        raise ValueError("oracle_plain_adam rejected its arguments")
+    return t2, m2, v2

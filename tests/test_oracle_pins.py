@@ -531,3 +531,51 @@ def test_compressed_emission_hand_example():
               flags=orc.F_RESELECT | orc.F_EMIT_COMPRESSED)
     want = np.tile(np.array([-8.0, 6.0, 2.0, 2.0], dtype=np.float32), 4)            # ties: the lower columns (1.0, 1.0)
     assert np.array_equal(bf16_bits_to_f32(out["w_fwd"]).reshape(-1), want)
+
+
+# --------------------------------------------------------------------------- gradient through the scaling (Eq. 12)
+
+@pytest.mark.parametrize("n_seg", [1, 2, 4])
+def test_gradient_of_the_scaled_weight_follows_autograd(n_seg):
+    """With g the gradient of the loss with respect to W_scale = Diag(A) W, the chain rule is checked against
+    torch autograd on the linear loss <W_scale, g>: dL/dA is the oracle's scale gradient, and dL/dW is what the
+    first moment sees (m_0 = 0, so m_1 = (1 - beta1) dL/dW)."""
+    rng = np.random.default_rng(80 + n_seg)
+    rows, cols = 6, 128
+    w = rng.normal(0, 0.02, size=(rows, cols)).astype(np.float32)
+    g32, g_bits = bf16_exact(rng.normal(0, 1e-3, size=(rows, cols)))
+    scale = (1.0 + 0.5 * rng.random((rows, n_seg))).astype(np.float32)
+    A = torch.tensor(scale, dtype=torch.float64, requires_grad=True)
+    W = torch.tensor(w, dtype=torch.float64, requires_grad=True)
+    loss = ((A.repeat_interleave(cols // n_seg, dim=1) * W) * torch.tensor(g32, dtype=torch.float64)).sum()
+    loss.backward()
+    h = Hyper(beta1=0.9)
+    out = run(w, g=g_bits, scale=scale, N=2, M=4, hyper=h, flags=orc.F_RESELECT | orc.F_META_BITMASK | orc.F_GRAD_OF_SCALED)
+    assert np.allclose(out["scale_grad"], A.grad.numpy(), rtol=1e-12, atol=0)
+    b1 = float(np.float32(0.9))
+    assert np.allclose(out["m"], ((1.0 - b1) * W.grad.numpy()).astype(np.float32), rtol=1e-6, atol=0)
+    # without the flag the same g is taken as dL/dW itself, and no scale gradient is produced
+    plain = run(w, g=g_bits, scale=scale, N=2, M=4, hyper=h)
+    assert plain["scale_grad"] is None
+    assert np.allclose(plain["m"], ((1.0 - b1) * g32).astype(np.float32), rtol=1e-6, atol=0)
+    # a unit scale makes the two readings coincide
+    ones = np.ones((rows, n_seg), dtype=np.float32)
+    a = run(w, g=g_bits, scale=ones, N=2, M=4, hyper=h, flags=orc.F_RESELECT | orc.F_META_BITMASK | orc.F_GRAD_OF_SCALED)
+    b = run(w, g=g_bits, scale=ones, N=2, M=4, hyper=h)
+    for k in ("w", "m", "v", "w_fwd", "meta"):
+        assert np.array_equal(a[k], b[k])
+
+
+def test_plain_adam_for_the_scale_matches_torch():
+    rng = np.random.default_rng(90)
+    theta0 = (1.0 + 0.1 * rng.random(64)).astype(np.float32)
+    theta, m, v = theta0.copy(), np.zeros(64, np.float32), np.zeros(64, np.float32)
+    p = torch.tensor(theta0.astype(np.float64), requires_grad=True)
+    opt = torch.optim.Adam([p], lr=1e-3, betas=(float(np.float32(0.9)), float(np.float32(0.95))), eps=float(np.float32(1e-8)))
+    for t in range(1, 6):
+        grad = rng.normal(0, 1e-2, size=64).astype(np.float32)
+        theta, m, v = orc.plain_adam(theta, m, v, grad, float(np.float32(1e-3)), 0.9, 0.95, 1e-8, t)
+        p.grad = torch.tensor(grad.astype(np.float64))
+        opt.step()
+        # the oracle stores fp32 state between steps, torch keeps fp64: a few fp32 roundings per step
+        assert np.allclose(theta, p.detach().numpy(), rtol=5e-7 * t, atol=0)
