@@ -76,6 +76,11 @@ enum cast_flags {
                                        into v; entries outside the kept set still feed mu~^2           */
     CAST_F_EMIT_DENSE    = 1u << 4, /* emit Diag(A~) W~ for all entries (the dense training-time forward
                                        weight of Alg. 2) instead of the pruned product                  */
+    CAST_F_GRAD_OF_SCALED = 1u << 6, /* `g` is the gradient with respect to the scaled weight Diag(A~) W~ that the
+                                       forward pass used (Eq. 12) instead of the gradient with respect to W: the
+                                       step applies the chain rule dL/dW = A (.) g itself and, where a scale_grad
+                                       buffer is given, adds dL/dA[r, s] = sum_{c in segment s} g[r, c] W_{t-1}[r, c]
+                                       to it                                                              */
     CAST_F_EMIT_COMPRESSED = 1u << 5 /* emit only the kept entries of the pruned product (Alg. 2, final loop):
                                        w_fwd_bf16 is then [rows][cols*N/M], the N kept values of each group in
                                        column order; with the metadata it is the whole pruned matrix, and a
@@ -117,7 +122,7 @@ CAST_API int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
                     uint32_t flags, unsigned long long* flip_count,
                     cast_stream_t stream);
 
-/* One matrix of a multi-tensor plan; fields as the arguments of cast_adams_step. */
+/* One matrix of a multi-tensor plan (or of cast_adams_step_ex); fields as the arguments of cast_adams_step. */
 typedef struct cast_tensor {
     float* w; float* m; float* v;
     const cast_bf16* g;
@@ -126,6 +131,8 @@ typedef struct cast_tensor {
     const float* scale;      /* may be NULL */
     int32_t scale_groups;    /* ignored when scale is NULL */
     int64_t rows, cols;
+    float* scale_grad;       /* device, fp32 [rows][scale_groups], ADDED to by steps that carry
+                                CAST_F_GRAD_OF_SCALED (zero it before the step); may be NULL; needs `scale` */
 } cast_tensor_t;
 
 /* Hyper-parameters of one iteration (Alg. 1 inputs); ranges as in cast_adams_step. */
@@ -136,15 +143,37 @@ typedef struct cast_hyper {
 } cast_hyper_t;
 
 /*
+ * cast_adams_step_ex -- cast_adams_step with the matrix and the hyper-parameters passed as structures, which
+ * also carries the optional scale-gradient buffer of CAST_F_GRAD_OF_SCALED.  Same checks, same kernel.
+ */
+CAST_API int cast_adams_step_ex(const cast_tensor_t* tensor, int N, int M, const cast_hyper_t* hyper,
+                       unsigned long long* flip_count, cast_stream_t stream);
+
+/*
+ * cast_scale_adam_step -- the optimizer step of the scale matrix A of Eq. 12, which the paper learns jointly
+ * with the weights (Sec. 4.2) without naming its optimizer: plain Adam with bias correction (Alg. 1 without
+ * its mask and decay lines), element-wise over `n` = rows * scale_groups entries, in fp64 internally.
+ *
+ *   a, m_a, v_a   device, fp32 [n], in/out: the scale entries and their two moments.
+ *   grad          device, fp32 [n]: dL/dA as accumulated by steps with CAST_F_GRAD_OF_SCALED; set to zero
+ *                 after use when clear_grad != 0 (ready for the next iteration's accumulation).
+ *   lr finite; beta1, beta2 in [0, 1); eps > 0; step >= 1.
+ * Asynchronous on `stream`; queue it after the AdamS steps of the iteration on the same stream.
+ */
+CAST_API int cast_scale_adam_step(float* a, float* m_a, float* v_a, float* grad, int64_t n,
+                         float lr, float beta1, float beta2, float eps, int64_t step,
+                         int clear_grad, cast_stream_t stream);
+
+/*
  * Multi-tensor plan: the AdamS iteration of Alg. 1 over "each parameter theta in Theta", i.e. over
- * every prunable matrix of the model, in ONE kernel launch per 384 matrices.
+ * every prunable matrix of the model, in ONE kernel launch per 320 matrices.
  *
  * cast_plan_create  validates `n_tensors` descriptors (host array, copied) and returns an opaque handle
  *                   in *plan_out.  The plan is host memory only: it holds the launch tables, which travel
  *                   to the device as kernel parameters at every step, and allocates nothing on the
  *                   device.  All matrices share N:M.  The buffers named by the descriptors stay owned by
  *                   the caller and must outlive the plan's use.
- * cast_plan_step    launches one grid over all matrices on `stream` (ceil(n_tensors / 384) grids for
+ * cast_plan_step    launches one grid over all matrices on `stream` (ceil(n_tensors / 320) grids for
  *                   larger lists); arguments as cast_adams_step.  The plan may be stepped any number of
  *                   times, on any stream of its device; two steps of one plan must not overlap in time
  *                   (they update the same state).
@@ -219,7 +248,7 @@ CAST_API int cast_mask_stats(const float* w, const uint32_t* meta, const uint32_
                     cast_mask_stats_t* stats, cast_stream_t stream);
 
 /*
- * cast_plan_mask_stats -- cast_mask_stats over every matrix of a plan in one launch (per 384 matrices), with
+ * cast_plan_mask_stats -- cast_mask_stats over every matrix of a plan in one launch (per 320 matrices), with
  * the weights and masks the plan's descriptors name.  `meta_ref` is a HOST array of n_tensors device pointers
  * (the reference mask of each matrix, same shape and form as its mask), or NULL for no reference.  `flags`
  * is CAST_F_META_BITMASK or 0 and must name the form the plan's steps write.  `stats` as in cast_mask_stats.

@@ -33,9 +33,10 @@ CAST_F_META_BITMASK = 1 << 2
 CAST_F_V_KEPT_FROM_G = 1 << 3
 CAST_F_EMIT_DENSE = 1 << 4
 CAST_F_EMIT_COMPRESSED = 1 << 5
+CAST_F_GRAD_OF_SCALED = 1 << 6
 
 EXPORTS = (
-    "cast_adams_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
+    "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
@@ -54,6 +55,7 @@ class cast_tensor_t(ctypes.Structure):
         ("g", ctypes.c_void_p), ("w_fwd", ctypes.c_void_p), ("meta", ctypes.c_void_p),
         ("scale", ctypes.c_void_p), ("scale_groups", ctypes.c_int32),
         ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+        ("scale_grad", ctypes.c_void_p),
     ]
 
 
@@ -90,6 +92,12 @@ def load_library() -> ctypes.CDLL:
     lib = ctypes.CDLL(LIB_PATH)
     lib.cast_adams_step.restype = ctypes.c_int
     lib.cast_adams_step.argtypes = _STEP_ARGS + [ctypes.c_void_p]
+    lib.cast_adams_step_ex.restype = ctypes.c_int
+    lib.cast_adams_step_ex.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.POINTER(cast_hyper_t),
+                                       ctypes.c_void_p, ctypes.c_void_p]
+    lib.cast_scale_adam_step.restype = ctypes.c_int
+    lib.cast_scale_adam_step.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_float,
+                                                                 ctypes.c_float, ctypes.c_int64, ctypes.c_int, ctypes.c_void_p]
     lib.cast_plan_create.restype = ctypes.c_int
     lib.cast_plan_create.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                      ctypes.POINTER(ctypes.c_void_p)]
@@ -174,9 +182,21 @@ def cast_adams_step(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, col
         int(flags), _ptr(flip_count), _stream(stream))
 
 
-def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols) -> cast_tensor_t:
+def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols, scale_grad=None) -> cast_tensor_t:
     return cast_tensor_t(_ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd), _ptr(meta), _ptr(scale),
-                         int(scale_groups), int(rows), int(cols))
+                         int(scale_groups), int(rows), int(cols), _ptr(scale_grad))
+
+
+def cast_adams_step_ex(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: Optional[cast_hyper_t],
+                       flip_count=None, stream=None) -> int:
+    t = ctypes.byref(tensor) if tensor is not None else None
+    h = ctypes.byref(hyper) if hyper is not None else None
+    return load_library().cast_adams_step_ex(t, int(N), int(M), h, _ptr(flip_count), _stream(stream))
+
+
+def cast_scale_adam_step(a, m_a, v_a, grad, n, lr, beta1, beta2, eps, step, clear_grad=True, stream=None) -> int:
+    return load_library().cast_scale_adam_step(_ptr(a), _ptr(m_a), _ptr(v_a), _ptr(grad), int(n), lr, beta1, beta2, eps,
+                                               int(step), 1 if clear_grad else 0, _stream(stream))
 
 
 def cast_plan_create(tensors: Sequence[cast_tensor_t], N: int, M: int):

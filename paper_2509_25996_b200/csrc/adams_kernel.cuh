@@ -36,6 +36,7 @@ constexpr uint32_t kMetaBitmask = 1u << 2;
 constexpr uint32_t kVKeptFromG = 1u << 3;
 constexpr uint32_t kEmitDense = 1u << 4;
 constexpr uint32_t kEmitCompressed = 1u << 5;
+constexpr uint32_t kGradOfScaled = 1u << 6;
 
 // Kernel modes: the flag word is a compile-time constant in the two common cases.
 constexpr int kModeGeneric = 0;        // any flags, read from StepConsts at run time
@@ -51,6 +52,7 @@ struct TensorDesc {
     uint16_t* w_fwd;
     uint32_t* meta;
     const float* scale;        // A[rows][n] or nullptr
+    float* scale_grad;         // dL/dA[rows][n], added to, or nullptr
     uint32_t n_units;          // rows * cols / 8
     uint32_t seg_magic;        // unit / seg_units == (uint64(unit) * seg_magic) >> seg_shift
     uint32_t seg_shift;
@@ -198,7 +200,7 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
 // roundings of 2^-24), i.e. below 2.5e-10 absolute for updates up to 5e-4, which is under both the
 // fp32 spacing of typical weights (1.9e-9 at 0.02) and the 1e-9 floor of the accepted error.
 template <int M, int MODE>
-__device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a)
+__device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a, float& gw_sum)
 {
     static_assert(MODE != kModeSelectIdx || M == 4, "index-form metadata is 2:4 only");
     const uint32_t flags = mode_flags<MODE>(c);
@@ -231,12 +233,20 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
     const bool v_from_g = (flags & kVKeptFromG) != 0;
     const bool dense = (flags & kEmitDense) != 0;
     const int sign_hi = __double2hiint(c.c_sign), sign_lo = __double2loint(c.c_sign);
+    // With kGradOfScaled the gradient is taken with respect to W_scale = Diag(A) W (Eq. 12): the chain rule
+    // gives dL/dW = A g (formed exactly in fp64) and dL/dA = sum of g W over the row segment, whose part
+    // for this unit is returned in gw_sum (fp32 chain of 8 fused multiply-adds on the weights before the update).
+    const bool of_scaled = (flags & kGradOfScaled) != 0;
+    const double omb1_g = of_scaled ? c.omb1 * (double)a : c.omb1;
+    gw_sum = 0.0f;
     float fwd[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        const float g32 = __uint_as_float((i & 1) ? (gw[i >> 1] & 0xFFFF0000u) : (gw[i >> 1] << 16));
+        float g32 = __uint_as_float((i & 1) ? (gw[i >> 1] & 0xFFFF0000u) : (gw[i >> 1] << 16));
+        if (of_scaled) gw_sum = fmaf(g32, u.w[i], gw_sum);
         // first moment, stored undecayed (Alg. 1)
-        const double mu = fma(c.beta1, (double)u.m[i], c.omb1 * (double)g32);
+        const double mu = fma(c.beta1, (double)u.m[i], omb1_g * (double)g32);
+        if (of_scaled) g32 *= a;                 // only the alternate reading of v below still uses g itself
         const float mu_f = (float)mu;
         u.m[i] = mu_f;
         // proportional L1 decay outside the kept set (Eq. 7): alpha lambda Sign(w), Sign(+-0) = 0
@@ -274,6 +284,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
     const uint32_t flags = mode_flags<MODE>(c);
     const bool need_prev = ((flags & kReselect) == 0) || (flags & kCountFlips);
     float a = 1.0f;
+    uint32_t seg = 0;
 
     if (active) {
         const float4 w0 = ld_f4(t.w + e), w1 = ld_f4(t.w + e + 4);
@@ -282,7 +293,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         u.g = *reinterpret_cast<const uint4*>(t.g + e);
         if (need_prev) u.prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[unit];
         if (t.scale != nullptr) {
-            const uint32_t seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
+            seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
             a = __ldg(t.scale + seg);
         }
         u.w[0] = w0.x; u.w[1] = w0.y; u.w[2] = w0.z; u.w[3] = w0.w; u.w[4] = w1.x; u.w[5] = w1.y; u.w[6] = w1.z; u.w[7] = w1.w;
@@ -293,7 +304,25 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         for (int i = 0; i < 8; ++i) { u.w[i] = 0.f; u.m[i] = 0.f; u.v[i] = 0.f; }
     }
 
-    const uint32_t flips = compute_unit<M, MODE>(u, c, a);
+    float gw_sum;
+    const uint32_t flips = compute_unit<M, MODE>(u, c, a, gw_sum);
+    if constexpr (MODE == kModeGeneric) {
+        if ((flags & kGradOfScaled) && t.scale_grad != nullptr) {     // uniform over the CTA: all lanes shuffle
+            // Sum gw_sum over the lanes of the warp that share a row segment (segments are runs of consecutive
+            // lanes), then one atomic per run.  Lanes without data carry a segment of their own and add nothing.
+            const unsigned lane = threadIdx.x & 31u;
+            const uint32_t my_seg = active ? seg : 0xFFFFFFFFu;
+            float p = active ? gw_sum : 0.0f;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const float q = __shfl_up_sync(0xFFFFFFFFu, p, d);
+                const uint32_t s = __shfl_up_sync(0xFFFFFFFFu, my_seg, d);
+                if (lane >= (unsigned)d && s == my_seg) p += q;
+            }
+            const uint32_t next_seg = __shfl_down_sync(0xFFFFFFFFu, my_seg, 1);
+            if (active && (lane == 31u || next_seg != my_seg)) atomicAdd(t.scale_grad + seg, p);
+        }
+    }
 
     if (active) {
         st_f4(t.w + e, make_float4(u.w[0], u.w[1], u.w[2], u.w[3]));
@@ -337,7 +366,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
 // tiles): tile_start[k] is the first tile of matrix k, tile_start[n] the total.
 // hint[b >> hint_shift] is the matrix that holds tile (b >> hint_shift) << hint_shift, from which the
 // CTA walks forward (usually zero or one step).
-constexpr int kMaxLaunchTensors = 384;
+constexpr int kMaxLaunchTensors = 320;
 constexpr int kHintEntries = 256;
 struct MultiParams {
     uint32_t n_tensors;

@@ -28,7 +28,8 @@ int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count)
     if (N < 1 || N > M) return CAST_ERR_NM;
     if (!(flags & CAST_F_META_BITMASK) && !(N == 2 && M == 4)) return CAST_ERR_NM;
     const uint32_t known = CAST_F_RESELECT | CAST_F_COUNT_FLIPS | CAST_F_META_BITMASK |
-                           CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE | CAST_F_EMIT_COMPRESSED;
+                           CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE | CAST_F_EMIT_COMPRESSED |
+                           CAST_F_GRAD_OF_SCALED;
     if (flags & ~known) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && (flags & CAST_F_EMIT_DENSE)) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && M > kUnitElems) return CAST_ERR_NM;
@@ -103,6 +104,22 @@ int check_pointers(const void* w, const void* m, const void* v, const void* g, c
     return CAST_OK;
 }
 
+int check_scale_grad(const float* scale_grad, const float* scale, int scale_groups, int64_t rows,
+                     const void* const* others, const uint64_t* other_bytes, int n_others)
+{
+    if (!scale_grad) return CAST_OK;
+    if (!scale) return CAST_ERR_NULL;
+    if ((uintptr_t)scale_grad & 15u) return CAST_ERR_ALIGN;
+    const Range r = {(uintptr_t)scale_grad, (uintptr_t)scale_grad + 4ull * (uint64_t)rows * (uint64_t)scale_groups};
+    for (int i = 0; i < n_others; ++i) {
+        if (!others[i]) continue;
+        const Range o = {(uintptr_t)others[i], (uintptr_t)others[i] + other_bytes[i]};
+        if (overlap(r, o)) return CAST_ERR_ALIAS;
+    }
+    const void* p[1] = {scale_grad};
+    return check_device_memory(p, 1);
+}
+
 int check_device_memory(const void* const* ptrs, int n)
 {
     for (int i = 0; i < n; ++i) {
@@ -126,11 +143,12 @@ static void fast_div(uint32_t d, uint32_t* magic, uint32_t* shift)
 }
 
 TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
-                     const float* scale, int scale_groups, int64_t rows, int64_t cols)
+                     const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad)
 {
     TensorDesc d;
     std::memset(&d, 0, sizeof d);
     d.w = w; d.m = m; d.v = v; d.g = g; d.w_fwd = w_fwd; d.meta = meta; d.scale = scale;
+    d.scale_grad = scale ? scale_grad : nullptr;
     d.n_units = (uint32_t)((uint64_t)rows * (uint64_t)cols / kUnitElems);
     if (scale) {
         const uint32_t seg_units = (uint32_t)(cols / scale_groups / kUnitElems);
@@ -309,6 +327,38 @@ extern "C" int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
     return launch_single(d, M, c, flip_count, (cudaStream_t)stream);
 }
 
+namespace {
+// Checks of one matrix descriptor beyond what check_shape / check_pointers do: the scale-gradient buffer.
+int check_tensor_scale_grad(const cast_tensor_t& t, int N, int M, uint32_t fwd_flags)
+{
+    const uint64_t P = (uint64_t)t.rows * (uint64_t)t.cols;
+    const void* others[7] = {t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale};
+    const uint64_t bytes[7] = {4 * P, 4 * P, 4 * P, 2 * P, 2 * fwd_elems_of(t.rows, t.cols, N, M, fwd_flags), P / 8,
+                               t.scale ? 4ull * (uint64_t)t.rows * (uint64_t)t.scale_groups : 0};
+    return check_scale_grad(t.scale_grad, t.scale, t.scale_groups, t.rows, others, bytes, 7);
+}
+}  // namespace
+
+extern "C" int cast_adams_step_ex(const cast_tensor_t* t, int N, int M, const cast_hyper_t* h,
+                                  unsigned long long* flip_count, cast_stream_t stream)
+{
+    if (!t || !h) return CAST_ERR_NULL;
+    int rc;
+    if ((rc = check_nm_flags(N, M, h->flags, flip_count)) != CAST_OK) return rc;
+    StepConsts c;
+    if ((rc = make_step_consts(h->lr, h->beta1, h->beta2, h->eps, h->l1_coeff, h->step, h->total_steps, N, h->flags, &c)) != CAST_OK) return rc;
+    if (!t->w || !t->m || !t->v || !t->g || !t->w_fwd || !t->meta) return CAST_ERR_NULL;
+    if ((rc = check_shape(t->rows, t->cols, M, t->scale != nullptr, t->scale_groups)) != CAST_OK) return rc;
+    if ((rc = check_pointers(t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, t->scale_groups, t->rows, t->cols,
+                             fwd_elems_of(t->rows, t->cols, N, M, h->flags))) != CAST_OK) return rc;
+    const void* ptrs[8] = {t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, (h->flags & CAST_F_COUNT_FLIPS) ? flip_count : nullptr};
+    if ((rc = check_device_memory(ptrs, 8)) != CAST_OK) return rc;
+    if ((rc = check_tensor_scale_grad(*t, N, M, h->flags)) != CAST_OK) return rc;
+    const TensorDesc d = make_desc(t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, t->scale_groups, t->rows, t->cols,
+                                   t->scale_grad);
+    return launch_single(d, M, c, flip_count, (cudaStream_t)stream);
+}
+
 extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out)
 {
     return cast_plan_create_ex(tensors, n_tensors, N, M, 0u, plan_out);
@@ -337,6 +387,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
         const cast_tensor_t& t = tensors[i];
         const void* ptrs[7] = {t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale};
         if ((rc = check_device_memory(ptrs, 7)) != CAST_OK) return rc;
+        if ((rc = check_tensor_scale_grad(t, N, M, plan_flags)) != CAST_OK) return rc;
     }
 
     Plan* p = new (std::nothrow) Plan;
@@ -354,7 +405,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
             uint64_t tiles = 0;
             while (i < n_tensors && mp.n_tensors < (uint32_t)kMaxLaunchTensors) {
                 const cast_tensor_t& t = tensors[i];
-                const TensorDesc d = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols);
+                const TensorDesc d = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols, t.scale_grad);
                 if (tiles + tiles_of(d) > kMaxTiles) break;      // a single matrix always fits (rows*cols < 2^31)
                 mp.desc[mp.n_tensors] = d;
                 mp.tile_start[mp.n_tensors] = (uint32_t)tiles;

@@ -49,7 +49,12 @@ int check_device_memory(const void* const* ptrs, int n);
 
 // Kernel-side description of one (already validated) matrix.
 TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
-                     const float* scale, int scale_groups, int64_t rows, int64_t cols);
+                     const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad = nullptr);
+
+// The optional scale-gradient buffer of one matrix: needs a scale, 16-byte alignment, device memory, no overlap
+// with the matrix's other buffers (checked by address only).
+int check_scale_grad(const float* scale_grad, const float* scale, int scale_groups, int64_t rows,
+                     const void* const* others, const uint64_t* other_bytes, int n_others);
 
 inline uint32_t tiles_of(const TensorDesc& d) { return (d.n_units + kTileUnits - 1) / kTileUnits; }
 

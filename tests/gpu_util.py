@@ -79,7 +79,8 @@ def oracle_flags(flags: int) -> int:
     out = 0
     for lib_bit, orc_bit in ((B.CAST_F_RESELECT, orc.F_RESELECT), (B.CAST_F_COUNT_FLIPS, orc.F_COUNT_FLIPS),
                              (B.CAST_F_META_BITMASK, orc.F_META_BITMASK), (B.CAST_F_V_KEPT_FROM_G, orc.F_V_KEPT_FROM_G),
-                             (B.CAST_F_EMIT_DENSE, orc.F_EMIT_DENSE), (B.CAST_F_EMIT_COMPRESSED, orc.F_EMIT_COMPRESSED)):
+                             (B.CAST_F_EMIT_DENSE, orc.F_EMIT_DENSE), (B.CAST_F_EMIT_COMPRESSED, orc.F_EMIT_COMPRESSED),
+                             (B.CAST_F_GRAD_OF_SCALED, orc.F_GRAD_OF_SCALED)):
         if flags & lib_bit:
             out |= orc_bit
     return out

@@ -31,7 +31,7 @@ def run_plan(inputs_list, N, M, hyper: Hyper, flags, metas=None, launches=1):
     cast.check(cast.cast_plan_step(plan, B.make_hyper(lr, b1, b2, eps, lam, hyper.step, hyper.total_steps, flags),
                                    flips, torch.cuda.current_stream()))
     torch.cuda.synchronize()
-    assert cast.cast_kernel_launch_count() == before + launches   # one grid covers up to 384 matrices
+    assert cast.cast_kernel_launch_count() == before + launches   # one grid covers up to 320 matrices
     cast.check(cast.cast_plan_destroy(plan))
     assert all(s.all_intact() for s in states)
     return [U.device_outputs(s) for s in states], (None if flips is None else int(flips.item()))
@@ -67,7 +67,7 @@ def test_plan_many_small_matrices_around_a_large_one():
 
 
 def test_plan_more_matrices_than_one_launch_holds():
-    """A launch carries the descriptors of at most 384 matrices: 400 small matrices take two launches."""
+    """A launch carries the descriptors of at most 320 matrices: 400 small matrices take two launches."""
     shapes = [(1 + i % 3, 32 * (1 + i % 5)) for i in range(400)]
     ins = [workloads.gen_tensor_inputs(r, c, seed=25, tensor_index=i, scale_mode="none") for i, (r, c) in enumerate(shapes)]
     fl = RS | B.CAST_F_COUNT_FLIPS
