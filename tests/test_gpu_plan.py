@@ -8,6 +8,7 @@ from paper_2509_25996_b200 import binding as B
 from paper_2509_25996_b200 import workloads
 from oracle.adams_oracle import Hyper
 import gpu_util as U
+from helpers import within_tol
 
 pytestmark = pytest.mark.gpu
 
@@ -103,6 +104,45 @@ def test_plan_decoder_d768_12_layers_full():
         U.assert_parity(got[i], U.run_oracle(inp, 2, 4, h, RS), f"tensor {i} {wl.shapes[i]}")
         ties += U.near_tie_groups(inp.w.numpy(), 2, 4)
     print(f"near-tie groups: {ties} of {wl.n_params // 4}; mask mismatches: 0")
+
+
+def test_plan_step_replayed_from_a_cuda_graph():
+    """A plan step is one kernel launch whose tables travel as parameters, so it can be recorded into a CUDA graph
+    and replayed: three replays are three iterations with the recorded hyper-parameters."""
+    shapes = [(64, 1056), (7, 2080), (33, 2048)]
+    ins = [workloads.gen_tensor_inputs(r, c, seed=27, tensor_index=i, scale_mode="jitter" if c % 64 == 0 else "none")
+           for i, (r, c) in enumerate(shapes)]
+    states = [U.to_device(inp, DEV) for inp in ins]
+    tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale,
+                             1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in states]
+    rc, plan = cast.cast_plan_create(tensors, 2, 4)
+    cast.check(rc)
+    h = Hyper()
+    lr, b1, b2, eps, lam = h.as_f32()
+    hs = B.make_hyper(lr, b1, b2, eps, lam, h.step, h.total_steps, RS)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        cast.check(cast.cast_plan_step(plan, hs, None, torch.cuda.current_stream()))
+    launches = cast.cast_kernel_launch_count()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == launches              # replays launch from the graph, not through the library
+    for i, (s, inp) in enumerate(zip(states, ins)):
+        cur = inp
+        for _ in range(3):
+            ref = U.run_oracle(cur, 2, 4, h, RS)
+            cur = workloads.TensorInputs(torch.from_numpy(ref["w"]), inp.g, torch.from_numpy(ref["m"]), torch.from_numpy(ref["v"]), inp.scale)
+        assert s.all_intact()
+        got = U.device_outputs(s)
+        # three chained steps: the fp32 state of step k feeds step k + 1, so the comparison is of the last step
+        # given slightly different inputs; bounds scale with the step count
+        for k in ("w", "m", "v"):
+            ok, worst = within_tol(got[k], ref[k], rel=3e-6, floor=3e-9)
+            assert ok, f"graph replay tensor {i} {k}: {worst:.3g}"
+    cast.check(cast.cast_plan_destroy(plan))
 
 
 def test_compressed_plan_and_host_step():
