@@ -42,6 +42,9 @@ def _load():
                 ctypes.c_uint32, ctypes.c_void_p,                                     # flags flip_count
                 ctypes.c_void_p,                                                      # scale_grad
             ]
+        lib.oracle_prune_fold.restype = ctypes.c_int
+        lib.oracle_prune_fold.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_uint32]
         lib.oracle_plain_adam.restype = ctypes.c_int
         lib.oracle_plain_adam.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                           ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int64]
@@ -162,3 +165,21 @@ def plain_adam(theta, m, v, grad, lr, beta1, beta2, eps, step):
     if rc != 0:
         raise ValueError("oracle_plain_adam rejected its arguments")
     return t2, m2, v2
+
+
+def prune_fold(w, scale, N, M, flags: int = F_RESELECT, meta_in=None):
+    """Final pruning with the scale folded in (Alg. 2, final loop).  flags: F_RESELECT, F_META_BITMASK,
+    F_EMIT_COMPRESSED.  Returns dict(out (uint16 bf16 bits, [rows, cols] or [rows, cols*N/M]), meta)."""
+    lib = _load()
+    rows, cols = w.shape
+    w = np.ascontiguousarray(w, dtype=np.float32)
+    meta = np.zeros(rows * cols // 32, dtype=np.uint32) if meta_in is None else \
+        np.ascontiguousarray(meta_in, dtype=np.uint32).copy().reshape(-1)
+    ocols = cols * N // M if flags & F_EMIT_COMPRESSED else cols
+    out = np.zeros(rows * ocols, dtype=np.uint16)
+    sc = None if scale is None else np.ascontiguousarray(scale, dtype=np.float32)
+    rc = lib.oracle_prune_fold(w.ctypes.data, None if sc is None else sc.ctypes.data, 1 if sc is None else sc.shape[1],
+                               meta.ctypes.data, out.ctypes.data, rows, cols, N, M, flags)
+    if rc != 0:
+        raise ValueError("oracle_prune_fold rejected its arguments")
+    return dict(out=out.reshape(rows, ocols), meta=meta.reshape(rows, cols // 32))

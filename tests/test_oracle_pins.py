@@ -579,3 +579,44 @@ def test_plain_adam_for_the_scale_matches_torch():
         opt.step()
         # the oracle stores fp32 state between steps, torch keeps fp64: a few fp32 roundings per step
         assert np.allclose(theta, p.detach().numpy(), rtol=5e-7 * t, atol=0)
+
+
+# --------------------------------------------------------------------------- final pruning (Alg. 2, final loop)
+
+@pytest.mark.parametrize("N,M,bitmask", [(2, 4, False), (2, 4, True), (1, 4, True), (4, 8, True), (3, 4, True), (5, 16, True), (8, 32, True)])
+def test_final_pruning_against_stable_argsort_and_library_bf16(N, M, bitmask):
+    """Kept set by numpy's stable sort of -|w| (equal magnitudes keep column order), values by torch's bf16
+    conversion of the fp32 product, the two output layouts by gather/scatter through the decoded mask."""
+    rng = np.random.default_rng(100 + M + N)
+    rows, cols = 6, 192
+    w = adversarial_groups(rng, rows * cols // M, M).reshape(rows, cols)
+    scale = np.ldexp(1.0, rng.integers(-2, 3, size=(rows, 2))).astype(np.float32)      # powers of two: a*w is exact in fp32
+    enc = orc.F_META_BITMASK if bitmask else 0
+    dense = orc.prune_fold(w, scale, N, M, orc.F_RESELECT | enc)
+    order = np.argsort(-np.abs(w.reshape(-1, M)), axis=1, kind="stable")[:, :N]
+    want_keep = np.zeros((rows * cols // M, M), dtype=bool)
+    np.put_along_axis(want_keep, order, True, axis=1)
+    want_keep = want_keep.reshape(rows, cols)
+    assert np.array_equal(keep_mask_from_meta(dense["meta"], cols, M, bitmask), want_keep)
+    a_full = np.repeat(scale, cols // 2, axis=1)
+    want = np.where(want_keep, torch_bf16_bits(a_full * w), 0).astype(np.uint16)
+    assert np.array_equal(dense["out"], want)
+    comp = orc.prune_fold(w, scale, N, M, orc.F_RESELECT | enc | orc.F_EMIT_COMPRESSED)
+    assert np.array_equal(comp["meta"], dense["meta"])
+    assert np.array_equal(comp["out"].reshape(-1), want[want_keep])
+    # a stored mask is used as it is, whatever the weights are now
+    other = rng.normal(0, 1, size=(rows, cols)).astype(np.float32)
+    reuse = orc.prune_fold(other, None, N, M, enc, meta_in=dense["meta"])
+    assert np.array_equal(reuse["meta"], dense["meta"])
+    assert np.array_equal(reuse["out"], np.where(want_keep, torch_bf16_bits(other), 0).astype(np.uint16))
+
+
+def test_final_pruning_is_the_step_emission_of_unmoved_weights():
+    """Consistency of the two oracles: with a zero learning rate the AdamS step leaves W alone, and its emitted
+    forward weight is the final pruning of W."""
+    rng = np.random.default_rng(110)
+    w = rng.normal(0, 0.02, size=(4, 128)).astype(np.float32)
+    scale = (1.0 + 0.1 * rng.random((4, 2))).astype(np.float32)
+    step = run(w, scale=scale, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT)
+    pf = orc.prune_fold(w, scale, 2, 4, orc.F_RESELECT)
+    assert np.array_equal(step["w_fwd"], pf["out"]) and np.array_equal(step["meta"], pf["meta"])
