@@ -54,7 +54,7 @@ def parse_args():
     p.add_argument("--e2e-steps", type=int, default=4)
     p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
     p.add_argument("--seed", type=int, default=0)
-    p.add_argument("--op", choices=["step", "mask_stats"], default="step",
+    p.add_argument("--op", choices=["step", "mask_stats", "prune_fold"], default="step",
                    help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass")
     return p.parse_args()
 
@@ -529,10 +529,76 @@ def stats_arm(args):
         "parity": {"ok": bool(ok), "sample": "first matrix against the CPU oracle"}}), flush=True)
 
 
+def prune_arm(args):
+    """The final pruning of Alg. 2 (cast_prune_fold, one launch per matrix) over the workload: 4 B read and
+    2 (compressed: 2 N / M) + 1/8 B written per parameter.  It runs once, at the end of training."""
+    import numpy as np
+    import torch
+    import paper_2509_25996_b200 as cast
+    from paper_2509_25996_b200 import binding as B
+    from paper_2509_25996_b200 import workloads
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    N, M = (int(x) for x in args.nm.split(":"))
+    wl = workloads.workload(args.workload)
+    compressed = args.emit == "compressed"
+    flags = B.CAST_F_RESELECT | (0 if (N, M) == (2, 4) else B.CAST_F_META_BITMASK) | (B.CAST_F_EMIT_COMPRESSED if compressed else 0)
+    mats = []
+    for i, (r, c) in enumerate(wl.shapes):
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(workloads.tensor_seed(args.seed, i, 0))
+        w = torch.randn((r, c), generator=gen, device=dev, dtype=torch.float32).mul_(workloads.W_STD)
+        mats.append((w, torch.ones((r, 2), device=dev), torch.zeros((r, c // 32), dtype=torch.int32, device=dev),
+                     torch.empty(r * c * N // M if compressed else r * c, dtype=torch.bfloat16, device=dev), r, c))
+    stream = torch.cuda.current_stream(dev)
+
+    def one_pass():
+        for w, sc, meta, out, r, c in mats:
+            cast.check(cast.cast_prune_fold(w, sc, 2, meta, out, r, c, N, M, flags, stream))
+
+    for _ in range(args.warmup):
+        one_pass()
+    torch.cuda.synchronize(dev)
+    launches0 = cast.cast_kernel_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        one_pass()
+    ev1.record(stream)
+    torch.cuda.synchronize(dev)
+    torch.cuda.profiler.stop()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    launches = cast.cast_kernel_launch_count() - launches0
+    from oracle import adams_oracle as orc
+    w, sc, meta, out, r, c = mats[0]
+    rows = 64
+    ref = orc.prune_fold(w[:rows].cpu().numpy(), sc[:rows].cpu().numpy(), N, M,
+                         orc.F_RESELECT | (0 if (N, M) == (2, 4) else orc.F_META_BITMASK) | (orc.F_EMIT_COMPRESSED if compressed else 0))
+    ocols = out.numel() // r
+    got = workloads.bf16_bits(out.view(r, ocols)[:rows])
+    ok = bool(np.array_equal(got, ref["out"]) and np.array_equal(meta[:rows].cpu().numpy().view(np.uint32), ref["meta"]))
+    bpp = 4.125 + (2.0 * N / M if compressed else 2.0)
+    gbs = wl.n_params * bpp / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    print(json.dumps({
+        "metric": "final pruning (Alg. 2) params/s", "value": wl.n_params / (ms * 1e-3), "unit": "params/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": wl.name, "nm": args.nm, "params": wl.n_params, "matrices": len(wl.shapes), "emit": args.emit,
+                   "l2": "inputs far larger than L2, no flush"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
+                     "kernel": f"prune_fold_kernel<{M}>", "bytes_per_param": bpp, "launches_per_step": launches // args.steps, "traffic": None},
+        "parity": {"ok": ok, "sample": f"first {rows} rows of the first matrix against the CPU oracle (unit scale: bit-exact)"}}), flush=True)
+
+
 def main():
     args = parse_args()
     if args.op == "mask_stats" and args.impl != "reference":
         return stats_arm(args)
+    if args.op == "prune_fold" and args.impl != "reference":
+        return prune_arm(args)
     if args.impl == "reference":
         reference_arm(args)
     else:

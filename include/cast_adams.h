@@ -219,6 +219,23 @@ CAST_API int cast_host_ctx_sync(void* ctx);
 CAST_API int cast_host_ctx_destroy(void* ctx);
 
 /*
+ * cast_prune_fold -- the final pruning of Alg. 2 (its last loop; the last lines of Alg. 1): W^ = W (.) M with the
+ * scale of Eq. 12 folded into the weights, as bf16.  No optimizer state is read or written.
+ *
+ *   w        device, fp32 [rows*cols]: the trained weights.
+ *   scale    device, fp32 [rows][scale_groups] or NULL (A = 1); shape rules as cast_adams_step.
+ *   meta     device, uint32 [rows*cols/32], in/out: with CAST_F_RESELECT the mask is chosen now from |w| (Eq. 6,
+ *            exactly N per group, ties to the lower column) and written; without it the stored mask is used
+ *            (and rewritten unchanged).
+ *   out      device, bf16 [rows*cols] (pruned slots +0.0), or with CAST_F_EMIT_COMPRESSED [rows*cols*N/M], the N
+ *            kept values of each group in column order (M <= 8).  Values are bf16(A * w), round to nearest even.
+ *   flags    OR of CAST_F_RESELECT, CAST_F_META_BITMASK (required unless N:M == 2:4), CAST_F_EMIT_COMPRESSED.
+ * Asynchronous on `stream`.  Errors as cast_adams_step; nothing is launched on an error.
+ */
+CAST_API int cast_prune_fold(const float* w, const float* scale, int scale_groups, uint32_t* meta, cast_bf16* out,
+                    int64_t rows, int64_t cols, int N, int M, uint32_t flags, cast_stream_t stream);
+
+/*
  * cast_mask_stats -- the mask statistics the paper monitors during training (App. C), for one matrix:
  *
  *   mask_diff      += ||M - M_ref||_0   numerator of the flip rate r_t when M_ref is the previous mask, of the

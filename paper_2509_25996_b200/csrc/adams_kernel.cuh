@@ -170,6 +170,29 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return r;
 }
 
+// Compressed form of the forward weight: only the kept entries, in column order, 8 N / M per unit (M <= 8).
+// `packed` holds the unit's 8 bf16 values.  Every group keeps exactly N, so the slot of a kept column is the
+// number of kept columns before it in the unit.  The values are scattered into a private 16-byte row of
+// shared memory and read back as a vector (16, 8 or 4 bytes; other counts go out as 2-byte stores).
+template <int M>
+__device__ __forceinline__ void store_kept_values(uint16_t* base, uint32_t unit, uint32_t keep, uint4 packed, int n_keep)
+{
+    __shared__ __align__(16) uint16_t s_comp[kThreads * 8];
+    uint16_t* mine = s_comp + threadIdx.x * 8;
+    const uint32_t hw[4] = {packed.x, packed.y, packed.z, packed.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        if ((keep >> i) & 1u)
+            mine[__popc(keep & ((1u << i) - 1u))] = (uint16_t)(hw[i >> 1] >> (16 * (i & 1)));
+    const uint32_t cnt = (uint32_t)(8 * n_keep) / (uint32_t)M;
+    uint16_t* dst = base + (size_t)unit * cnt;
+    if (cnt == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(mine);
+    else if (cnt == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(mine);
+    else if (cnt == 2) *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(mine);
+    else
+        for (uint32_t k = 0; k < cnt; ++k) dst[k] = mine[k];
+}
+
 // Registers of one unit: state and gradient in, updated state, forward weight and metadata out.
 struct UnitRegs {
     float w[8], m[8], v[8];
@@ -336,23 +359,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         if (!compressed) {
             *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
         } else {
-            // Compressed form: only the kept entries, in column order, 8 N / M per unit.  Every group keeps
-            // exactly N, so the slot of a kept column is the number of kept columns before it in the unit.
-            // The values are scattered into a private 16-byte row of shared memory and read back as a vector.
-            __shared__ __align__(16) uint16_t s_comp[kThreads * 8];
-            uint16_t* mine = s_comp + threadIdx.x * 8;
-            const uint32_t hw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                if ((u.keep >> i) & 1u)
-                    mine[__popc(u.keep & ((1u << i) - 1u))] = (uint16_t)(hw[i >> 1] >> (16 * (i & 1)));
-            const uint32_t cnt = (uint32_t)(8 * c.n_keep) / (uint32_t)M;
-            uint16_t* dst = t.w_fwd + (size_t)unit * cnt;
-            if (cnt == 8) *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(mine);
-            else if (cnt == 4) *reinterpret_cast<uint2*>(dst) = *reinterpret_cast<const uint2*>(mine);
-            else if (cnt == 2) *reinterpret_cast<uint32_t*>(dst) = *reinterpret_cast<const uint32_t*>(mine);
-            else
-                for (uint32_t k = 0; k < cnt; ++k) dst[k] = mine[k];
+            store_kept_values<M>(t.w_fwd, unit, u.keep, u.g, c.n_keep);
         }
         reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;
     }
