@@ -236,6 +236,13 @@ CAST_API int cast_prune_fold(const float* w, const float* scale, int scale_group
                     int64_t rows, int64_t cols, int N, int M, uint32_t flags, cast_stream_t stream);
 
 /*
+ * cast_plan_prune_fold -- cast_prune_fold over every matrix of a plan in one launch (per 320 matrices): weights,
+ * scales and metadata are the ones the plan's descriptors name; `out` is a HOST array of n_tensors device pointers,
+ * one output buffer per matrix (sizes as in cast_prune_fold).  flags as cast_prune_fold.
+ */
+CAST_API int cast_plan_prune_fold(void* plan, cast_bf16* const* out, uint32_t flags, cast_stream_t stream);
+
+/*
  * cast_mask_stats -- the mask statistics the paper monitors during training (App. C), for one matrix:
  *
  *   mask_diff      += ||M - M_ref||_0   numerator of the flip rate r_t when M_ref is the previous mask, of the

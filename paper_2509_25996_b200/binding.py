@@ -38,7 +38,7 @@ CAST_F_GRAD_OF_SCALED = 1 << 6
 EXPORTS = (
     "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
-    "cast_host_step_static", "cast_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
+    "cast_host_step_static", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
 )
 
@@ -117,6 +117,8 @@ def load_library() -> ctypes.CDLL:
     lib.cast_prune_fold.restype = ctypes.c_int
     lib.cast_prune_fold.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_uint32, ctypes.c_void_p]
+    lib.cast_plan_prune_fold.restype = ctypes.c_int
+    lib.cast_plan_prune_fold.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_uint32, ctypes.c_void_p]
     lib.cast_mask_stats.restype = ctypes.c_int
     lib.cast_mask_stats.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p]
@@ -264,6 +266,12 @@ def cast_host_step_static(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, row
 def cast_prune_fold(w, scale, scale_groups, meta, out, rows, cols, N, M, flags, stream=None) -> int:
     return load_library().cast_prune_fold(_ptr(w), _ptr(scale), int(scale_groups), _ptr(meta), _ptr(out), int(rows), int(cols),
                                           int(N), int(M), int(flags), _stream(stream))
+
+
+def cast_plan_prune_fold(plan, outs, flags, stream=None) -> int:
+    """`outs`: a sequence of one output buffer per matrix of the plan."""
+    arr = None if outs is None else (ctypes.c_void_p * len(outs))(*[_ptr(o) for o in outs])
+    return load_library().cast_plan_prune_fold(plan, arr, int(flags), _stream(stream))
 
 
 class cast_mask_stats_t(ctypes.Structure):

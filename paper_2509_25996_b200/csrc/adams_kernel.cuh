@@ -14,7 +14,7 @@
 //
 // Instruction budget: at ~6.8 TB/s an SM retires ~0.85 parameters per clock, so the body has to stay
 // well under ~100 thread instructions per parameter or instruction issue (and, under the board's
-// power cap, the SM clock) becomes the limit.  Hence: flags are compile-time constants in the two
+// power cap, the SM clock) becomes the limit.  Hence: flags are compile-time constants in the three
 // common modes, the 2:4 selection is six comparisons and four 3-input predicate functions per group,
 // and the update uses the approximate reciprocal and square root units (error analysis below).
 #pragma once
@@ -38,10 +38,11 @@ constexpr uint32_t kEmitDense = 1u << 4;
 constexpr uint32_t kEmitCompressed = 1u << 5;
 constexpr uint32_t kGradOfScaled = 1u << 6;
 
-// Kernel modes: the flag word is a compile-time constant in the two common cases.
+// Kernel modes: the flag word is a compile-time constant in the common cases.
 constexpr int kModeGeneric = 0;        // any flags, read from StepConsts at run time
 constexpr int kModeSelectIdx = 1;      // flags == kReselect, 2:4, index-form metadata
 constexpr int kModeSelectMask = 2;     // flags == kReselect | kMetaBitmask, any N:M
+constexpr int kModeSelectIdxPacked = 3;   // flags == kReselect | kEmitCompressed, 2:4, index-form metadata
 
 // One matrix as the kernel sees it.
 struct TensorDesc {
@@ -174,9 +175,27 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 // `packed` holds the unit's 8 bf16 values.  Every group keeps exactly N, so the slot of a kept column is the
 // number of kept columns before it in the unit.  The values are scattered into a private 16-byte row of
 // shared memory and read back as a vector (16, 8 or 4 bytes; other counts go out as 2-byte stores).
+// 2:4: the kept pair of a group (columns lo < hi: two of the four bf16 halves of registers r01, r23) picked by
+// one byte permute.  Half h of the register pair is bytes 2h, 2h + 1: selector = (2lo, 2lo + 1, 2hi, 2hi + 1).
+__device__ __forceinline__ uint32_t kept_pair_by_index(uint32_t r01, uint32_t r23, uint32_t lo, uint32_t hi)
+{
+    return __byte_perm(r01, r23, 0x1010u + 0x22u * lo + 0x2200u * hi);
+}
+__device__ __forceinline__ uint32_t kept_pair_2of4(uint32_t r01, uint32_t r23, uint32_t nibble)   // nibble = keep bits
+{
+    const uint32_t lo = (nibble & 1u) ? 0u : ((nibble & 2u) ? 1u : 2u);
+    const uint32_t hi = (nibble & 8u) ? 3u : ((nibble & 4u) ? 2u : 1u);
+    return kept_pair_by_index(r01, r23, lo, hi);
+}
+
 template <int M>
 __device__ __forceinline__ void store_kept_values(uint16_t* base, uint32_t unit, uint32_t keep, uint4 packed, int n_keep)
 {
+    if (M == 4 && n_keep == 2) {              // uniform: 4 values per unit, no shared memory needed
+        *reinterpret_cast<uint2*>(base + (size_t)unit * 4) =
+            make_uint2(kept_pair_2of4(packed.x, packed.y, keep & 0xFu), kept_pair_2of4(packed.z, packed.w, keep >> 4));
+        return;
+    }
     __shared__ __align__(16) uint16_t s_comp[kThreads * 8];
     uint16_t* mine = s_comp + threadIdx.x * 8;
     const uint32_t hw[4] = {packed.x, packed.y, packed.z, packed.w};
@@ -206,6 +225,7 @@ template <int MODE>
 __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
 {
     if constexpr (MODE == kModeSelectIdx) return kReselect;
+    else if constexpr (MODE == kModeSelectIdxPacked) return kReselect | kEmitCompressed;
     else if constexpr (MODE == kModeSelectMask) return kReselect | kMetaBitmask;
     else return c.flags;
 }
@@ -225,7 +245,7 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
 template <int M, int MODE>
 __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a, float& gw_sum)
 {
-    static_assert(MODE != kModeSelectIdx || M == 4, "index-form metadata is 2:4 only");
+    static_assert((MODE != kModeSelectIdx && MODE != kModeSelectIdxPacked) || M == 4, "index-form metadata is 2:4 only");
     const uint32_t flags = mode_flags<MODE>(c);
     const bool bitmask = (flags & kMetaBitmask) != 0;
     uint32_t ab[8];
@@ -234,7 +254,7 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
 
     bool kept[8];
     uint32_t flips = 0;
-    if constexpr (MODE == kModeSelectIdx) {
+    if constexpr (MODE == kModeSelectIdx || MODE == kModeSelectIdxPacked) {
         select_2of4(ab, kept);
         select_2of4(ab + 4, kept + 4);
         u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
@@ -356,7 +376,13 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         st_f4(t.v + e + 4, make_float4(u.v[4], u.v[5], u.v[6], u.v[7]));
         bool compressed = false;
         if constexpr (MODE == kModeGeneric && M <= 8) compressed = (flags & kEmitCompressed) != 0;
-        if (!compressed) {
+        if constexpr (MODE == kModeSelectIdxPacked) {
+            // the index-form metadata byte holds the kept positions of both groups: lo | hi << 2 per nibble
+            const uint32_t mb = u.meta_byte;
+            *reinterpret_cast<uint2*>(t.w_fwd + (size_t)unit * 4) =
+                make_uint2(kept_pair_by_index(u.g.x, u.g.y, mb & 3u, (mb >> 2) & 3u),
+                           kept_pair_by_index(u.g.z, u.g.w, (mb >> 4) & 3u, mb >> 6));
+        } else if (!compressed) {
             *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
         } else {
             store_kept_values<M>(t.w_fwd, unit, u.keep, u.g, c.n_keep);

@@ -166,6 +166,7 @@ namespace {
 int mode_of(const StepConsts& c, int M)
 {
     if (c.flags == kReselect && M == 4 && c.n_keep == 2) return kModeSelectIdx;
+    if (c.flags == (kReselect | kEmitCompressed) && M == 4 && c.n_keep == 2) return kModeSelectIdxPacked;
     if (c.flags == (kReselect | kMetaBitmask)) return kModeSelectMask;
     return kModeGeneric;
 }
@@ -201,6 +202,9 @@ int launch_single_m(const TensorDesc& d, const StepConsts& c, unsigned long long
         case kModeSelectIdx:
             if constexpr (M == 4) return launch_single_t<4, kModeSelectIdx>(d, c, flip_count, stream);
             break;
+        case kModeSelectIdxPacked:
+            if constexpr (M == 4) return launch_single_t<4, kModeSelectIdxPacked>(d, c, flip_count, stream);
+            break;
         case kModeSelectMask: return launch_single_t<M, kModeSelectMask>(d, c, flip_count, stream);
     }
     return launch_single_t<M, kModeGeneric>(d, c, flip_count, stream);
@@ -212,6 +216,9 @@ int launch_multi_m(const MultiParams& p, const StepConsts& c, unsigned long long
     switch (mode_of(c, M)) {
         case kModeSelectIdx:
             if constexpr (M == 4) return launch_multi_t<4, kModeSelectIdx>(p, c, flip_count, stream);
+            break;
+        case kModeSelectIdxPacked:
+            if constexpr (M == 4) return launch_multi_t<4, kModeSelectIdxPacked>(p, c, flip_count, stream);
             break;
         case kModeSelectMask: return launch_multi_t<M, kModeSelectMask>(p, c, flip_count, stream);
     }
@@ -281,6 +288,22 @@ int plan_tensor_count(const void* plan)
     const Plan* p = (const Plan*)plan;
     if (!p || p->magic != kPlanMagic) return -1;
     return p->n_tensors;
+}
+
+bool plan_tensor_desc(const void* plan, int i, int* N, int* M, TensorDesc* desc)
+{
+    const Plan* p = (const Plan*)plan;
+    if (!p || p->magic != kPlanMagic || i < 0 || i >= p->n_tensors) return false;
+    for (const MultiParams& mp : p->launches) {
+        if (i < (int)mp.n_tensors) {
+            *N = p->N;
+            *M = p->M;
+            *desc = mp.desc[i];
+            return true;
+        }
+        i -= (int)mp.n_tensors;
+    }
+    return false;
 }
 
 bool plan_tensor(const void* plan, int i, int* M, const float** w, const uint32_t** meta, uint32_t* n_units)

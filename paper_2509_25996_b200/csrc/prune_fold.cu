@@ -3,63 +3,155 @@
 // metadata.  The mask is chosen now by magnitude (Eq. 6, exactly N per group) or read from stored metadata.
 // No optimizer state is touched.  Streaming, HBM-bound: 4 B read, 2 (or 2 N / M) + 1/8 B written per parameter.
 //
-// Same thread layout as the AdamS step (one unit of 8 columns per thread, one CTA of 128 threads per tile of
-// 1024 parameters) and the same selection code.
+// Same unit layout (8 columns per thread and access) and the same selection code as the AdamS step; a CTA of
+// 128 threads takes 4 units per thread (4096 parameters); all matrices of a plan go in one grid.
+#include <cstring>
+
 #include "cast_internal.h"
 
 namespace cast {
+
+// Host-side view of a plan (defined with the plan in cast_adams.cu).
+int plan_tensor_count(const void* plan);
+bool plan_tensor_desc(const void* plan, int i, int* N, int* M, TensorDesc* desc);
+
 namespace {
 
+// One matrix of a pruning launch, and the tables of the launch (kernel parameter space, like the step's).
+struct PruneDesc {
+    const float* w;
+    const float* scale;
+    uint8_t* meta;
+    uint16_t* out;
+    uint32_t n_units, seg_magic, seg_shift, pad_;
+};
+struct PruneParams {
+    uint32_t n_tensors;
+    uint32_t hint_shift;
+    uint16_t hint[kHintEntries];
+    uint32_t tile_start[kMaxLaunchTensors + 1];
+    PruneDesc desc[kMaxLaunchTensors];
+};
+
+constexpr int kPruneUnitsPerThread = 4;                               // units a thread handles, loads issued together
+constexpr int kPruneTileUnits = kThreads * kPruneUnitsPerThread;      // 512 units = 4096 parameters per CTA
+
+// A CTA of the step moves 28 KB; this pass moves 6 bytes per parameter, so a CTA takes four times the
+// parameters (with one unit per thread the grid launched CTAs faster than they could be scheduled).
 template <int M>
 __global__ void __launch_bounds__(kThreads)
-prune_fold_kernel(const float* __restrict__ w, const float* __restrict__ scale, uint32_t seg_magic, uint32_t seg_shift,
-                  uint8_t* __restrict__ meta, uint16_t* __restrict__ out, uint32_t n_units, int n_keep, uint32_t flags)
+prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t flags)
 {
-    const uint32_t unit = blockIdx.x * kTileUnits + threadIdx.x;
-    const bool active = unit < n_units;
+    const uint32_t tile = blockIdx.x;
+    uint32_t k = p.hint[tile >> p.hint_shift];
+    while (tile >= p.tile_start[k + 1]) ++k;
+    const PruneDesc& t = p.desc[k];
+    const uint32_t first = (tile - p.tile_start[k]) * kPruneTileUnits + threadIdx.x;
     const bool bitmask = (flags & kMetaBitmask) != 0;
-    float x[8];
-    uint32_t ab[8];
-    float a = 1.0f;
-    uint32_t stored = 0;
+    float x[kPruneUnitsPerThread][8];
+    float a[kPruneUnitsPerThread];
+    uint32_t stored[kPruneUnitsPerThread];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) x[i] = 0.0f;
-    if (active) {
-        const float4 lo = ld_f4(w + (size_t)unit * kUnitElems), hi = ld_f4(w + (size_t)unit * kUnitElems + 4);
-        x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w; x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
-        if (!(flags & kReselect)) stored = meta[unit];
-        if (scale != nullptr) a = __ldg(scale + (uint32_t)(((uint64_t)unit * seg_magic) >> seg_shift));
+    for (int j = 0; j < kPruneUnitsPerThread; ++j) {
+        const uint32_t unit = first + j * kThreads;
+        a[j] = 1.0f;
+        stored[j] = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[j][i] = 0.0f;
+        if (unit < t.n_units) {
+            const float4 lo = ld_f4(t.w + (size_t)unit * kUnitElems), hi = ld_f4(t.w + (size_t)unit * kUnitElems + 4);
+            x[j][0] = lo.x; x[j][1] = lo.y; x[j][2] = lo.z; x[j][3] = lo.w; x[j][4] = hi.x; x[j][5] = hi.y; x[j][6] = hi.z; x[j][7] = hi.w;
+            if (!(flags & kReselect)) stored[j] = t.meta[unit];
+            if (t.scale != nullptr) a[j] = __ldg(t.scale + (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift));
+        }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i) ab[i] = abs_bits(x[i]);
-    uint32_t keep;
-    if (flags & kReselect) keep = select_by_rank<M>(ab, n_keep);      // uniform branch: all lanes shuffle
-    else keep = keep_from_meta_byte(stored, bitmask);
-    if (!active) return;
-    bool kept[8];
-    float f[8];
+    for (int j = 0; j < kPruneUnitsPerThread; ++j) {
+        const uint32_t unit = first + j * kThreads;
+        const bool active = unit < t.n_units;
+        uint32_t ab[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        kept[i] = (keep >> i) & 1u;
-        f[i] = kept[i] ? a * x[i] : 0.0f;
+        for (int i = 0; i < 8; ++i) ab[i] = abs_bits(x[j][i]);
+        bool kept[8];
+        uint32_t keep = 0;
+        const bool fast_2of4 = (flags & kReselect) && M == 4 && n_keep == 2;      // uniform
+        if (fast_2of4) {                                                          // the predicate network of the step
+            select_2of4(ab, kept);
+            select_2of4(ab + 4, kept + 4);
+        } else {
+            if (flags & kReselect) keep = select_by_rank<M>(ab, n_keep);          // uniform branch: all lanes shuffle
+            else keep = keep_from_meta_byte(stored[j], bitmask);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+        }
+        if (!active) continue;
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = kept[i] ? a[j] * x[j][i] : 0.0f;
+        const uint4 packed = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
+        const uint32_t idx_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);   // kept positions, lo | hi << 2 per group
+        if (fast_2of4 && bitmask) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) keep |= (kept[i] ? 1u : 0u) << i;
+        }
+        bool compressed = false;
+        if constexpr (M <= 8) compressed = (flags & kEmitCompressed) != 0;
+        if (compressed && M == 4 && n_keep == 2)
+            *reinterpret_cast<uint2*>(t.out + (size_t)unit * 4) =
+                make_uint2(kept_pair_by_index(packed.x, packed.y, idx_byte & 3u, (idx_byte >> 2) & 3u),
+                           kept_pair_by_index(packed.z, packed.w, (idx_byte >> 4) & 3u, idx_byte >> 6));
+        else if (compressed) store_kept_values<M>(t.out, unit, keep, packed, n_keep);
+        else *reinterpret_cast<uint4*>(t.out + (size_t)unit * kUnitElems) = packed;
+        t.meta[unit] = (uint8_t)(bitmask ? keep : idx_byte);
     }
-    const uint4 packed = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
-    bool compressed = false;
-    if constexpr (M <= 8) compressed = (flags & kEmitCompressed) != 0;
-    if (compressed) store_kept_values<M>(out, unit, keep, packed, n_keep);
-    else *reinterpret_cast<uint4*>(out + (size_t)unit * kUnitElems) = packed;
-    meta[unit] = (uint8_t)(bitmask ? keep : (idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4)));
+}
+
+inline uint32_t prune_tiles(uint32_t n_units) { return (n_units + kPruneTileUnits - 1) / kPruneTileUnits; }
+
+void fill_prune_hints(PruneParams* p)
+{
+    const uint64_t tiles = p->tile_start[p->n_tensors];
+    uint32_t shift = 0;
+    while (((tiles + (1ull << shift) - 1) >> shift) > (uint64_t)kHintEntries) ++shift;
+    p->hint_shift = shift;
+    const size_t n_hints = (size_t)((tiles + (1ull << shift) - 1) >> shift);
+    size_t k = 0;
+    for (size_t b = 0; b < (size_t)kHintEntries; ++b) {
+        if (b < n_hints) {
+            const uint64_t first = (uint64_t)b << shift;
+            while (first >= p->tile_start[k + 1]) ++k;
+        }
+        p->hint[b] = (uint16_t)k;
+    }
 }
 
 template <int M>
-int launch(const float* w, const float* scale, uint32_t magic, uint32_t shift, uint32_t* meta, uint16_t* out,
-           uint32_t n_units, int N, uint32_t flags, cudaStream_t s)
+int launch_t(const PruneParams& p, int N, uint32_t flags, cudaStream_t s)
 {
-    const uint32_t tiles = (n_units + kTileUnits - 1) / kTileUnits;
-    prune_fold_kernel<M><<<tiles, kThreads, 0, s>>>(w, scale, magic, shift, (uint8_t*)meta, out, n_units, N, flags);
+    prune_fold_kernel<M><<<p.tile_start[p.n_tensors], kThreads, 0, s>>>(p, N, flags);
     CAST_CUDA_TRY(cudaGetLastError());
     count_launch();
     return CAST_OK;
+}
+
+int launch(PruneParams* p, int N, int M, uint32_t flags, cudaStream_t s)
+{
+    fill_prune_hints(p);
+    if (p->tile_start[p->n_tensors] == 0) return CAST_OK;
+    switch (M) {
+        case 2:  return launch_t<2>(*p, N, flags, s);
+        case 4:  return launch_t<4>(*p, N, flags, s);
+        case 8:  return launch_t<8>(*p, N, flags, s);
+        case 16: return launch_t<16>(*p, N, flags, s);
+        case 32: return launch_t<32>(*p, N, flags, s);
+    }
+    return CAST_ERR_NM;
+}
+
+int check_prune_flags(int N, int M, uint32_t flags)
+{
+    if (flags & ~(uint32_t)(CAST_F_RESELECT | CAST_F_META_BITMASK | CAST_F_EMIT_COMPRESSED)) return CAST_ERR_HYPER;
+    return check_nm_flags(N, M, flags, nullptr);
 }
 
 }  // namespace
@@ -71,9 +163,8 @@ extern "C" int cast_prune_fold(const float* w, const float* scale, int scale_gro
                                int64_t rows, int64_t cols, int N, int M, uint32_t flags, cast_stream_t stream)
 {
     if (!w || !meta || !out) return CAST_ERR_NULL;
-    if (flags & ~(uint32_t)(CAST_F_RESELECT | CAST_F_META_BITMASK | CAST_F_EMIT_COMPRESSED)) return CAST_ERR_HYPER;
     int rc;
-    if ((rc = check_nm_flags(N, M, flags, nullptr)) != CAST_OK) return rc;
+    if ((rc = check_prune_flags(N, M, flags)) != CAST_OK) return rc;
     if ((rc = check_shape(rows, cols, M, scale != nullptr, scale_groups)) != CAST_OK) return rc;
     const uint64_t P = (uint64_t)rows * (uint64_t)cols;
     const uint64_t out_bytes = 2 * fwd_elems_of(rows, cols, N, M, flags);
@@ -87,13 +178,50 @@ extern "C" int cast_prune_fold(const float* w, const float* scale, int scale_gro
     }
     if ((rc = check_device_memory(ptrs, 4)) != CAST_OK) return rc;
     const TensorDesc d = make_desc(nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, scale, scale_groups, rows, cols);
-    cudaStream_t s = (cudaStream_t)stream;
-    switch (M) {
-        case 2:  return launch<2>(w, scale, d.seg_magic, d.seg_shift, meta, out, d.n_units, N, flags, s);
-        case 4:  return launch<4>(w, scale, d.seg_magic, d.seg_shift, meta, out, d.n_units, N, flags, s);
-        case 8:  return launch<8>(w, scale, d.seg_magic, d.seg_shift, meta, out, d.n_units, N, flags, s);
-        case 16: return launch<16>(w, scale, d.seg_magic, d.seg_shift, meta, out, d.n_units, N, flags, s);
-        case 32: return launch<32>(w, scale, d.seg_magic, d.seg_shift, meta, out, d.n_units, N, flags, s);
+    PruneParams p;
+    std::memset(&p, 0, sizeof p);
+    p.n_tensors = 1;
+    p.desc[0] = PruneDesc{w, scale, (uint8_t*)meta, out, d.n_units, d.seg_magic, d.seg_shift, 0};
+    p.tile_start[1] = prune_tiles(d.n_units);
+    return launch(&p, N, M, flags, (cudaStream_t)stream);
+}
+
+extern "C" int cast_plan_prune_fold(void* plan, cast_bf16* const* out, uint32_t flags, cast_stream_t stream)
+{
+    const int n = plan_tensor_count(plan);
+    if (n < 0) return CAST_ERR_PLAN;
+    if (!out) return CAST_ERR_NULL;
+    int N = 0, M = 0, rc;
+    TensorDesc d;
+    plan_tensor_desc(plan, 0, &N, &M, &d);
+    if ((rc = check_prune_flags(N, M, flags)) != CAST_OK) return rc;
+    for (int i = 0; i < n; ++i) {
+        if (!out[i]) return CAST_ERR_NULL;
+        if ((uintptr_t)out[i] & 15u) return CAST_ERR_ALIGN;
+        plan_tensor_desc(plan, i, &N, &M, &d);
+        const uint64_t P = (uint64_t)d.n_units * kUnitElems;
+        const uint64_t ob = 2 * ((flags & CAST_F_EMIT_COMPRESSED) ? P / (uint64_t)M * (uint64_t)N : P);
+        const uintptr_t o = (uintptr_t)out[i];
+        if ((o < (uintptr_t)d.w + 4 * P && (uintptr_t)d.w < o + ob) || (o < (uintptr_t)d.meta + P / 8 && (uintptr_t)d.meta < o + ob))
+            return CAST_ERR_ALIAS;
+        const void* op[1] = {out[i]};
+        if ((rc = check_device_memory(op, 1)) != CAST_OK) return rc;
     }
-    return CAST_ERR_NM;
+    int i = 0;
+    while (i < n) {
+        PruneParams p;
+        std::memset(&p, 0, sizeof p);
+        uint64_t tiles = 0;
+        while (i < n && p.n_tensors < (uint32_t)kMaxLaunchTensors) {
+            plan_tensor_desc(plan, i, &N, &M, &d);
+            p.desc[p.n_tensors] = PruneDesc{d.w, d.scale, (uint8_t*)d.meta, out[i], d.n_units, d.seg_magic, d.seg_shift, 0};
+            p.tile_start[p.n_tensors] = (uint32_t)tiles;
+            tiles += prune_tiles(d.n_units);
+            ++p.n_tensors;
+            ++i;
+        }
+        p.tile_start[p.n_tensors] = (uint32_t)tiles;
+        if ((rc = launch(&p, N, M, flags, (cudaStream_t)stream)) != CAST_OK) return rc;
+    }
+    return CAST_OK;
 }

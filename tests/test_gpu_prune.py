@@ -81,6 +81,36 @@ def test_prune_fold_adversarial_values_and_exact_scale():
         assert np.array_equal(got_meta, ref["meta"]) and np.array_equal(got_out, ref["out"])           # bit for bit
 
 
+@pytest.mark.parametrize("N,M,enc,compressed", [(2, 4, 0, False), (2, 4, 0, True), (4, 8, BM, True), (8, 16, BM, False)])
+def test_plan_prune_fold_one_launch(N, M, enc, compressed):
+    """Every matrix of a plan in one grid: ragged tiles, one-unit matrices, with and without a scale."""
+    shapes = [(1, 32), (3, 96), (64, 1056), (7, 2080), (1, 32), (33, 2048)]
+    extra = C if compressed else 0
+    ins = [workloads.gen_tensor_inputs(r, c, seed=310, tensor_index=i, scale_mode="jitter" if (c // 2) % max(M, 8) == 0 else "none")
+           for i, (r, c) in enumerate(shapes)]
+    states = [U.to_device(inp, DEV) for inp in ins]
+    tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale,
+                             1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in states]
+    rc, plan = cast.cast_plan_create(tensors, N, M)
+    cast.check(rc)
+    outs = [U.Guarded(r * c * N // M if compressed else r * c, torch.bfloat16, DEV) for r, c in shapes]
+    before = cast.cast_kernel_launch_count()
+    cast.check(cast.cast_plan_prune_fold(plan, [o.view for o in outs], RS | enc | extra, torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == before + 1
+    for i, (s, inp, o) in enumerate(zip(states, ins, outs)):
+        assert s.all_intact() and o.intact()
+        ref = orc.prune_fold(inp.w.numpy(), None if inp.scale is None else inp.scale.numpy(), N, M, oracle_flags(RS | enc | extra))
+        assert np.array_equal(s.meta.view.cpu().numpy().view(np.uint32).reshape(ref["meta"].shape), ref["meta"]), f"tensor {i}"
+        d = bf16_ulp_distance(workloads.bf16_bits(o.view).reshape(ref["out"].shape), ref["out"])
+        assert d.max(initial=0) <= 1, f"tensor {i}"
+        assert torch.equal(s.w.view.cpu(), inp.w.reshape(-1))                 # state untouched
+    assert cast.cast_plan_prune_fold(plan, None, RS | enc, None) == B.CAST_ERR_NULL
+    assert cast.cast_plan_prune_fold(None, [o.view for o in outs], RS | enc, None) == B.CAST_ERR_PLAN
+    assert cast.cast_plan_prune_fold(plan, [s.w.view for s in states], RS | enc, None) == B.CAST_ERR_ALIAS
+    cast.check(cast.cast_plan_destroy(plan))
+
+
 def test_prune_fold_rejections():
     w = torch.zeros(4 * 64, device=DEV)
     meta = torch.zeros(4 * 2, dtype=torch.int32, device=DEV)
