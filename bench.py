@@ -53,6 +53,10 @@ def parse_args():
     p.add_argument("--e2e-layers", type=int, default=1, help="LLaMA layers held in host memory for the e2e leg (0 = skip)")
     p.add_argument("--e2e-steps", type=int, default=4)
     p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
+    p.add_argument("--schedule", choices=["every-step", "t1"], default="every-step",
+                   help="every-step: reselect the mask at every step (the headline, worst case); t1: the paper's training "
+                        "schedule (Sec. 4.1, App. C): stored mask and dense forward weight, mask refreshed and flips counted "
+                        "every 10th step")
     p.add_argument("--seed", type=int, default=0)
     p.add_argument("--op", choices=["step", "mask_stats", "prune_fold"], default="step",
                    help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass")
@@ -257,6 +261,21 @@ def cuda_arm(args):
         oracle_repeats = 1
     hyper = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl.total_steps)
     stream = torch.cuda.current_stream(dev)
+    if args.schedule == "t1":
+        if (N, M) != (2, 4) or args.emit != "pruned" or wl.resident_layers or args.count_flips:
+            raise SystemExit("--schedule t1 is wired for 2:4 on a resident workload")
+        refresh = B.CAST_F_RESELECT | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE
+        between = B.CAST_F_EMIT_DENSE
+        state.step(hyper, B.CAST_F_RESELECT, stream)           # establishes the stored mask (untimed)
+        # reuse steps move 28.125 B/param (the metadata is read, not rewritten), refresh steps 28.25
+        bytes_per_param = 28.125 + 0.125 / 10
+        args.cpu_baseline = 0
+
+        def flags_at(step_no):
+            return refresh if step_no % 10 == 0 else between
+    else:
+        def flags_at(step_no):
+            return flags
 
     # parity sample (checked in the CPU-baseline leg): a few rows of the first and last matrices, copied
     # before the first step and again after it
@@ -278,7 +297,7 @@ def cuda_arm(args):
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
     parity_out = {}
     for i in range(args.warmup):
-        state.step(hyper, flags, stream)
+        state.step(hyper, flags_at(hyper.step), stream)
         hyper.step += 1
         if i == 0 and parity_in:
             torch.cuda.synchronize(dev)
@@ -304,7 +323,7 @@ def cuda_arm(args):
     if flush is None:
         ev0.record(stream)
         for _ in range(args.steps):
-            state.step(hyper, flags, stream)
+            state.step(hyper, flags_at(hyper.step), stream)
             hyper.step += 1
         ev1.record(stream)
         barrier()
@@ -315,7 +334,7 @@ def cuda_arm(args):
             flush.fill_(1)
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(stream)
-            state.step(hyper, flags, stream)
+            state.step(hyper, flags_at(hyper.step), stream)
             b.record(stream)
             hyper.step += 1
             pairs.append((a, b))
@@ -326,7 +345,7 @@ def cuda_arm(args):
         wa, wb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         wa.record(stream)
         for _ in range(args.steps):
-            state.step(hyper, flags, stream)
+            state.step(hyper, flags_at(hyper.step), stream)
             hyper.step += 1
         wb.record(stream)
         barrier()
@@ -451,7 +470,7 @@ def cuda_arm(args):
                                                                                   else "L2 flushed by a 512 MB write before every step, steps timed one by one"),
                    "resident_layers": wl.resident_layers, "streams": 2 if wl.resident_layers else 1,
                    "lr": hyper.lr, "betas": [hyper.beta1, hyper.beta2], "eps": hyper.eps, "l1_coeff": hyper.l1_coeff,
-                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "seed": args.seed},
+                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "schedule": args.schedule, "seed": args.seed},
         "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
         "warm_l2": (None if warm_ms_per_step is None else
                     {"ms_per_step": warm_ms_per_step, "value": wl.n_params / (warm_ms_per_step * 1e-3),
@@ -462,7 +481,7 @@ def cuda_arm(args):
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": launches // args.steps,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params * args.steps / max(launches, 1),
-                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None or args.emit != "pruned" or args.count_flips or (N, M) != (2, 4)
+                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None or args.emit != "pruned" or args.count_flips or (N, M) != (2, 4) or args.schedule != "every-step"
                                  else NCU_DRAM_BYTES_PER_PARAM * wl.n_params * args.steps / max(launches, 1))},
         "cpu_baseline": cpu_baseline, "parity": parity,
     }

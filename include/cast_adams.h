@@ -99,7 +99,8 @@ enum cast_flags {
  *                kept, +0.0 (0x0000) elsewhere (all entries with CAST_F_EMIT_DENSE).  Rounding is to
  *                nearest even of the fp32 product.
  *   meta         device, uint32 [rows*cols/32], in/out (layout above).  Read when CAST_F_RESELECT is
- *                absent or CAST_F_COUNT_FLIPS is set; always written.
+ *                absent or CAST_F_COUNT_FLIPS is set; written when CAST_F_RESELECT is set (a reused mask
+ *                is left as it is).
  *   scale        device, fp32 [rows][scale_groups] (the matrix A of Eq. 12, n = scale_groups), or NULL
  *                for A = 1.  Requires scale_groups >= 1, cols % scale_groups == 0 and
  *                (cols/scale_groups) % max(M, 8) == 0.

@@ -43,6 +43,8 @@ constexpr int kModeGeneric = 0;        // any flags, read from StepConsts at run
 constexpr int kModeSelectIdx = 1;      // flags == kReselect, 2:4, index-form metadata
 constexpr int kModeSelectMask = 2;     // flags == kReselect | kMetaBitmask, any N:M
 constexpr int kModeSelectIdxPacked = 3;   // flags == kReselect | kEmitCompressed, 2:4, index-form metadata
+constexpr int kModeReuseIdx = 4;       // flags == 0: the stored 2:4 mask is reused (between the paper's refreshes)
+constexpr int kModeReuseIdxDense = 5;  // flags == kEmitDense: stored 2:4 mask, dense forward weight (Alg. 2's training step)
 
 // One matrix as the kernel sees it.
 struct TensorDesc {
@@ -227,6 +229,8 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
     if constexpr (MODE == kModeSelectIdx) return kReselect;
     else if constexpr (MODE == kModeSelectIdxPacked) return kReselect | kEmitCompressed;
     else if constexpr (MODE == kModeSelectMask) return kReselect | kMetaBitmask;
+    else if constexpr (MODE == kModeReuseIdx) return 0u;
+    else if constexpr (MODE == kModeReuseIdxDense) return kEmitDense;
     else return c.flags;
 }
 
@@ -245,7 +249,7 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
 template <int M, int MODE>
 __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a, float& gw_sum)
 {
-    static_assert((MODE != kModeSelectIdx && MODE != kModeSelectIdxPacked) || M == 4, "index-form metadata is 2:4 only");
+    static_assert(MODE == kModeGeneric || MODE == kModeSelectMask || M == 4, "index-form metadata is 2:4 only");
     const uint32_t flags = mode_flags<MODE>(c);
     const bool bitmask = (flags & kMetaBitmask) != 0;
     uint32_t ab[8];
@@ -259,17 +263,24 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
         select_2of4(ab + 4, kept + 4);
         u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
     } else {
+        // `flags` is a compile-time constant in every mode but the generic one: the branches below fold away
+        const bool need_prev = !(flags & kReselect) || (flags & kCountFlips);
+        const uint32_t prev_keep = need_prev ? keep_from_meta_byte(u.prev_byte, bitmask) : 0u;
         uint32_t keep;
-        uint32_t prev_keep = 0;
-        if constexpr (MODE == kModeGeneric) prev_keep = keep_from_meta_byte(u.prev_byte, bitmask);
-        if (flags & kReselect) keep = select_by_rank<M>(ab, c.n_keep);     // uniform branch: all lanes shuffle
-        else keep = prev_keep;
+        if (flags & kReselect) {
+            keep = select_by_rank<M>(ab, c.n_keep);     // uniform branch: all lanes shuffle
 #pragma unroll
-        for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+            for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+            if (bitmask) u.meta_byte = keep;
+            else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+        } else {
+            keep = prev_keep;                           // the stored mask, as it is
+#pragma unroll
+            for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+            u.meta_byte = u.prev_byte;
+        }
         u.keep = keep;
-        if (bitmask) u.meta_byte = keep;
-        else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
-        if constexpr (MODE == kModeGeneric) flips = (uint32_t)__popc(keep ^ prev_keep);
+        if (flags & kCountFlips) flips = (uint32_t)__popc(keep ^ prev_keep);
     }
 
     const uint32_t gw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
@@ -349,7 +360,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
 
     float gw_sum;
     const uint32_t flips = compute_unit<M, MODE>(u, c, a, gw_sum);
-    if constexpr (MODE == kModeGeneric) {
+    {
         if ((flags & kGradOfScaled) && t.scale_grad != nullptr) {     // uniform over the CTA: all lanes shuffle
             // Sum gw_sum over the lanes of the warp that share a row segment (segments are runs of consecutive
             // lanes), then one atomic per run.  Lanes without data carry a segment of their own and add nothing.
@@ -375,7 +386,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         st_f4(t.v + e, make_float4(u.v[0], u.v[1], u.v[2], u.v[3]));
         st_f4(t.v + e + 4, make_float4(u.v[4], u.v[5], u.v[6], u.v[7]));
         bool compressed = false;
-        if constexpr (MODE == kModeGeneric && M <= 8) compressed = (flags & kEmitCompressed) != 0;
+        if constexpr (M <= 8) compressed = (flags & kEmitCompressed) != 0;
         if constexpr (MODE == kModeSelectIdxPacked) {
             // the index-form metadata byte holds the kept positions of both groups: lo | hi << 2 per nibble
             const uint32_t mb = u.meta_byte;
@@ -387,7 +398,7 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         } else {
             store_kept_values<M>(t.w_fwd, unit, u.keep, u.g, c.n_keep);
         }
-        reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;
+        if (flags & kReselect) reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;   // else unchanged
     }
     return active ? flips : 0u;
 }
@@ -435,8 +446,7 @@ adams_nm_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ St
 {
     const uint32_t unit = blockIdx.x * kTileUnits + threadIdx.x;
     const uint32_t flips = process_unit<M, MODE>(t, c, unit, unit < t.n_units);
-    if constexpr (MODE == kModeGeneric)
-        if (c.flags & kCountFlips) add_flips(flips, flip_count);
+    if (mode_flags<MODE>(c) & kCountFlips) add_flips(flips, flip_count);
 }
 
 // Up to kMaxLaunchTensors matrices in one grid: CTA b handles tile b of the concatenated index space.
@@ -451,8 +461,7 @@ adams_nm_multi_kernel(const __grid_constant__ MultiParams p, const __grid_consta
     const TensorDesc& t = p.desc[k];
     const uint32_t unit = (tile - p.tile_start[k]) * kTileUnits + threadIdx.x;
     const uint32_t flips = process_unit<M, MODE>(t, c, unit, unit < t.n_units);
-    if constexpr (MODE == kModeGeneric)
-        if (c.flags & kCountFlips) add_flips(flips, flip_count);
+    if (mode_flags<MODE>(c) & kCountFlips) add_flips(flips, flip_count);
 }
 
 }  // namespace cast

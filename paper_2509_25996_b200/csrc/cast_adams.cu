@@ -167,6 +167,8 @@ int mode_of(const StepConsts& c, int M)
 {
     if (c.flags == kReselect && M == 4 && c.n_keep == 2) return kModeSelectIdx;
     if (c.flags == (kReselect | kEmitCompressed) && M == 4 && c.n_keep == 2) return kModeSelectIdxPacked;
+    if (c.flags == 0u && M == 4 && c.n_keep == 2) return kModeReuseIdx;
+    if (c.flags == kEmitDense && M == 4 && c.n_keep == 2) return kModeReuseIdxDense;
     if (c.flags == (kReselect | kMetaBitmask)) return kModeSelectMask;
     return kModeGeneric;
 }
@@ -205,6 +207,12 @@ int launch_single_m(const TensorDesc& d, const StepConsts& c, unsigned long long
         case kModeSelectIdxPacked:
             if constexpr (M == 4) return launch_single_t<4, kModeSelectIdxPacked>(d, c, flip_count, stream);
             break;
+        case kModeReuseIdx:
+            if constexpr (M == 4) return launch_single_t<4, kModeReuseIdx>(d, c, flip_count, stream);
+            break;
+        case kModeReuseIdxDense:
+            if constexpr (M == 4) return launch_single_t<4, kModeReuseIdxDense>(d, c, flip_count, stream);
+            break;
         case kModeSelectMask: return launch_single_t<M, kModeSelectMask>(d, c, flip_count, stream);
     }
     return launch_single_t<M, kModeGeneric>(d, c, flip_count, stream);
@@ -219,6 +227,12 @@ int launch_multi_m(const MultiParams& p, const StepConsts& c, unsigned long long
             break;
         case kModeSelectIdxPacked:
             if constexpr (M == 4) return launch_multi_t<4, kModeSelectIdxPacked>(p, c, flip_count, stream);
+            break;
+        case kModeReuseIdx:
+            if constexpr (M == 4) return launch_multi_t<4, kModeReuseIdx>(p, c, flip_count, stream);
+            break;
+        case kModeReuseIdxDense:
+            if constexpr (M == 4) return launch_multi_t<4, kModeReuseIdxDense>(p, c, flip_count, stream);
             break;
         case kModeSelectMask: return launch_multi_t<M, kModeSelectMask>(p, c, flip_count, stream);
     }

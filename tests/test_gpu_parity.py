@@ -144,6 +144,18 @@ def test_mask_reuse_and_flip_count(bitmask):
     assert got["flips"] == ref["flips"] > 0
 
 
+@pytest.mark.parametrize("flags", [0, B.CAST_F_EMIT_DENSE, B.CAST_F_EMIT_DENSE | B.CAST_F_GRAD_OF_SCALED, BM | B.CAST_F_EMIT_DENSE])
+def test_training_step_with_a_stored_mask(flags):
+    """The step between two mask refreshes (Sec. 4.1: masks are refreshed every T1 iterations): the stored 2:4 mask
+    gates the decay, the forward weight is pruned or dense (Alg. 2's training step), the metadata is left alone."""
+    rows, cols = 9, 2080
+    inp = inputs(rows, cols, seed=16)
+    stored = U.run_oracle(inputs(rows, cols, seed=17), 2, 4, Hyper(), RS | (flags & BM))["meta"]
+    got = U.run_cuda_single(inp, 2, 4, Hyper(), flags, meta_in=stored)
+    U.assert_parity(got, U.run_oracle(inp, 2, 4, Hyper(), flags, meta_in=stored), f"stored mask, flags {flags}")
+    assert np.array_equal(got["meta"], stored)
+
+
 def test_general_nm_flip_count():
     inp = inputs(4, 512, seed=6)
     prev = U.run_oracle(inputs(4, 512, seed=7), 4, 8, Hyper(), RS | BM)["meta"]
