@@ -45,6 +45,18 @@ constexpr int kModeSelectMask = 2;     // flags == kReselect | kMetaBitmask, any
 constexpr int kModeSelectIdxPacked = 3;   // flags == kReselect | kEmitCompressed, 2:4, index-form metadata
 constexpr int kModeReuseIdx = 4;       // flags == 0: the stored 2:4 mask is reused (between the paper's refreshes)
 constexpr int kModeReuseIdxDense = 5;  // flags == kEmitDense: stored 2:4 mask, dense forward weight (Alg. 2's training step)
+constexpr int kModeSelectIdxFlips = 6;       // flags == kReselect | kCountFlips, 2:4, index-form metadata
+constexpr int kModeSelectMaskFlips = 7;      // flags == kReselect | kMetaBitmask | kCountFlips, any N:M
+constexpr int kModeSelectIdxFlipsDense = 8;  // flags == kReselect | kCountFlips | kEmitDense, 2:4: the refresh step of training
+constexpr int kModeCount = 9;
+
+// Modes whose kept set comes from the 2:4 comparison network (N = 2, M = 4, index-form metadata).
+__host__ __device__ constexpr bool mode_selects_2of4(int mode)
+{
+    return mode == kModeSelectIdx || mode == kModeSelectIdxPacked || mode == kModeSelectIdxFlips || mode == kModeSelectIdxFlipsDense;
+}
+// Modes that exist for M = 4 only.
+__host__ __device__ constexpr bool mode_is_2of4_only(int mode) { return mode_selects_2of4(mode) || mode == kModeReuseIdx || mode == kModeReuseIdxDense; }
 
 // One matrix as the kernel sees it.
 struct TensorDesc {
@@ -70,9 +82,9 @@ struct StepConsts {
     double c_sign;      // alpha_t * lambda             (Eq. 7)
     float beta2;        // beta2
     float omb2;         // 1 - beta2
-    float inv_bc2;      // 1 / (1 - beta2^t)
-    float lr_bc1;       // lr / (1 - beta1^t)
-    float eps;
+    float inv_bc2_s;    // 2^64 / (1 - beta2^t)        the update runs on sqrt(v^) and eps scaled by 2^32 (see
+    float lr_bc1_s;     // 2^32 lr / (1 - beta1^t)      update_term), so that the flushing sqrt/rcp units never
+    float eps_s;        // 2^32 eps                     see a subnormal
     int32_t n_keep;     // N
     uint32_t flags;
 };
@@ -80,10 +92,19 @@ struct StepConsts {
 __device__ __forceinline__ float4 ld_f4(const float* p) { return *reinterpret_cast<const float4*>(p); }
 __device__ __forceinline__ void st_f4(float* p, float4 x) { *reinterpret_cast<float4*>(p) = x; }
 
-// Approximate units: sqrt.approx.f32 has a maximum relative error of 2^-23 over the positive finite
-// range, rcp.approx.f32 of 1 ulp (PTX ISA).  Neither flushes subnormals in this (non-ftz) form.
-__device__ __forceinline__ float sqrt_approx(float x) { float r; asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
-__device__ __forceinline__ float rcp_approx(float x) { float r; asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+// Approximate units: sqrt.approx.ftz.f32 has a maximum relative error of 2^-23 over the positive normal range,
+// rcp.approx.ftz.f32 of 1 ulp (PTX ISA); both are single instructions and flush subnormals to zero.
+__device__ __forceinline__ float sqrt_approx_ftz(float x) { float r; asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+__device__ __forceinline__ float rcp_approx_ftz(float x) { float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x)); return r; }
+
+// lr mu^ / (sqrt(v^) + eps) with numerator and denominator both scaled by 2^32 (exact, powers of two):
+//   sqrt(2^64 v^) = 2^32 sqrt(v^)  -- a subnormal v (down to 2^-149) becomes normal before the flushing sqrt;
+//   2^32 eps is normal for every positive float eps, so the denominator and its reciprocal are normal too
+//   (the reciprocal would only be flushed for v^ > 2^188, where the true update is below 1e-28 anyway).
+__device__ __forceinline__ float update_term(float mu_t, float v_new, const StepConsts& c)
+{
+    return (c.lr_bc1_s * mu_t) * rcp_approx_ftz(sqrt_approx_ftz(v_new * c.inv_bc2_s) + c.eps_s);
+}
 
 // |w| as an integer: for non-NaN floats the bit pattern without the sign orders exactly like the
 // absolute value, and -0 equals +0.
@@ -231,6 +252,9 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
     else if constexpr (MODE == kModeSelectMask) return kReselect | kMetaBitmask;
     else if constexpr (MODE == kModeReuseIdx) return 0u;
     else if constexpr (MODE == kModeReuseIdxDense) return kEmitDense;
+    else if constexpr (MODE == kModeSelectIdxFlips) return kReselect | kCountFlips;
+    else if constexpr (MODE == kModeSelectMaskFlips) return kReselect | kMetaBitmask | kCountFlips;
+    else if constexpr (MODE == kModeSelectIdxFlipsDense) return kReselect | kCountFlips | kEmitDense;
     else return c.flags;
 }
 
@@ -249,7 +273,7 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
 template <int M, int MODE>
 __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a, float& gw_sum)
 {
-    static_assert(MODE == kModeGeneric || MODE == kModeSelectMask || M == 4, "index-form metadata is 2:4 only");
+    static_assert(!mode_is_2of4_only(MODE) || M == 4, "index-form metadata is 2:4 only");
     const uint32_t flags = mode_flags<MODE>(c);
     const bool bitmask = (flags & kMetaBitmask) != 0;
     uint32_t ab[8];
@@ -258,10 +282,12 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
 
     bool kept[8];
     uint32_t flips = 0;
-    if constexpr (MODE == kModeSelectIdx || MODE == kModeSelectIdxPacked) {
+    if constexpr (mode_selects_2of4(MODE)) {
         select_2of4(ab, kept);
         select_2of4(ab + 4, kept + 4);
         u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+        if (flags & kCountFlips)                        // both masks as index bytes: decode and compare
+            flips = (uint32_t)__popc(keep_from_meta_byte(u.meta_byte, false) ^ keep_from_meta_byte(u.prev_byte, false));
     } else {
         // `flags` is a compile-time constant in every mode but the generic one: the branches below fold away
         const bool need_prev = !(flags & kReselect) || (flags & kCountFlips);
@@ -313,7 +339,7 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
         const float vn = fmaf(c.beta2, u.v[i], (c.omb2 * src) * src);
         u.v[i] = vn;
         // bias-corrected update (Alg. 1): w - (lr / bc1) mu~ / (sqrt(v / bc2) + eps)
-        const float wn = fmaf(-(c.lr_bc1 * mu_t), rcp_approx(sqrt_approx(vn * c.inv_bc2) + c.eps), u.w[i]);
+        const float wn = u.w[i] - update_term(mu_t, vn, c);
         u.w[i] = wn;
         // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for
         fwd[i] = (kept[i] || dense) ? a * wn : 0.0f;
@@ -436,7 +462,7 @@ __device__ __forceinline__ void add_flips(uint32_t flips, unsigned long long* fl
     }
 }
 
-#define CAST_LAUNCH_BOUNDS(M) __launch_bounds__(kThreads, ((M) <= 8) ? kMinCtasPerSm : 5)
+#define CAST_LAUNCH_BOUNDS(M) __launch_bounds__(kThreads, ((M) <= 8) ? kMinCtasPerSm : 4)
 
 // One matrix: CTA b handles tile b.
 template <int M, int MODE>

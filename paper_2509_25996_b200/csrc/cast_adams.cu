@@ -55,9 +55,10 @@ int make_step_consts(float lr, float beta1, float beta2, float eps, float l1_coe
     c.c_sign = alpha * (double)l1_coeff;
     c.beta2 = beta2;
     c.omb2 = (float)(1.0 - (double)beta2);
-    c.inv_bc2 = (float)(1.0 / bc2);
-    c.lr_bc1 = (float)((double)lr / bc1);
-    c.eps = eps;
+    c.inv_bc2_s = (float)(18446744073709551616.0 / bc2);             // 2^64 / bc2
+    c.lr_bc1_s = (float)(4294967296.0 * (double)lr / bc1);            // 2^32 lr / bc1
+    c.eps_s = (float)(4294967296.0 * (double)eps);                    // 2^32 eps
+    if (!std::isfinite(c.lr_bc1_s) || !std::isfinite(c.eps_s) || !std::isfinite(c.inv_bc2_s)) return CAST_ERR_HYPER;
     c.n_keep = N;
     c.flags = flags;
     *out = c;
@@ -162,14 +163,20 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
 
 namespace {
 
-// The flag word is a compile-time constant of the kernel in the two common cases.
+// The flag word is a compile-time constant of the kernel in the common cases.
 int mode_of(const StepConsts& c, int M)
 {
-    if (c.flags == kReselect && M == 4 && c.n_keep == 2) return kModeSelectIdx;
-    if (c.flags == (kReselect | kEmitCompressed) && M == 4 && c.n_keep == 2) return kModeSelectIdxPacked;
-    if (c.flags == 0u && M == 4 && c.n_keep == 2) return kModeReuseIdx;
-    if (c.flags == kEmitDense && M == 4 && c.n_keep == 2) return kModeReuseIdxDense;
-    if (c.flags == (kReselect | kMetaBitmask)) return kModeSelectMask;
+    const bool two_four = M == 4 && c.n_keep == 2;
+    switch (c.flags) {
+        case kReselect:                                return two_four ? kModeSelectIdx : kModeGeneric;
+        case kReselect | kEmitCompressed:              return two_four ? kModeSelectIdxPacked : kModeGeneric;
+        case 0u:                                       return two_four ? kModeReuseIdx : kModeGeneric;
+        case kEmitDense:                               return two_four ? kModeReuseIdxDense : kModeGeneric;
+        case kReselect | kCountFlips:                  return two_four ? kModeSelectIdxFlips : kModeGeneric;
+        case kReselect | kCountFlips | kEmitDense:     return two_four ? kModeSelectIdxFlipsDense : kModeGeneric;
+        case kReselect | kMetaBitmask:                 return kModeSelectMask;
+        case kReselect | kMetaBitmask | kCountFlips:   return kModeSelectMaskFlips;
+    }
     return kModeGeneric;
 }
 
@@ -197,46 +204,29 @@ int launch_multi_t(const MultiParams& p, const StepConsts& c, unsigned long long
     return CAST_OK;
 }
 
-template <int M>
-int launch_single_m(const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+// Walks the mode list at compile time: instantiates the kernel of every mode that exists for this M.
+template <int M, int MODE = 0>
+int launch_single_m(int mode, const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    switch (mode_of(c, M)) {
-        case kModeSelectIdx:
-            if constexpr (M == 4) return launch_single_t<4, kModeSelectIdx>(d, c, flip_count, stream);
-            break;
-        case kModeSelectIdxPacked:
-            if constexpr (M == 4) return launch_single_t<4, kModeSelectIdxPacked>(d, c, flip_count, stream);
-            break;
-        case kModeReuseIdx:
-            if constexpr (M == 4) return launch_single_t<4, kModeReuseIdx>(d, c, flip_count, stream);
-            break;
-        case kModeReuseIdxDense:
-            if constexpr (M == 4) return launch_single_t<4, kModeReuseIdxDense>(d, c, flip_count, stream);
-            break;
-        case kModeSelectMask: return launch_single_t<M, kModeSelectMask>(d, c, flip_count, stream);
+    if constexpr (MODE >= kModeCount) {
+        return CAST_ERR_NM;
+    } else {
+        if constexpr (M == 4 || !mode_is_2of4_only(MODE))
+            if (mode == MODE) return launch_single_t<M, MODE>(d, c, flip_count, stream);
+        return launch_single_m<M, MODE + 1>(mode, d, c, flip_count, stream);
     }
-    return launch_single_t<M, kModeGeneric>(d, c, flip_count, stream);
 }
 
-template <int M>
-int launch_multi_m(const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+template <int M, int MODE = 0>
+int launch_multi_m(int mode, const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    switch (mode_of(c, M)) {
-        case kModeSelectIdx:
-            if constexpr (M == 4) return launch_multi_t<4, kModeSelectIdx>(p, c, flip_count, stream);
-            break;
-        case kModeSelectIdxPacked:
-            if constexpr (M == 4) return launch_multi_t<4, kModeSelectIdxPacked>(p, c, flip_count, stream);
-            break;
-        case kModeReuseIdx:
-            if constexpr (M == 4) return launch_multi_t<4, kModeReuseIdx>(p, c, flip_count, stream);
-            break;
-        case kModeReuseIdxDense:
-            if constexpr (M == 4) return launch_multi_t<4, kModeReuseIdxDense>(p, c, flip_count, stream);
-            break;
-        case kModeSelectMask: return launch_multi_t<M, kModeSelectMask>(p, c, flip_count, stream);
+    if constexpr (MODE >= kModeCount) {
+        return CAST_ERR_NM;
+    } else {
+        if constexpr (M == 4 || !mode_is_2of4_only(MODE))
+            if (mode == MODE) return launch_multi_t<M, MODE>(p, c, flip_count, stream);
+        return launch_multi_m<M, MODE + 1>(mode, p, c, flip_count, stream);
     }
-    return launch_multi_t<M, kModeGeneric>(p, c, flip_count, stream);
 }
 
 }  // namespace
@@ -244,11 +234,11 @@ int launch_multi_m(const MultiParams& p, const StepConsts& c, unsigned long long
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
     switch (M) {
-        case 2:  return launch_single_m<2>(d, c, flip_count, stream);
-        case 4:  return launch_single_m<4>(d, c, flip_count, stream);
-        case 8:  return launch_single_m<8>(d, c, flip_count, stream);
-        case 16: return launch_single_m<16>(d, c, flip_count, stream);
-        case 32: return launch_single_m<32>(d, c, flip_count, stream);
+        case 2:  return launch_single_m<2>(mode_of(c, 2), d, c, flip_count, stream);
+        case 4:  return launch_single_m<4>(mode_of(c, 4), d, c, flip_count, stream);
+        case 8:  return launch_single_m<8>(mode_of(c, 8), d, c, flip_count, stream);
+        case 16: return launch_single_m<16>(mode_of(c, 16), d, c, flip_count, stream);
+        case 32: return launch_single_m<32>(mode_of(c, 32), d, c, flip_count, stream);
     }
     return CAST_ERR_NM;
 }
@@ -256,11 +246,11 @@ int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
     switch (M) {
-        case 2:  return launch_multi_m<2>(p, c, flip_count, stream);
-        case 4:  return launch_multi_m<4>(p, c, flip_count, stream);
-        case 8:  return launch_multi_m<8>(p, c, flip_count, stream);
-        case 16: return launch_multi_m<16>(p, c, flip_count, stream);
-        case 32: return launch_multi_m<32>(p, c, flip_count, stream);
+        case 2:  return launch_multi_m<2>(mode_of(c, 2), p, c, flip_count, stream);
+        case 4:  return launch_multi_m<4>(mode_of(c, 4), p, c, flip_count, stream);
+        case 8:  return launch_multi_m<8>(mode_of(c, 8), p, c, flip_count, stream);
+        case 16: return launch_multi_m<16>(mode_of(c, 16), p, c, flip_count, stream);
+        case 32: return launch_multi_m<32>(mode_of(c, 32), p, c, flip_count, stream);
     }
     return CAST_ERR_NM;
 }

@@ -60,6 +60,14 @@ def adversarial(rows, cols, M):
     w[6::9, 0] = 3e4
     w[6::9, 1 % M] = 1e-30
     w[7::9, M // 2] = 0.0
+    # state and gradient corners: exact zeros, subnormal and tiny moments, zero gradients
+    inp.v.view(-1)[0::7] = 0.0
+    inp.v.view(-1)[1::7] = 1e-40
+    inp.v.view(-1)[2::7] = 1e-30
+    inp.m.view(-1)[0::5] = 0.0
+    inp.m.view(-1)[1::5] = 1e-30
+    inp.m.view(-1)[2::5] = -1e-42
+    inp.g.view(-1)[0::3] = 0.0
     return inp
 
 
@@ -137,11 +145,12 @@ def test_mask_reuse_and_flip_count(bitmask):
     got = U.run_cuda_single(inp2, 2, 4, h, enc, meta_in=first["meta"])
     U.assert_parity(got, U.run_oracle(inp2, 2, 4, h, enc, meta_in=first["meta"]), "reuse")
     assert np.array_equal(got["meta"], first["meta"])
-    fl = RS | enc | B.CAST_F_COUNT_FLIPS
-    got = U.run_cuda_single(inp2, 2, 4, h, fl, meta_in=first["meta"])
-    ref = U.run_oracle(inp2, 2, 4, h, fl, meta_in=first["meta"])
-    U.assert_parity(got, ref, "flips")
-    assert got["flips"] == ref["flips"] > 0
+    for more in (0, B.CAST_F_EMIT_DENSE):                 # the refresh step of training also emits the dense weight
+        fl = RS | enc | B.CAST_F_COUNT_FLIPS | more
+        got = U.run_cuda_single(inp2, 2, 4, h, fl, meta_in=first["meta"])
+        ref = U.run_oracle(inp2, 2, 4, h, fl, meta_in=first["meta"])
+        U.assert_parity(got, ref, f"flips, extra flags {more}")
+        assert got["flips"] == ref["flips"] > 0
 
 
 @pytest.mark.parametrize("flags", [0, B.CAST_F_EMIT_DENSE, B.CAST_F_EMIT_DENSE | B.CAST_F_GRAD_OF_SCALED, BM | B.CAST_F_EMIT_DENSE])
