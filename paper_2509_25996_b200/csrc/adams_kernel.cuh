@@ -14,7 +14,7 @@
 //
 // Instruction budget: at ~6.8 TB/s an SM retires ~0.85 parameters per clock, so the body has to stay
 // well under ~100 thread instructions per parameter or instruction issue (and, under the board's
-// power cap, the SM clock) becomes the limit.  Hence: flags are compile-time constants in the three
+// power cap, the SM clock) becomes the limit.  Hence: flags are compile-time constants in the
 // common modes, the 2:4 selection is six comparisons and four 3-input predicate functions per group,
 // and the update uses the approximate reciprocal and square root units (error analysis below).
 #pragma once
