@@ -241,7 +241,7 @@ struct UnitRegs {
     uint4 g;               // 8 bf16 gradients in; 8 bf16 forward weights out
     uint32_t prev_byte;    // metadata byte of the unit before the step (when it is read)
     uint32_t meta_byte;    // metadata byte after the step
-    uint32_t keep;         // keep mask of the unit (bit j = column j kept); not set in the 2:4 index mode
+    uint32_t keep;         // keep mask of the unit (bit j = column j kept); not set by the 2:4 comparison-network modes
 };
 
 template <int MODE>

@@ -27,6 +27,9 @@ def sample_blocks(shapes, n_random, rows_per_block, seed):
 
 
 def check_sampled(wl_name, N, M, flags, n_random=14, rows_per_block=6, need_gb=0.0):
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                                     # blocks cached by earlier tests count as used
     free, _ = torch.cuda.mem_get_info()
     if free < need_gb * 1e9:
         pytest.skip(f"needs {need_gb} GB of device memory, {free / 1e9:.0f} GB free")
@@ -71,6 +74,64 @@ def test_llama2_7b_full_set_sampled():
 @pytest.mark.parametrize("N,M", [(4, 8), (1, 4)])
 def test_llama2_7b_layer_general_nm_sampled(N, M):
     check_sampled("llama2_7b_layer", N, M, B.CAST_F_RESELECT | B.CAST_F_META_BITMASK, n_random=8, need_gb=5)
+
+
+def test_llama2_7b_full_set_4_8_with_flips_sampled():
+    """The full LLaMA2-7B set under 4:8 with flip counting (one launch, bitmask metadata): sampled row blocks
+    against the oracle, Eq. 4 on whole matrices, and the flip total is even (groups keep exactly N, so a group
+    that changes its kept set changes it in pairs) and equals the mask statistics pass against the old masks."""
+    import ctypes
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()                                     # blocks cached by earlier tests count as used
+    free, _ = torch.cuda.mem_get_info()
+    if free < 125e9:
+        pytest.skip("needs 125 GB of device memory")
+    wl = workloads.workload("llama2_7b")
+    N, M = 4, 8
+    flags = B.CAST_F_RESELECT | B.CAST_F_META_BITMASK
+    state = DeviceModelState(wl.shapes, N, M, seed=0, device=DEV, scale_mode="jitter")
+    h = RunHyper(total_steps=wl.total_steps)
+    state.step(h, flags)                                         # masks of the initial weights
+    picks = sample_blocks(wl.shapes, 10, 6, seed=2)
+    before, old_meta = [], []
+    for t, r0 in picks:
+        s = state.mats[t]
+        sl = slice(r0, r0 + 6)
+        before.append((workloads.TensorInputs(s.w[sl].cpu(), s.g[sl].cpu(), s.m[sl].cpu(), s.v[sl].cpu(), s.scale[sl].cpu()),
+                       s.meta[sl].cpu().numpy().view(np.uint32).copy()))
+    refs = [m.meta.clone() for m in state.mats[:8]]              # reference masks of the first layer and a bit
+    h.step += 1
+    state.flips.zero_()
+    state.step(h, flags | B.CAST_F_COUNT_FLIPS)
+    torch.cuda.synchronize()
+    flips = int(state.flips.item())
+    assert flips > 0 and flips % 2 == 0
+    oh = orc.Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
+    sampled_flips = 0
+    for (t, r0), (inp, meta_in) in zip(picks, before):
+        s = state.mats[t]
+        sl = slice(r0, r0 + 6)
+        got = dict(w=s.w[sl].cpu().numpy(), m=s.m[sl].cpu().numpy(), v=s.v[sl].cpu().numpy(),
+                   w_fwd=workloads.bf16_bits(s.w_fwd[sl]), meta=s.meta[sl].cpu().numpy().view(np.uint32))
+        ref = U.run_oracle(inp, N, M, oh, flags | B.CAST_F_COUNT_FLIPS, meta_in=meta_in)
+        U.assert_parity(got, ref, f"4:8 tensor {t} rows {r0}+")
+        sampled_flips += ref["flips"]
+    assert sampled_flips <= flips
+    # the flips of the first matrices, counted a second way by the statistics pass
+    stats = torch.zeros(ctypes.sizeof(B.cast_mask_stats_t), dtype=torch.uint8, device=DEV)
+    part = 0
+    for mat, ref_meta in zip(state.mats[:8], refs):
+        cast.check(cast.cast_mask_stats(mat.w, mat.meta, ref_meta, mat.rows, mat.cols, M, B.CAST_F_META_BITMASK, stats, None))
+        pop = sum((((mat.meta ^ ref_meta) >> b) & 1).sum(dtype=torch.int64) for b in range(32))
+        part += int(pop.item())
+    torch.cuda.synchronize()
+    assert B.cast_mask_stats_t.from_buffer_copy(stats.cpu().numpy().tobytes()).mask_diff == part
+    for t in (0, len(wl.shapes) - 1):
+        s = state.mats[t]
+        pop = sum(((s.meta >> b) & 1).sum(dtype=torch.int64) for b in range(32))
+        assert int(pop.item()) == s.rows * s.cols * N // M
+    state.close()
 
 
 def test_llama2_13b_layer_sampled():
