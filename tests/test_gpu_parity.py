@@ -201,6 +201,32 @@ def test_two_runs_are_bit_identical():
         assert np.array_equal(a[k].view(np.uint8), b[k].view(np.uint8))
 
 
+def test_resumed_run_is_bit_identical():
+    """The library keeps no state of its own: w, m, v, the metadata and the step number are the whole checkpoint.
+    Two steps in a row equal one step, a round trip of the state through host memory into fresh buffers, and the
+    second step."""
+    rows, cols = 48, 1056
+    inp = inputs(rows, cols, seed=18)
+    g2 = workloads.gen_gradient(rows, cols, 18, 0, 2)
+    h1, h2 = Hyper(step=1, total_steps=100), Hyper(step=2, total_steps=100)
+    fl = RS | B.CAST_F_COUNT_FLIPS
+
+    def second_step(state_w, state_m, state_v, meta):
+        nxt = workloads.TensorInputs(state_w, g2, state_m, state_v, inp.scale)
+        return U.run_cuda_single(nxt, 2, 4, h2, fl, meta_in=meta)
+
+    a1 = U.run_cuda_single(inp, 2, 4, h1, RS)
+    straight = second_step(*(torch.from_numpy(a1[k]) for k in ("w", "m", "v")), a1["meta"])
+    # "checkpoint": bytes on the host, reloaded into new tensors
+    blob = {k: a1[k].tobytes() for k in ("w", "m", "v", "meta")}
+    re_w, re_m, re_v = (torch.from_numpy(np.frombuffer(blob[k], dtype=np.float32).reshape(rows, cols).copy()) for k in ("w", "m", "v"))
+    re_meta = np.frombuffer(blob["meta"], dtype=np.uint32).reshape(rows, cols // 32).copy()
+    resumed = second_step(re_w, re_m, re_v, re_meta)
+    for k in ("w", "m", "v", "w_fwd", "meta"):
+        assert np.array_equal(straight[k].view(np.uint8), resumed[k].view(np.uint8))
+    assert straight["flips"] == resumed["flips"]
+
+
 def test_three_steps_with_refresh_schedule():
     """Steps t = 9, 10, 11 with the paper's refresh every T1 = 10 iterations: step 10 reselects and counts
     flips, the others reuse the stored mask.  Each step starts from the CUDA path's own previous state,
