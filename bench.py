@@ -33,7 +33,7 @@ FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
 # capture of one LLaMA2-7B layer (202,375,168 parameters) summarised under profiles/; every byte is touched
 # once, so the traffic of a launch is this figure times its parameter count.  Set to None when the kernel
 # changes until the counters are taken again.
-NCU_DRAM_BYTES_PER_PARAM = 27.850
+NCU_DRAM_BYTES_PER_PARAM = 27.863
 
 METRIC = "AdamS 2:4 step params/s"
 
