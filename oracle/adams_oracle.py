@@ -45,6 +45,9 @@ def _load():
         lib.oracle_prune_fold.restype = ctypes.c_int
         lib.oracle_prune_fold.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                           ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_uint32]
+        lib.oracle_kd_loss.restype = ctypes.c_int
+        lib.oracle_kd_loss.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64,
+                                       ctypes.c_double, ctypes.c_double, ctypes.c_void_p, ctypes.c_void_p]
         lib.oracle_plain_adam.restype = ctypes.c_int
         lib.oracle_plain_adam.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                           ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_double, ctypes.c_int64]
@@ -183,3 +186,21 @@ def prune_fold(w, scale, N, M, flags: int = F_RESELECT, meta_in=None):
     if rc != 0:
         raise ValueError("oracle_prune_fold rejected its arguments")
     return dict(out=out.reshape(rows, ocols), meta=meta.reshape(rows, cols // 32))
+
+
+def kd_loss(student_bits, teacher_bits, labels, eta: float, grad_scale: float = 1.0, want_grad: bool = True):
+    """Per-token loss of Eq. 13 and its gradient with respect to the student logits (both fp64).
+    student_bits, teacher_bits: uint16 (raw bf16) [tokens, vocab]; labels: int32 [tokens] (negative: no target)."""
+    lib = _load()
+    s = np.ascontiguousarray(student_bits, dtype=np.uint16)
+    t = np.ascontiguousarray(teacher_bits, dtype=np.uint16)
+    y = np.ascontiguousarray(labels, dtype=np.int32)
+    tokens, vocab = s.shape
+    assert t.shape == s.shape and y.shape == (tokens,)
+    loss = np.zeros(tokens, dtype=np.float64)
+    grad = np.zeros((tokens, vocab), dtype=np.float64) if want_grad else None
+    rc = lib.oracle_kd_loss(s.ctypes.data, t.ctypes.data, y.ctypes.data, tokens, vocab, float(np.float32(eta)),
+                            float(np.float32(grad_scale)), loss.ctypes.data, None if grad is None else grad.ctypes.data)
+    if rc != 0:
+        raise ValueError("oracle_kd_loss rejected its arguments")
+    return loss, grad

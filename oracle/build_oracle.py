@@ -15,6 +15,7 @@ SRC = os.path.join(HERE, "adams_oracle.c")
 STATS_SRC = os.path.join(HERE, "mask_stats_oracle.c")
 ADAM_SRC = os.path.join(HERE, "plain_adam_oracle.c")
 PRUNE_SRC = os.path.join(HERE, "prune_fold_oracle.c")
+KD_SRC = os.path.join(HERE, "kd_loss_oracle.c")
 LIB = os.path.join(HERE, "liboracle_adams.so")
 
 # No fast-math, no contraction: the fp32 build must perform exactly the
@@ -23,14 +24,14 @@ CFLAGS = ["-O2", "-fPIC", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-W
 
 
 def build(force: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= max(os.path.getmtime(SRC), os.path.getmtime(STATS_SRC), os.path.getmtime(ADAM_SRC), os.path.getmtime(PRUNE_SRC)):
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= max(os.path.getmtime(SRC), os.path.getmtime(STATS_SRC), os.path.getmtime(ADAM_SRC), os.path.getmtime(PRUNE_SRC), os.path.getmtime(KD_SRC)):
         return LIB
     objs = []
     for real, entry in (("double", "oracle_adams_step_f64"), ("float", "oracle_adams_step_f32")):
         obj = os.path.join(HERE, f"adams_oracle_{real}.o")
         subprocess.check_call(["gcc", *CFLAGS, f"-DREAL={real}", f"-DENTRY={entry}", "-c", SRC, "-o", obj])
         objs.append(obj)
-    for src in (STATS_SRC, ADAM_SRC, PRUNE_SRC):
+    for src in (STATS_SRC, ADAM_SRC, PRUNE_SRC, KD_SRC):
         obj = src[:-2] + ".o"
         subprocess.check_call(["gcc", *CFLAGS, "-c", src, "-o", obj])
         objs.append(obj)

@@ -620,3 +620,49 @@ def test_final_pruning_is_the_step_emission_of_unmoved_weights():
     step = run(w, scale=scale, N=2, M=4, hyper=Hyper(lr=0.0), flags=orc.F_RESELECT)
     pf = orc.prune_fold(w, scale, 2, 4, orc.F_RESELECT)
     assert np.array_equal(step["w_fwd"], pf["out"]) and np.array_equal(step["meta"], pf["meta"])
+
+
+# --------------------------------------------------------------------------- distillation loss (Eq. 13)
+
+def _logits(rng, tokens, vocab, spread):
+    x = torch.tensor(rng.normal(0, spread, size=(tokens, vocab)), dtype=torch.float32).to(torch.bfloat16)
+    return x, x.view(torch.int16).numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("eta", [0.0, 1.0 / 3.0, 1.0])
+def test_distillation_loss_and_gradient_follow_torch(eta):
+    rng = np.random.default_rng(120)
+    tokens, vocab = 5, 257
+    s, s_bits = _logits(rng, tokens, vocab, 3.0)
+    t, t_bits = _logits(rng, tokens, vocab, 4.0)
+    labels = np.array([3, 256, 0, -100, 17], dtype=np.int32)
+    eta32 = float(np.float32(eta))
+    loss, grad = orc.kd_loss(s_bits, t_bits, labels, eta, grad_scale=0.25)
+    S = s.to(torch.float64).requires_grad_(True)
+    T = t.to(torch.float64)
+    log_ps = torch.log_softmax(S, dim=-1)
+    kl = torch.nn.functional.kl_div(log_ps, torch.softmax(T, dim=-1), reduction="none").sum(-1)
+    ce = torch.nn.functional.cross_entropy(S, torch.tensor(labels, dtype=torch.long), ignore_index=-100, reduction="none")
+    want = eta32 * kl + (1.0 - eta32) * ce
+    assert np.allclose(loss, want.detach().numpy(), rtol=1e-12, atol=1e-13)
+    (float(np.float32(0.25)) * want.sum()).backward()
+    assert np.allclose(grad, S.grad.numpy(), rtol=1e-10, atol=1e-15)
+
+
+def test_distillation_loss_closed_forms():
+    rng = np.random.default_rng(121)
+    s, s_bits = _logits(rng, 3, 64, 2.0)
+    labels = np.array([1, 2, 3], dtype=np.int32)
+    # teacher == student: the KL term vanishes, and so does its gradient
+    loss, grad = orc.kd_loss(s_bits, s_bits, labels, 1.0)
+    assert np.all(np.abs(loss) < 1e-15) and np.all(np.abs(grad) < 1e-15)
+    # a uniform student: cross-entropy is log V whatever the label; gradient 1/V - onehot
+    zeros = np.zeros((3, 64), dtype=np.uint16)
+    loss, grad = orc.kd_loss(zeros, s_bits, labels, 0.0)
+    assert np.allclose(loss, np.log(64.0), rtol=1e-15)
+    want = np.full((3, 64), 1.0 / 64)
+    want[np.arange(3), labels] -= 1.0
+    assert np.allclose(grad, want, rtol=1e-13, atol=1e-16)
+    # gradients of a token sum to zero when it has a target (probabilities sum to one on both sides)
+    loss, grad = orc.kd_loss(s_bits, _logits(rng, 3, 64, 2.0)[1], labels, 1.0 / 3.0)
+    assert np.all(np.abs(grad.sum(-1)) < 1e-14)
