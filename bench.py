@@ -58,8 +58,11 @@ def parse_args():
                         "schedule (Sec. 4.1, App. C): stored mask and dense forward weight, mask refreshed and flips counted "
                         "every 10th step")
     p.add_argument("--seed", type=int, default=0)
-    p.add_argument("--op", choices=["step", "mask_stats", "prune_fold"], default="step",
-                   help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass")
+    p.add_argument("--op", choices=["step", "mask_stats", "prune_fold", "kd_loss"], default="step",
+                   help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass; prune_fold: the "
+                        "final pruning of Alg. 2; kd_loss: the distillation loss of Eq. 13 with its gradient")
+    p.add_argument("--tokens", type=int, default=16384, help="kd_loss: tokens per step")
+    p.add_argument("--vocab", type=int, default=32000, help="kd_loss: vocabulary size (LLaMA2: 32000)")
     return p.parse_args()
 
 
@@ -623,8 +626,69 @@ def prune_arm(args):
         "parity": {"ok": ok, "sample": f"first {rows} rows of the first matrix against the CPU oracle (unit scale: bit-exact)"}}), flush=True)
 
 
+def kd_arm(args):
+    """The distillation loss of Eq. 13 with its gradient (cast_kd_loss): 2 + 2 B read and 2 B written per logit.
+    Synthetic logits: student ~ N(0, 3^2), teacher = student + N(0, 1) (a teacher close to the student), bf16."""
+    import numpy as np
+    import torch
+    import paper_2509_25996_b200 as cast
+    from paper_2509_25996_b200 import workloads
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    T, V = args.tokens, args.vocab
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(workloads.tensor_seed(args.seed, 0, 5))
+    base = torch.randn((T, V), generator=gen, device=dev, dtype=torch.float32) * 3.0
+    student = base.to(torch.bfloat16)
+    teacher = (base + torch.randn((T, V), generator=gen, device=dev, dtype=torch.float32)).to(torch.bfloat16)
+    del base
+    labels = torch.randint(0, V, (T,), generator=gen, device=dev, dtype=torch.int32)
+    loss = torch.empty(T, device=dev)
+    grad = torch.empty((T, V), dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream(dev)
+    eta = 1.0 / 3.0
+
+    def one_pass():
+        cast.check(cast.cast_kd_loss(student, teacher, labels, loss, grad, T, V, eta, 1.0 / T, stream))
+
+    for _ in range(args.warmup):
+        one_pass()
+    torch.cuda.synchronize(dev)
+    launches0 = cast.cast_kernel_launch_count()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.profiler.start()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        one_pass()
+    ev1.record(stream)
+    torch.cuda.synchronize(dev)
+    torch.cuda.profiler.stop()
+    ms = ev0.elapsed_time(ev1) / args.steps
+    launches = cast.cast_kernel_launch_count() - launches0
+    from oracle import adams_oracle as orc
+    rows = min(T, 8)
+    ref_loss, _ = orc.kd_loss(workloads.bf16_bits(student[:rows]), workloads.bf16_bits(teacher[:rows]), labels[:rows].cpu().numpy(),
+                              eta, 1.0 / T, want_grad=False)
+    got = loss[:rows].cpu().numpy().astype(np.float64)
+    ok = bool(np.all(np.abs(got - ref_loss) <= 2e-5 + 1e-5 * np.abs(ref_loss)))
+    gbs = T * V * 6.0 / (ms * 1e-3) / 1e9
+    peak, peak_kind = measured_hbm_peak()
+    print(json.dumps({
+        "metric": "distillation loss + gradient (Eq. 13) tokens/s", "value": T / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{T} tokens x {V} logits", "eta": eta, "l2": "inputs far larger than L2, no flush"},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
+                     "kernel": "kd_loss_kernel", "bytes_per_logit": 6.0, "launches_per_step": 1, "traffic": None},
+        "mean_loss": float(loss.double().mean().item()),
+        "parity": {"ok": ok, "sample": f"losses of the first {rows} tokens against the CPU oracle"}}), flush=True)
+
+
 def main():
     args = parse_args()
+    if args.op == "kd_loss" and args.impl != "reference":
+        return kd_arm(args)
     if args.op == "mask_stats" and args.impl != "reference":
         return stats_arm(args)
     if args.op == "prune_fold" and args.impl != "reference":

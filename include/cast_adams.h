@@ -220,6 +220,27 @@ CAST_API int cast_host_ctx_sync(void* ctx);
 CAST_API int cast_host_ctx_destroy(void* ctx);
 
 /*
+ * cast_kd_loss -- the training loss of Sec. 4.3 (Eq. 13) for every token, and its gradient:
+ *
+ *     loss[i] = eta * D_KL(P_t || P_s) + (1 - eta) * L_ce,   P_s = softmax(student row i), P_t = softmax(teacher row i),
+ *               L_ce = -log P_s(labels[i])
+ *     grad    = grad_scale * (P_s - eta P_t - (1 - eta) onehot(labels[i]))      (d loss[i] / d student row i)
+ *
+ *   student_logits, teacher_logits   device, bf16 [tokens][vocab].
+ *   labels        device, int32 [tokens]; a negative label (or one >= vocab) means the token has no target: its
+ *                 cross-entropy term and that term's gradient are left out (the paper does not treat padding).
+ *   loss          device, fp32 [tokens], out.  The paper does not say how tokens are reduced; sum or average them.
+ *   grad_logits   device, bf16 [tokens][vocab], out, or NULL for the loss alone.  grad_scale carries the
+ *                 reduction (1/tokens for a mean) and any loss scaling.
+ *   eta in [0, 1]; grad_scale finite.  Logits are expected to be finite.
+ * Rows with vocab % 8 == 0 and 16-byte aligned buffers take the vector path; anything else a slower scalar path
+ * with the same results.  Asynchronous on `stream`.
+ */
+CAST_API int cast_kd_loss(const cast_bf16* student_logits, const cast_bf16* teacher_logits, const int32_t* labels,
+                 float* loss, cast_bf16* grad_logits, int64_t tokens, int64_t vocab,
+                 float eta, float grad_scale, cast_stream_t stream);
+
+/*
  * cast_prune_fold -- the final pruning of Alg. 2 (its last loop; the last lines of Alg. 1): W^ = W (.) M with the
  * scale of Eq. 12 folded into the weights, as bf16.  No optimizer state is read or written.
  *

@@ -38,7 +38,7 @@ CAST_F_GRAD_OF_SCALED = 1 << 6
 EXPORTS = (
     "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
-    "cast_host_step_static", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
+    "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
 )
 
@@ -114,6 +114,8 @@ def load_library() -> ctypes.CDLL:
     lib.cast_host_step.argtypes = [ctypes.c_void_p] + _STEP_ARGS
     lib.cast_host_step_static.restype = ctypes.c_int
     lib.cast_host_step_static.argtypes = _STEP_ARGS + [ctypes.c_void_p]
+    lib.cast_kd_loss.restype = ctypes.c_int
+    lib.cast_kd_loss.argtypes = [ctypes.c_void_p] * 5 + [ctypes.c_int64, ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_void_p]
     lib.cast_prune_fold.restype = ctypes.c_int
     lib.cast_prune_fold.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
                                     ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_uint32, ctypes.c_void_p]
@@ -261,6 +263,11 @@ def cast_host_step_static(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, row
         _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
         int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
         int(flags), _ptr(flip_count), _stream(stream))
+
+
+def cast_kd_loss(student_logits, teacher_logits, labels, loss, grad_logits, tokens, vocab, eta, grad_scale=1.0, stream=None) -> int:
+    return load_library().cast_kd_loss(_ptr(student_logits), _ptr(teacher_logits), _ptr(labels), _ptr(loss), _ptr(grad_logits),
+                                       int(tokens), int(vocab), eta, grad_scale, _stream(stream))
 
 
 def cast_prune_fold(w, scale, scale_groups, meta, out, rows, cols, N, M, flags, stream=None) -> int:
