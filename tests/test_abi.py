@@ -159,3 +159,46 @@ def test_mask_stats_argument_checks():
     assert call_stats(stats=SC + 4) == B.CAST_ERR_ALIGN
     assert call_stats() in (B.CAST_ERR_CUDA, B.CAST_ERR_MEMORY)   # fake addresses are not device memory
     assert cast.cast_kernel_launch_count() == before
+
+
+def test_later_entry_points_check_their_arguments_without_a_gpu():
+    """Every check that needs no device runs before the first CUDA call, so these hold on a machine without a GPU."""
+    before = cast.cast_kernel_launch_count()
+    # final pruning
+    assert cast.cast_prune_fold(None, None, 1, META, F, 4, 64, 2, 4, B.CAST_F_RESELECT) == B.CAST_ERR_NULL
+    assert cast.cast_prune_fold(W, None, 1, META, F, 4, 64, 3, 8, B.CAST_F_RESELECT) == B.CAST_ERR_NM
+    assert cast.cast_prune_fold(W, None, 1, META, F, 4, 64, 2, 4, B.CAST_F_EMIT_DENSE) == B.CAST_ERR_HYPER
+    assert cast.cast_prune_fold(W, None, 1, META, F + 2, 4, 64, 2, 4, B.CAST_F_RESELECT) == B.CAST_ERR_ALIGN
+    assert cast.cast_prune_fold(W, None, 1, META, W + 64, 4, 64, 2, 4, B.CAST_F_RESELECT) == B.CAST_ERR_ALIAS
+    assert cast.cast_plan_prune_fold(None, None, B.CAST_F_RESELECT) == B.CAST_ERR_PLAN
+    # distillation loss
+    assert cast.cast_kd_loss(W, M_, None, V, None, 4, 64, 0.5) == B.CAST_ERR_NULL
+    assert cast.cast_kd_loss(W, M_, G, V, None, 4, 0, 0.5) == B.CAST_ERR_SHAPE
+    assert cast.cast_kd_loss(W, M_, G, V, None, 4, 64, -0.1) == B.CAST_ERR_HYPER
+    assert cast.cast_kd_loss(W, M_, G, V, None, 4, 64, 0.5, float("inf")) == B.CAST_ERR_HYPER
+    assert cast.cast_kd_loss(W + 1, M_, G, V, None, 4, 64, 0.5) == B.CAST_ERR_ALIGN
+    assert cast.cast_kd_loss(W, M_, G, V, W + 128, 4, 64, 0.5) == B.CAST_ERR_ALIAS
+    # scale training
+    assert cast.cast_scale_adam_step(W, M_, V, None, 8, 1e-3, 0.9, 0.95, 1e-8, 1) == B.CAST_ERR_NULL
+    assert cast.cast_scale_adam_step(W, M_, V, G, 8, float("nan"), 0.9, 0.95, 1e-8, 1) == B.CAST_ERR_HYPER
+    assert cast.cast_scale_adam_step(W, W + 16, V, G, 8, 1e-3, 0.9, 0.95, 1e-8, 1) == B.CAST_ERR_ALIAS
+    hyper = B.make_hyper(1e-4, 0.9, 0.95, 1e-8, 1e-3, 10, 100, B.CAST_F_RESELECT)
+    t = B.make_tensor(W, M_, V, G, F, META, None, 1, 4, 64)
+    assert cast.cast_adams_step_ex(None, 2, 4, hyper) == B.CAST_ERR_NULL
+    assert cast.cast_adams_step_ex(t, 2, 4, None) == B.CAST_ERR_NULL
+    assert cast.cast_adams_step_ex(t, 5, 4, hyper) == B.CAST_ERR_NM
+    bad = B.make_hyper(1e-4, 0.9, 0.95, 1e-8, 1e-3, 10, 100, B.CAST_F_RESELECT | B.CAST_F_EMIT_DENSE | B.CAST_F_EMIT_COMPRESSED)
+    assert cast.cast_adams_step_ex(t, 2, 4, bad) == B.CAST_ERR_HYPER
+    wide = B.make_hyper(1e-4, 0.9, 0.95, 1e-8, 1e-3, 10, 100, B.CAST_F_RESELECT | B.CAST_F_META_BITMASK | B.CAST_F_EMIT_COMPRESSED)
+    assert cast.cast_adams_step_ex(t, 8, 16, wide) == B.CAST_ERR_NM                   # compressed form needs M <= 8
+    huge_lr = B.make_hyper(3e38, 0.9, 0.95, 1e-8, 1e-3, 10, 100, B.CAST_F_RESELECT)
+    assert cast.cast_adams_step_ex(t, 2, 4, huge_lr) == B.CAST_ERR_HYPER              # 2^32 lr / bc1 is not a float
+    rc, plan = cast.cast_plan_create_ex([t], 2, 4, B.CAST_F_RESELECT)
+    assert rc == B.CAST_ERR_HYPER and plan is None                                    # only the compressed flag is a plan property
+    rc, plan = cast.cast_plan_create_ex([t], 8, 16, B.CAST_F_EMIT_COMPRESSED)
+    assert rc == B.CAST_ERR_NM and plan is None
+    # the static staging entry point refuses oversize matrices before touching CUDA
+    big_rows = B.CAST_STATIC_MAX_PARAMS // 64 + 1
+    assert cast.cast_host_step_static(W, M_, V, G, F, META, None, 1, big_rows, 64, 2, 4, 1e-4, 0.9, 0.95, 1e-8, 1e-3, 1, 10,
+                                      B.CAST_F_RESELECT) == B.CAST_ERR_PLAN
+    assert cast.cast_kernel_launch_count() == before
