@@ -102,7 +102,7 @@ static int popcount32(uint32_t x)
 /* Metadata field of group i of row r (M bits wide, packed LSB first into
  * row-major 32-bit words, cols/32 words per row; a word always describes 32
  * consecutive columns of one row).  The paper fixes only the size, one bit per
- * parameter (Remark in Sec. 4.1); the layout is this build's. */
+ * parameter (Remark in Sec. 4.1); the layout is defined here. */
 static uint32_t meta_get_field(const uint32_t *meta, int64_t r, int64_t cols, int64_t i, int M)
 {
     int64_t bit = i * M;
