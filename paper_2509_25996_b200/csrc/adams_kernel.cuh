@@ -48,15 +48,22 @@ constexpr int kModeReuseIdxDense = 5;  // flags == kEmitDense: stored 2:4 mask, 
 constexpr int kModeSelectIdxFlips = 6;       // flags == kReselect | kCountFlips, 2:4, index-form metadata
 constexpr int kModeSelectMaskFlips = 7;      // flags == kReselect | kMetaBitmask | kCountFlips, any N:M
 constexpr int kModeSelectIdxFlipsDense = 8;  // flags == kReselect | kCountFlips | kEmitDense, 2:4: the refresh step of training
-constexpr int kModeCount = 9;
+constexpr int kModeReuseIdxDenseScaled = 9;        // flags == kEmitDense | kGradOfScaled: mode 5 with the gradient taken
+                                                   // through the scaling (the common step of training with a learned scale)
+constexpr int kModeSelectIdxFlipsDenseScaled = 10; // flags == mode 8 | kGradOfScaled: its refresh step
+constexpr int kModeCount = 11;
 
 // Modes whose kept set comes from the 2:4 comparison network (N = 2, M = 4, index-form metadata).
 __host__ __device__ constexpr bool mode_selects_2of4(int mode)
 {
-    return mode == kModeSelectIdx || mode == kModeSelectIdxPacked || mode == kModeSelectIdxFlips || mode == kModeSelectIdxFlipsDense;
+    return mode == kModeSelectIdx || mode == kModeSelectIdxPacked || mode == kModeSelectIdxFlips || mode == kModeSelectIdxFlipsDense ||
+           mode == kModeSelectIdxFlipsDenseScaled;
 }
 // Modes that exist for M = 4 only.
-__host__ __device__ constexpr bool mode_is_2of4_only(int mode) { return mode_selects_2of4(mode) || mode == kModeReuseIdx || mode == kModeReuseIdxDense; }
+__host__ __device__ constexpr bool mode_is_2of4_only(int mode)
+{
+    return mode_selects_2of4(mode) || mode == kModeReuseIdx || mode == kModeReuseIdxDense || mode == kModeReuseIdxDenseScaled;
+}
 
 // One matrix as the kernel sees it.
 struct TensorDesc {
@@ -255,6 +262,8 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
     else if constexpr (MODE == kModeSelectIdxFlips) return kReselect | kCountFlips;
     else if constexpr (MODE == kModeSelectMaskFlips) return kReselect | kMetaBitmask | kCountFlips;
     else if constexpr (MODE == kModeSelectIdxFlipsDense) return kReselect | kCountFlips | kEmitDense;
+    else if constexpr (MODE == kModeReuseIdxDenseScaled) return kEmitDense | kGradOfScaled;
+    else if constexpr (MODE == kModeSelectIdxFlipsDenseScaled) return kReselect | kCountFlips | kEmitDense | kGradOfScaled;
     else return c.flags;
 }
 

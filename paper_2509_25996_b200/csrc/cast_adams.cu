@@ -174,6 +174,9 @@ int mode_of(const StepConsts& c, int M)
         case kEmitDense:                               return two_four ? kModeReuseIdxDense : kModeGeneric;
         case kReselect | kCountFlips:                  return two_four ? kModeSelectIdxFlips : kModeGeneric;
         case kReselect | kCountFlips | kEmitDense:     return two_four ? kModeSelectIdxFlipsDense : kModeGeneric;
+        case kEmitDense | kGradOfScaled:               return two_four ? kModeReuseIdxDenseScaled : kModeGeneric;
+        case kReselect | kCountFlips | kEmitDense | kGradOfScaled:
+                                                       return two_four ? kModeSelectIdxFlipsDenseScaled : kModeGeneric;
         case kReselect | kMetaBitmask:                 return kModeSelectMask;
         case kReselect | kMetaBitmask | kCountFlips:   return kModeSelectMaskFlips;
     }

@@ -63,6 +63,31 @@ def test_step_with_gradient_of_scaled_weight(rows, cols, n_seg, N, M, extra):
     assert_scale_grad(sg.cpu().numpy(), inp, ref["scale_grad"], n_seg, f"scale grad {rows}x{cols}/{n_seg}")
 
 
+@pytest.mark.parametrize("flags", [B.CAST_F_EMIT_DENSE | GS, RS | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE | GS])
+def test_training_steps_with_a_learned_scale(flags):
+    """The two steps of training with a learned scale (Alg. 2 with Eq. 12): the common one (stored mask, dense
+    forward weight, gradient through the scaling) and the refresh one (mask reselected, flips counted)."""
+    rows, cols, n_seg = 9, 2080, 2
+    inp = scaled_inputs(rows, cols, n_seg, seed=230)
+    h = Hyper()
+    stored = U.run_oracle(scaled_inputs(rows, cols, n_seg, seed=231), 2, 4, h, RS)["meta"]
+    st = U.to_device(inp, DEV, stored)
+    sg = torch.zeros((rows, n_seg), dtype=torch.float32, device=DEV)
+    flips = torch.zeros(1, dtype=torch.int64, device=DEV)
+    t = B.make_tensor(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale, n_seg, rows, cols, sg)
+    cast.check(cast.cast_adams_step_ex(t, 2, 4, hyper_struct(h, flags), flips, torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    assert st.all_intact()
+    ref = U.run_oracle(inp, 2, 4, h, flags, meta_in=stored)
+    got = U.device_outputs(st)
+    U.assert_parity(got, ref, f"learned scale, flags {flags}")
+    assert_scale_grad(sg.cpu().numpy(), inp, ref["scale_grad"], n_seg, "scale grad")
+    if flags & B.CAST_F_COUNT_FLIPS:
+        assert int(flips.item()) == ref["flips"] > 0
+    else:
+        assert np.array_equal(got["meta"], stored)
+
+
 def test_scale_gradient_is_added_and_optional_and_plain_step_is_unchanged():
     rows, cols, n_seg = 6, 1056, 2
     inp = scaled_inputs(rows, cols, n_seg, seed=210)
