@@ -166,6 +166,17 @@ CAST_API int cast_scale_adam_step(float* a, float* m_a, float* v_a, float* grad,
                          int clear_grad, cast_stream_t stream);
 
 /*
+ * cast_plan_scale_adam_step -- cast_scale_adam_step for the scale matrix of every matrix of a plan in one launch.
+ * The scales and their gradients are the `scale` and `scale_grad` buffers the plan's descriptors name (every matrix
+ * must have both; the scale buffers are UPDATED by this call although the descriptor declares them const for the
+ * step); `m_a` and `v_a` are HOST arrays of n_tensors device pointers to the two moments of each scale matrix
+ * (fp32 [rows * scale_groups]).  Other arguments as cast_scale_adam_step.
+ */
+CAST_API int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* const* v_a,
+                              float lr, float beta1, float beta2, float eps, int64_t step,
+                              int clear_grad, cast_stream_t stream);
+
+/*
  * Multi-tensor plan: the AdamS iteration of Alg. 1 over "each parameter theta in Theta", i.e. over
  * every prunable matrix of the model, in ONE kernel launch per 320 matrices.
  *

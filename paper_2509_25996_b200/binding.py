@@ -36,7 +36,7 @@ CAST_F_EMIT_COMPRESSED = 1 << 5
 CAST_F_GRAD_OF_SCALED = 1 << 6
 
 EXPORTS = (
-    "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
+    "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_scale_adam_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
@@ -98,6 +98,10 @@ def load_library() -> ctypes.CDLL:
     lib.cast_scale_adam_step.restype = ctypes.c_int
     lib.cast_scale_adam_step.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_float,
                                                                  ctypes.c_float, ctypes.c_int64, ctypes.c_int, ctypes.c_void_p]
+    lib.cast_plan_scale_adam_step.restype = ctypes.c_int
+    lib.cast_plan_scale_adam_step.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_void_p),
+                                              ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_int64,
+                                              ctypes.c_int, ctypes.c_void_p]
     lib.cast_plan_create.restype = ctypes.c_int
     lib.cast_plan_create.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                      ctypes.POINTER(ctypes.c_void_p)]
@@ -187,6 +191,14 @@ def cast_adams_step(w, m, v, g, w_fwd_bf16, meta, scale, scale_groups, rows, col
         _ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd_bf16), _ptr(meta), _ptr(scale), int(scale_groups),
         int(rows), int(cols), int(N), int(M), lr, beta1, beta2, eps, l1_coeff, int(step), int(total_steps),
         int(flags), _ptr(flip_count), _stream(stream))
+
+
+def cast_plan_scale_adam_step(plan, m_as, v_as, lr, beta1, beta2, eps, step, clear_grad=True, stream=None) -> int:
+    """`m_as`, `v_as`: sequences of one moment buffer per matrix of the plan."""
+    pm = None if m_as is None else (ctypes.c_void_p * len(m_as))(*[_ptr(x) for x in m_as])
+    pv = None if v_as is None else (ctypes.c_void_p * len(v_as))(*[_ptr(x) for x in v_as])
+    return load_library().cast_plan_scale_adam_step(plan, pm, pv, lr, beta1, beta2, eps, int(step), 1 if clear_grad else 0,
+                                                    _stream(stream))
 
 
 def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols, scale_grad=None) -> cast_tensor_t:

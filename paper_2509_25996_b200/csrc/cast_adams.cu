@@ -258,20 +258,20 @@ int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long
     return CAST_ERR_NM;
 }
 
-void fill_hints(MultiParams* p)
+void fill_hint_table(uint32_t n_tensors, const uint32_t* tile_start, uint16_t* hint, uint32_t* hint_shift)
 {
-    const uint64_t tiles = p->tile_start[p->n_tensors];
+    const uint64_t tiles = tile_start[n_tensors];
     uint32_t shift = 0;
     while (((tiles + (1ull << shift) - 1) >> shift) > (uint64_t)kHintEntries) ++shift;
-    p->hint_shift = shift;
+    *hint_shift = shift;
     const size_t n_hints = (size_t)((tiles + (1ull << shift) - 1) >> shift);
     size_t k = 0;
     for (size_t b = 0; b < (size_t)kHintEntries; ++b) {
         if (b < n_hints) {
             const uint64_t first = (uint64_t)b << shift;
-            while (first >= p->tile_start[k + 1]) ++k;
+            while (first >= tile_start[k + 1]) ++k;
         }
-        p->hint[b] = (uint16_t)k;
+        hint[b] = (uint16_t)k;
     }
 }
 

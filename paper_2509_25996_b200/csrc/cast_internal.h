@@ -63,8 +63,14 @@ int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long
                   cudaStream_t stream);
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
 
-// Fill hint_shift and hint[] of a table whose n_tensors and tile_start[] are set.
-void fill_hints(MultiParams* p);
+// Fill the tile-to-matrix hint table (kHintEntries entries) of a launch whose tile_start[0..n_tensors] is set:
+// hint[b] = the matrix that holds tile b << *hint_shift.
+void fill_hint_table(uint32_t n_tensors, const uint32_t* tile_start, uint16_t* hint, uint32_t* hint_shift);
+inline void fill_hints(MultiParams* p) { fill_hint_table(p->n_tensors, p->tile_start, p->hint, &p->hint_shift); }
+
+// Host-side view of a plan (for the entry points that work on a plan's matrices).
+int plan_tensor_count(const void* plan);
+bool plan_tensor_desc(const void* plan, int i, int* N, int* M, TensorDesc* desc);
 
 // A grid holds at most this many tiles (one CTA per tile, gridDim.x < 2^31).
 constexpr uint64_t kMaxTiles = 0x7FFFFFFFull;

@@ -15,8 +15,6 @@
 
 namespace cast {
 
-// Host-side view of a plan, for the statistics pass (defined with the plan in cast_adams.cu).
-int plan_tensor_count(const void* plan);
 bool plan_tensor(const void* plan, int i, int* M, const float** w, const uint32_t** meta, uint32_t* n_units);
 
 namespace {
@@ -115,26 +113,9 @@ mask_stats_kernel(const __grid_constant__ StatsParams p, bool bitmask, cast_mask
     }
 }
 
-void fill_stats_hints(StatsParams* p)
-{
-    const uint64_t tiles = p->tile_start[p->n_tensors];
-    uint32_t shift = 0;
-    while (((tiles + (1ull << shift) - 1) >> shift) > (uint64_t)kHintEntries) ++shift;
-    p->hint_shift = shift;
-    const size_t n_hints = (size_t)((tiles + (1ull << shift) - 1) >> shift);
-    size_t k = 0;
-    for (size_t b = 0; b < (size_t)kHintEntries; ++b) {
-        if (b < n_hints) {
-            const uint64_t first = (uint64_t)b << shift;
-            while (first >= p->tile_start[k + 1]) ++k;
-        }
-        p->hint[b] = (uint16_t)k;
-    }
-}
-
 int launch_stats(StatsParams* p, bool bitmask, cast_mask_stats_t* stats, cudaStream_t s)
 {
-    fill_stats_hints(p);
+    fill_hint_table(p->n_tensors, p->tile_start, p->hint, &p->hint_shift);
     const uint32_t tiles = p->tile_start[p->n_tensors];
     if (tiles == 0) return CAST_OK;
     mask_stats_kernel<<<tiles, kStatsThreads, 0, s>>>(*p, bitmask, stats);

@@ -11,10 +11,6 @@
 
 namespace cast {
 
-// Host-side view of a plan (defined with the plan in cast_adams.cu).
-int plan_tensor_count(const void* plan);
-bool plan_tensor_desc(const void* plan, int i, int* N, int* M, TensorDesc* desc);
-
 namespace {
 
 // One matrix of a pruning launch, and the tables of the launch (kernel parameter space, like the step's).
@@ -108,23 +104,6 @@ prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t fl
 
 inline uint32_t prune_tiles(uint32_t n_units) { return (n_units + kPruneTileUnits - 1) / kPruneTileUnits; }
 
-void fill_prune_hints(PruneParams* p)
-{
-    const uint64_t tiles = p->tile_start[p->n_tensors];
-    uint32_t shift = 0;
-    while (((tiles + (1ull << shift) - 1) >> shift) > (uint64_t)kHintEntries) ++shift;
-    p->hint_shift = shift;
-    const size_t n_hints = (size_t)((tiles + (1ull << shift) - 1) >> shift);
-    size_t k = 0;
-    for (size_t b = 0; b < (size_t)kHintEntries; ++b) {
-        if (b < n_hints) {
-            const uint64_t first = (uint64_t)b << shift;
-            while (first >= p->tile_start[k + 1]) ++k;
-        }
-        p->hint[b] = (uint16_t)k;
-    }
-}
-
 template <int M>
 int launch_t(const PruneParams& p, int N, uint32_t flags, cudaStream_t s)
 {
@@ -136,7 +115,7 @@ int launch_t(const PruneParams& p, int N, uint32_t flags, cudaStream_t s)
 
 int launch(PruneParams* p, int N, int M, uint32_t flags, cudaStream_t s)
 {
-    fill_prune_hints(p);
+    fill_hint_table(p->n_tensors, p->tile_start, p->hint, &p->hint_shift);
     if (p->tile_start[p->n_tensors] == 0) return CAST_OK;
     switch (M) {
         case 2:  return launch_t<2>(*p, N, flags, s);

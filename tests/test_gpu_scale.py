@@ -164,6 +164,45 @@ def test_plan_with_scale_gradients_then_scale_adam():
     assert all(s.all_intact() for s in states)
 
 
+def test_plan_scale_adam_one_launch():
+    """The Adam step of every scale matrix of a plan in one grid (scale matrices of 2 to 600 entries)."""
+    shapes = [(1, 64), (3, 96), (64, 1056), (300, 64), (33, 2048)]
+    ins = [scaled_inputs(r, c, 2, seed=240 + i) for i, (r, c) in enumerate(shapes)]
+    states = [U.to_device(inp, DEV) for inp in ins]
+    rng = np.random.default_rng(7)
+    grads_h = [rng.normal(0, 1e-2, size=(r, 2)).astype(np.float32) for r, _ in shapes]
+    grads = [torch.from_numpy(g.copy()).to(DEV) for g in grads_h]
+    m_as = [torch.zeros(r * 2, device=DEV) for r, _ in shapes]
+    v_as = [torch.zeros(r * 2, device=DEV) for r, _ in shapes]
+    tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale, 2, s.rows, s.cols, gr)
+               for s, gr in zip(states, grads)]
+    rc, plan = cast.cast_plan_create(tensors, 2, 4)
+    cast.check(rc)
+    lr_a = float(np.float32(1e-3))
+    before = cast.cast_kernel_launch_count()
+    cast.check(cast.cast_plan_scale_adam_step(plan, m_as, v_as, lr_a, 0.9, 0.95, 1e-8, 3, True, torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == before + 1
+    for s, inp, gh, gr, ma, va in zip(states, ins, grads_h, grads, m_as, v_as):
+        n = s.rows * 2
+        th, mm, vv = orc.plain_adam(inp.scale.numpy().reshape(-1), np.zeros(n, np.float32), np.zeros(n, np.float32),
+                                    gh.reshape(-1), lr_a, 0.9, 0.95, 1e-8, 3)
+        for got, want in ((s.scale, th), (ma, mm), (va, vv)):
+            assert np.allclose(got.cpu().numpy().reshape(-1), want, rtol=1e-6, atol=1e-30)
+        assert float(gr.abs().max().item()) == 0.0
+        assert s.all_intact()
+    assert cast.cast_plan_scale_adam_step(plan, None, v_as, lr_a, 0.9, 0.95, 1e-8, 3) == B.CAST_ERR_NULL
+    assert cast.cast_plan_scale_adam_step(None, m_as, v_as, lr_a, 0.9, 0.95, 1e-8, 3) == B.CAST_ERR_PLAN
+    assert cast.cast_plan_scale_adam_step(plan, m_as, v_as, lr_a, 0.9, 0.95, 1e-8, 0) == B.CAST_ERR_HYPER
+    cast.check(cast.cast_plan_destroy(plan))
+    # a plan whose matrices carry no scale gradient cannot train the scale
+    tensors = [B.make_tensor(s.w.view, s.m.view, s.v.view, s.g.view, s.w_fwd.view, s.meta.view, s.scale, 2, s.rows, s.cols) for s in states]
+    rc, plan = cast.cast_plan_create(tensors, 2, 4)
+    cast.check(rc)
+    assert cast.cast_plan_scale_adam_step(plan, m_as, v_as, lr_a, 0.9, 0.95, 1e-8, 3) == B.CAST_ERR_NULL
+    cast.check(cast.cast_plan_destroy(plan))
+
+
 def test_scale_adam_rejections():
     x = torch.zeros(64, dtype=torch.float32, device=DEV)
     y, z, g = x.clone(), x.clone(), x.clone()
