@@ -57,6 +57,9 @@ def parse_args():
                    help="every-step: reselect the mask at every step (the headline, worst case); t1: the paper's training "
                         "schedule (Sec. 4.1, App. C): stored mask and dense forward weight, mask refreshed and flips counted "
                         "every 10th step")
+    p.add_argument("--learned-scale", action="store_true",
+                   help="with --schedule t1: the gradient is taken through the weight scaling (Eq. 12), the scale gradient is "
+                        "accumulated by the step and every scale matrix takes its own Adam step in each iteration")
     p.add_argument("--seed", type=int, default=0)
     p.add_argument("--op", choices=["step", "mask_stats", "prune_fold", "kd_loss"], default="step",
                    help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass; prune_fold: the "
@@ -259,7 +262,8 @@ def cuda_arm(args):
         mats = state.slots[0].mats
         oracle_repeats = len(wl.shapes) // wl.layer_matrices // wl.resident_layers   # steps a slot takes per pass
     else:
-        state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones", compressed=compressed)
+        state = DeviceModelState(wl.shapes, N, M, seed=args.seed, device=dev, scale_mode="ones", compressed=compressed,
+                                 learned_scale=args.learned_scale)
         mats = state.mats
         oracle_repeats = 1
     hyper = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl.total_steps)
@@ -267,8 +271,9 @@ def cuda_arm(args):
     if args.schedule == "t1":
         if (N, M) != (2, 4) or args.emit != "pruned" or wl.resident_layers or args.count_flips:
             raise SystemExit("--schedule t1 is wired for 2:4 on a resident workload")
-        refresh = B.CAST_F_RESELECT | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE
-        between = B.CAST_F_EMIT_DENSE
+        scaled = B.CAST_F_GRAD_OF_SCALED if args.learned_scale else 0
+        refresh = B.CAST_F_RESELECT | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE | scaled
+        between = B.CAST_F_EMIT_DENSE | scaled
         state.step(hyper, B.CAST_F_RESELECT, stream)           # establishes the stored mask (untimed)
         # reuse steps move 28.125 B/param (the metadata is read, not rewritten), refresh steps 28.25
         bytes_per_param = 28.125 + 0.125 / 10
@@ -277,8 +282,17 @@ def cuda_arm(args):
         def flags_at(step_no):
             return refresh if step_no % 10 == 0 else between
     else:
+        if args.learned_scale:
+            raise SystemExit("--learned-scale goes with --schedule t1")
+
         def flags_at(step_no):
             return flags
+
+    def one_step():
+        state.step(hyper, flags_at(hyper.step), stream)
+        if args.learned_scale:
+            state.scale_step(1e-3, hyper, stream)
+        hyper.step += 1
 
     # parity sample (checked in the CPU-baseline leg): a few rows of the first and last matrices, copied
     # before the first step and again after it
@@ -300,8 +314,7 @@ def cuda_arm(args):
     sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid)) if rank == 0 else None
     parity_out = {}
     for i in range(args.warmup):
-        state.step(hyper, flags_at(hyper.step), stream)
-        hyper.step += 1
+        one_step()
         if i == 0 and parity_in:
             torch.cuda.synchronize(dev)
             for t in picks:
@@ -326,8 +339,7 @@ def cuda_arm(args):
     if flush is None:
         ev0.record(stream)
         for _ in range(args.steps):
-            state.step(hyper, flags_at(hyper.step), stream)
-            hyper.step += 1
+            one_step()
         ev1.record(stream)
         barrier()
         ms_local = ev0.elapsed_time(ev1)
@@ -363,6 +375,8 @@ def cuda_arm(args):
         clocks = sampler.summary(t_wall0, t_wall1)
 
     ms_per_step = ms / args.steps
+    # launches of the step kernel per step: one per resident-layer call, else one per 320 matrices
+    step_launches = (len(wl.shapes) // wl.layer_matrices) if wl.resident_layers else -(-len(wl.shapes) // 320)
     per_gpu_gbs = wl.n_params * bytes_per_param / (ms_per_step * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
 
@@ -473,7 +487,7 @@ def cuda_arm(args):
                                                                                   else "L2 flushed by a 512 MB write before every step, steps timed one by one"),
                    "resident_layers": wl.resident_layers, "streams": 2 if wl.resident_layers else 1,
                    "lr": hyper.lr, "betas": [hyper.beta1, hyper.beta2], "eps": hyper.eps, "l1_coeff": hyper.l1_coeff,
-                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "schedule": args.schedule, "seed": args.seed},
+                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "schedule": args.schedule, "learned_scale": bool(args.learned_scale), "seed": args.seed},
         "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
         "warm_l2": (None if warm_ms_per_step is None else
                     {"ms_per_step": warm_ms_per_step, "value": wl.n_params / (warm_ms_per_step * 1e-3),
@@ -482,10 +496,10 @@ def cuda_arm(args):
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
                      "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}>",
                      "bytes_per_param": bytes_per_param,
-                     "launches_per_step": launches // args.steps,
-                     "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params * args.steps / max(launches, 1),
+                     "launches_per_step": step_launches,
+                     "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,
                      "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None or args.emit != "pruned" or args.count_flips or (N, M) != (2, 4) or args.schedule != "every-step"
-                                 else NCU_DRAM_BYTES_PER_PARAM * wl.n_params * args.steps / max(launches, 1))},
+                                 else NCU_DRAM_BYTES_PER_PARAM * wl.n_params / step_launches)},
         "cpu_baseline": cpu_baseline, "parity": parity,
     }
     if world > 1:

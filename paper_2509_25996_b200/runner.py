@@ -25,6 +25,9 @@ class MatrixState:
     w_fwd: torch.Tensor
     meta: torch.Tensor                 # int32 [rows, cols/32]
     scale: Optional[torch.Tensor]
+    scale_grad: Optional[torch.Tensor] = None      # fp32 [rows, n]; with a learned scale
+    scale_m: Optional[torch.Tensor] = None         # Adam moments of the scale
+    scale_v: Optional[torch.Tensor] = None
 
 
 @dataclass
@@ -42,9 +45,12 @@ class DeviceModelState:
     """All prunable matrices of a model on one GPU plus the plan that steps them in one launch."""
 
     def __init__(self, shapes: Sequence[Tuple[int, int]], N: int = 2, M: int = 4, seed: int = 0,
-                 device="cuda:0", scale_mode: str = "ones", first_tensor_index: int = 0, compressed: bool = False):
+                 device="cuda:0", scale_mode: str = "ones", first_tensor_index: int = 0, compressed: bool = False,
+                 learned_scale: bool = False):
         """compressed: the forward-weight buffers hold only the kept entries ([rows, cols*N/M]); every step of
-        this state then carries CAST_F_EMIT_COMPRESSED."""
+        this state then carries CAST_F_EMIT_COMPRESSED.
+        learned_scale: every matrix gets a scale-gradient buffer (filled by steps that carry
+        CAST_F_GRAD_OF_SCALED) and Adam moments for its scale; scale_step() then trains the scales."""
         self.device = torch.device(device)
         self.N, self.M = N, M
         self.compressed = compressed
@@ -57,10 +63,17 @@ class DeviceModelState:
                 torch.empty((rows, cols * N // M if compressed else cols), dtype=torch.bfloat16, device=self.device),
                 torch.zeros((rows, cols // 32), dtype=torch.int32, device=self.device),
                 inp.scale))
+            if learned_scale:
+                if inp.scale is None:
+                    raise ValueError("a learned scale needs a scale tensor")
+                mat = self.mats[-1]
+                mat.scale_grad = torch.zeros_like(inp.scale)
+                mat.scale_m = torch.zeros_like(inp.scale)
+                mat.scale_v = torch.zeros_like(inp.scale)
         self.n_params = sum(s.rows * s.cols for s in self.mats)
         self.flips = torch.zeros(1, dtype=torch.int64, device=self.device)
         tensors = [B.make_tensor(s.w, s.m, s.v, s.g, s.w_fwd, s.meta, s.scale,
-                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols) for s in self.mats]
+                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad) for s in self.mats]
         rc, self.plan = B.cast_plan_create_ex(tensors, N, M, B.CAST_F_EMIT_COMPRESSED if compressed else 0)
         B.check(rc)
 
@@ -72,6 +85,12 @@ class DeviceModelState:
                          hyper.step, hyper.total_steps, flags)
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
         B.check(B.cast_plan_step(self.plan, h, self.flips if flags & B.CAST_F_COUNT_FLIPS else None, s))
+
+    def scale_step(self, lr: float, hyper: Hyper, stream=None) -> None:
+        """Adam step of every scale matrix from the accumulated scale gradients (which it clears), one launch."""
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        B.check(B.cast_plan_scale_adam_step(self.plan, [m.scale_m for m in self.mats], [m.scale_v for m in self.mats],
+                                            lr, hyper.beta1, hyper.beta2, hyper.eps, hyper.step, True, s))
 
     def close(self) -> None:
         if self.plan is not None:
