@@ -340,7 +340,7 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
         u.m[i] = mu_f;
         // proportional L1 decay outside the kept set (Eq. 7): alpha lambda Sign(w), Sign(+-0) = 0
         const bool w_zero = ab[i] == 0u;
-        const double sgn_term = __hiloint2double(w_zero ? 0 : (sign_hi | (int)(__float_as_uint(u.w[i]) & 0x80000000u)),
+        const double sgn_term = __hiloint2double(w_zero ? 0 : (sign_hi ^ (int)(__float_as_uint(u.w[i]) & 0x80000000u)),
                                                  w_zero ? 0 : sign_lo);
         const float mu_t = kept[i] ? mu_f : (float)fma(c.c_mu, mu, sgn_term);
         // second moment from the decayed first moment (Eq. 8)

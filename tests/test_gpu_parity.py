@@ -201,6 +201,25 @@ def test_two_runs_are_bit_identical():
         assert np.array_equal(a[k].view(np.uint8), b[k].view(np.uint8))
 
 
+@pytest.mark.parametrize("case", range(12))
+def test_random_hyper_parameters(case):
+    """Hyper-parameters drawn over their useful ranges (first steps with small bias corrections, alpha from 1/T to 1,
+    beta1 = 0, eps from 1e-12 to 1e-6, zero and negative decay coefficients), learning rates for which the
+    tolerance is reachable in fp32 (update below ~1e-3 per step)."""
+    rng = np.random.default_rng(1000 + case)
+    N, M = [(2, 4), (2, 4), (4, 8), (1, 4)][case % 4]
+    total = int(rng.choice([1, 10, 7500, 10 ** 6]))
+    step = int(rng.integers(1, total + 1)) if case % 3 else 1
+    h = Hyper(lr=float(10 ** rng.uniform(-6, -3.9)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.99])),
+              beta2=float(rng.choice([0.9, 0.95, 0.999])), eps=float(10 ** rng.uniform(-12, -6)),
+              l1_coeff=float(rng.choice([0.0, 1e-4, 1e-3, -1e-3])), step=step, total_steps=max(total, step))
+    flags = RS | (0 if (N, M) == (2, 4) and case % 2 else BM) | (B.CAST_F_COUNT_FLIPS if case % 5 == 0 else 0)
+    inp = inputs(11, 1056, seed=500 + case)
+    prev = U.run_oracle(inputs(11, 1056, seed=600 + case), N, M, Hyper(), RS | (flags & BM))["meta"]
+    got = U.run_cuda_single(inp, N, M, h, flags, meta_in=prev)
+    U.assert_parity(got, U.run_oracle(inp, N, M, h, flags, meta_in=prev), f"case {case}: {h}")
+
+
 def test_resumed_run_is_bit_identical():
     """The library keeps no state of its own: w, m, v, the metadata and the step number are the whole checkpoint.
     Two steps in a row equal one step, a round trip of the state through host memory into fresh buffers, and the
