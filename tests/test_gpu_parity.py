@@ -220,6 +220,43 @@ def test_random_hyper_parameters(case):
     U.assert_parity(got, U.run_oracle(inp, N, M, h, flags, meta_in=prev), f"case {case}: {h}")
 
 
+@pytest.mark.parametrize("case", range(48))
+def test_random_shapes_patterns_and_flag_combinations(case):
+    """Every valid combination of flags can be asked for at run time; most take the run-time-flag mode of the
+    kernel.  Shapes, N:M, scale segments and flags are drawn at random (seeded)."""
+    rng = np.random.default_rng(2000 + case)
+    M = int(rng.choice([2, 4, 8, 16, 32]))
+    N = int(rng.integers(1, M + 1))
+    if case % 4 == 0:
+        N, M = 2, 4
+    n_seg = int(rng.choice([1, 2, 4]))
+    seg = max(M, 8) * int(rng.integers(1, 40))
+    while (seg * n_seg) % 32:
+        seg += max(M, 8)
+    rows, cols = int(rng.integers(1, 10)), seg * n_seg
+    flags = 0
+    if rng.random() < 0.7:
+        flags |= RS
+    if (N, M) != (2, 4) or rng.random() < 0.5:
+        flags |= BM
+    for bit, p in ((B.CAST_F_COUNT_FLIPS, 0.4), (B.CAST_F_V_KEPT_FROM_G, 0.3), (B.CAST_F_GRAD_OF_SCALED, 0.4)):
+        if rng.random() < p:
+            flags |= bit
+    emit = rng.random()
+    if emit < 0.3:
+        flags |= B.CAST_F_EMIT_DENSE
+    elif emit < 0.6 and M <= 8:
+        flags |= B.CAST_F_EMIT_COMPRESSED
+    inp = inputs(rows, cols, seed=700 + case, scale_mode=("none" if rng.random() < 0.2 else "jitter"))
+    if inp.scale is not None:
+        gen = torch.Generator().manual_seed(case)
+        inp.scale = 0.5 + torch.rand((rows, n_seg), generator=gen)
+    h = Hyper(l1_coeff=float(rng.choice([1e-3, 0.0, 1e-2])), step=int(rng.integers(1, 2000)), total_steps=2000)
+    prev = U.run_oracle(inputs(rows, cols, seed=800 + case, scale_mode="none"), N, M, Hyper(), RS | (flags & BM))["meta"]
+    got = U.run_cuda_single(inp, N, M, h, flags, meta_in=prev)
+    U.assert_parity(got, U.run_oracle(inp, N, M, h, flags, meta_in=prev), f"case {case}: {N}:{M} {rows}x{cols}/{n_seg} flags {flags:#x}")
+
+
 def test_resumed_run_is_bit_identical():
     """The library keeps no state of its own: w, m, v, the metadata and the step number are the whole checkpoint.
     Two steps in a row equal one step, a round trip of the state through host memory into fresh buffers, and the
