@@ -106,6 +106,71 @@ def test_plan_decoder_d768_12_layers_full():
     print(f"near-tie groups: {ties} of {wl.n_params // 4}; mask mismatches: 0")
 
 
+@pytest.mark.parametrize("case", range(16))
+def test_random_plans(case):
+    """Random lists of matrices, N:M, flags, scale segments and scale-gradient buffers through the multi-tensor path."""
+    rng = np.random.default_rng(3000 + case)
+    M = int(rng.choice([2, 4, 8, 16, 32]))
+    N = int(rng.integers(1, M + 1))
+    if case % 3 == 0:
+        N, M = 2, 4
+    flags = RS if rng.random() < 0.7 else 0
+    if (N, M) != (2, 4) or rng.random() < 0.5:
+        flags |= BM
+    for bit, p in ((B.CAST_F_COUNT_FLIPS, 0.5), (B.CAST_F_V_KEPT_FROM_G, 0.2), (B.CAST_F_GRAD_OF_SCALED, 0.5)):
+        if rng.random() < p:
+            flags |= bit
+    compressed = M <= 8 and rng.random() < 0.4
+    if compressed:
+        flags |= B.CAST_F_EMIT_COMPRESSED
+    elif rng.random() < 0.4:
+        flags |= B.CAST_F_EMIT_DENSE
+    h = Hyper(step=int(rng.integers(1, 500)), total_steps=500)
+    ins, states, grads, prevs, tensors = [], [], [], [], []
+    for i in range(int(rng.integers(1, 13))):
+        n_seg = int(rng.choice([1, 2, 4]))
+        seg = max(M, 8) * int(rng.integers(1, 30))
+        while (seg * n_seg) % 32:
+            seg += max(M, 8)
+        rows, cols = int(rng.integers(1, 8)), seg * n_seg
+        inp = workloads.gen_tensor_inputs(rows, cols, seed=900 + case, tensor_index=i, scale_mode="jitter")
+        gen = torch.Generator().manual_seed(case * 100 + i)
+        inp.scale = None if rng.random() < 0.25 else 0.5 + torch.rand((rows, n_seg), generator=gen)
+        prev = U.run_oracle(workloads.gen_tensor_inputs(rows, cols, seed=950 + case, tensor_index=i, scale_mode="none"),
+                            N, M, Hyper(), RS | (flags & BM))["meta"]
+        st = U.to_device(inp, DEV, prev, rows * cols * N // M if compressed else None)
+        sg = None
+        if inp.scale is not None and rng.random() < 0.7:
+            sg = torch.zeros((rows, n_seg), dtype=torch.float32, device=DEV)
+        ins.append(inp); states.append(st); grads.append(sg); prevs.append(prev)
+        tensors.append(B.make_tensor(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale,
+                                     1 if st.scale is None else n_seg, rows, cols, sg))
+    rc, plan = cast.cast_plan_create_ex(tensors, N, M, B.CAST_F_EMIT_COMPRESSED if compressed else 0)
+    cast.check(rc)
+    flips = torch.zeros(1, dtype=torch.int64, device=DEV)
+    lr, b1, b2, eps, lam = h.as_f32()
+    cast.check(cast.cast_plan_step(plan, B.make_hyper(lr, b1, b2, eps, lam, h.step, h.total_steps, flags), flips,
+                                   torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    cast.check(cast.cast_plan_destroy(plan))
+    total = 0
+    for i, (inp, st, sg, prev) in enumerate(zip(ins, states, grads, prevs)):
+        assert st.all_intact()
+        ref = U.run_oracle(inp, N, M, h, flags, meta_in=prev)
+        got = U.device_outputs(st)
+        U.assert_parity(got, ref, f"case {case} tensor {i}: {N}:{M} {inp.w.shape} flags {flags:#x}")
+        total += ref["flips"]
+        if sg is not None and flags & B.CAST_F_GRAD_OF_SCALED:
+            rows, cols = inp.w.shape
+            n_seg = inp.scale.shape[1]
+            bound = 2e-6 * np.abs(inp.g.double().numpy() * inp.w.double().numpy()).reshape(rows, n_seg, cols // n_seg).sum(-1) + 1e-30
+            assert np.all(np.abs(sg.cpu().numpy().astype(np.float64) - ref["scale_grad"]) <= bound)
+        elif sg is not None:
+            assert float(sg.abs().max().item()) == 0.0            # untouched without the flag
+    if flags & B.CAST_F_COUNT_FLIPS:
+        assert int(flips.item()) == total
+
+
 def test_plan_step_replayed_from_a_cuda_graph():
     """A plan step is one kernel launch whose tables travel as parameters, so it can be recorded into a CUDA graph
     and replayed: three replays are three iterations with the recorded hyper-parameters."""
