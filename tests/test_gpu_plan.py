@@ -332,6 +332,51 @@ def test_host_step_blocks_match_oracle(block, slots):
     cast.check(cast.cast_host_ctx_destroy(ctx))
 
 
+@pytest.mark.parametrize("case", range(10))
+def test_random_host_steps(case):
+    """Host-resident state through staged blocks (allocated slots and the built-in staging area) with random shapes,
+    block sizes, N:M and flags."""
+    rng = np.random.default_rng(4000 + case)
+    N, M = [(2, 4), (4, 8), (1, 4), (2, 4), (3, 8)][case % 5]
+    flags = (RS if rng.random() < 0.8 else 0) | (0 if (N, M) == (2, 4) and rng.random() < 0.5 else BM)
+    if rng.random() < 0.5:
+        flags |= B.CAST_F_COUNT_FLIPS
+    emit = rng.random()
+    if emit < 0.3:
+        flags |= B.CAST_F_EMIT_COMPRESSED
+    elif emit < 0.6:
+        flags |= B.CAST_F_EMIT_DENSE
+    rows, cols = int(rng.integers(1, 60)), 64 * int(rng.integers(1, 20))
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=4100 + case, scale_mode=("jitter" if rng.random() < 0.7 else "none"))
+    prev = U.run_oracle(workloads.gen_tensor_inputs(rows, cols, seed=4200 + case, scale_mode="none"), N, M, Hyper(), RS | (flags & BM))["meta"]
+    h = Hyper(step=int(rng.integers(1, 100)), total_steps=100)
+    ref = U.run_oracle(inp, N, M, h, flags, meta_in=prev)
+    lr, b1, b2, eps, lam = h.as_f32()
+    fcols = cols * N // M if flags & B.CAST_F_EMIT_COMPRESSED else cols
+    n_seg = 1 if inp.scale is None else inp.scale.shape[1]
+    block = max(1024, cols * int(rng.integers(1, 8)))
+    block += (-block) % 32
+    rc, ctx = cast.cast_host_ctx_create(block, int(rng.integers(2, 5)))
+    cast.check(rc)
+    for which in ("slots", "static"):
+        w, m, v = inp.w.clone(), inp.m.clone(), inp.v.clone()
+        fwd = torch.zeros((rows, fcols), dtype=torch.bfloat16)
+        meta = torch.from_numpy(prev.view(np.int32).copy())
+        flips = np.zeros(1, dtype=np.uint64)
+        if which == "slots":
+            cast.check(cast.cast_host_step(ctx, w, m, v, inp.g, fwd, meta, inp.scale, n_seg, rows, cols, N, M, lr, b1, b2, eps, lam,
+                                           h.step, h.total_steps, flags, flips))
+            cast.check(cast.cast_host_ctx_sync(ctx))
+        else:
+            cast.check(cast.cast_host_step_static(w, m, v, inp.g, fwd, meta, inp.scale, n_seg, rows, cols, N, M, lr, b1, b2, eps, lam,
+                                                  h.step, h.total_steps, flags, flips, None))
+        got = dict(w=w.numpy(), m=m.numpy(), v=v.numpy(), w_fwd=workloads.bf16_bits(fwd), meta=meta.numpy().view(np.uint32))
+        if flags & B.CAST_F_COUNT_FLIPS:
+            got["flips"] = int(flips[0])
+        U.assert_parity(got, ref, f"case {case} {which}: {N}:{M} {rows}x{cols} block {block} flags {flags:#x}")
+    cast.check(cast.cast_host_ctx_destroy(ctx))
+
+
 def test_host_step_pageable_memory():
     rows, cols = 8, 512
     inp = workloads.gen_tensor_inputs(rows, cols, seed=32, scale_mode="none")
