@@ -695,6 +695,12 @@ def kd_arm(args):
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
                      "kernel": "kd_loss_kernel", "bytes_per_logit": 6.0, "launches_per_step": 1, "traffic": None},
+        # the op needs four exponentials per logit on the special-function unit (16 lanes per SM and clock): at the
+        # maximum SM clock that is the same order as the HBM bound, so both are reported
+        "xu_roofline": {"bound": "alu", "unit": "logits/s", "achieved": T * V / (ms * 1e-3),
+                        "peak": torch.cuda.get_device_properties(dev).multi_processor_count * 16 * 1.965e9 / 4.0,
+                        "frac": (T * V / (ms * 1e-3)) / (torch.cuda.get_device_properties(dev).multi_processor_count * 16 * 1.965e9 / 4.0),
+                        "peak_kind": "derived: SMs x 16 ex2 per clock x 1.965 GHz / 4 ex2 per logit"},
         "mean_loss": float(loss.double().mean().item()),
         "parity": {"ok": ok, "sample": f"losses of the first {rows} tokens against the CPU oracle"}}), flush=True)
 
