@@ -11,6 +11,7 @@ from paper_2509_25996_b200 import workloads
 from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
 from oracle import adams_oracle as orc
 import gpu_util as U
+from helpers import within_tol
 
 pytestmark = pytest.mark.gpu
 
@@ -136,3 +137,45 @@ def test_llama2_7b_full_set_4_8_with_flips_sampled():
 
 def test_llama2_13b_layer_sampled():
     check_sampled("llama2_13b_layer", 2, 4, B.CAST_F_RESELECT, n_random=8, need_gb=8)
+
+
+def test_llama2_13b_streamed_full_sampled():
+    """LLaMA2-13B layer shapes, 40 layers in per-layer calls on 2 streams over 10 resident layer slots (51 GB): every
+    slot takes 4 steps per pass; sampled row blocks of slots 0 and 9 against 4 chained oracle steps."""
+    import gc
+    from paper_2509_25996_b200.runner import StreamedModelState
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 60e9:
+        pytest.skip("needs 60 GB of device memory")
+    wl = workloads.workload("llama2_13b")
+    layer = wl.shapes[:wl.layer_matrices]
+    st = StreamedModelState(layer, len(wl.shapes) // wl.layer_matrices, wl.resident_layers, 2, 2, 4, seed=0, device=DEV,
+                            scale_mode="jitter")
+    rng = np.random.default_rng(3)
+    picks = [(slot, t, int(rng.integers(0, layer[t][0] - 4))) for slot in (0, 9) for t in (0, 4, 6)]
+    before = []
+    for slot, t, r0 in picks:
+        m = st.slots[slot].mats[t]
+        sl = slice(r0, r0 + 4)
+        before.append(workloads.TensorInputs(m.w[sl].cpu(), m.g[sl].cpu(), m.m[sl].cpu(), m.v[sl].cpu(), m.scale[sl].cpu()))
+    h = RunHyper(total_steps=wl.total_steps)
+    launches = cast.cast_kernel_launch_count()
+    st.step(h, B.CAST_F_RESELECT)
+    torch.cuda.synchronize()
+    assert cast.cast_kernel_launch_count() == launches + 40
+    oh = orc.Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
+    for (slot, t, r0), inp in zip(picks, before):
+        cur = inp
+        for _ in range(4):
+            ref = U.run_oracle(cur, 2, 4, oh, B.CAST_F_RESELECT)
+            cur = workloads.TensorInputs(torch.from_numpy(ref["w"]), inp.g, torch.from_numpy(ref["m"]), torch.from_numpy(ref["v"]), inp.scale)
+        m = st.slots[slot].mats[t]
+        sl = slice(r0, r0 + 4)
+        got = dict(w=m.w[sl].cpu().numpy(), m=m.m[sl].cpu().numpy(), v=m.v[sl].cpu().numpy())
+        # four chained steps: the fp32 state of one step feeds the next, so the bound grows with the step count
+        for k in ("w", "m", "v"):
+            ok, worst = within_tol(got[k], ref[k], rel=4e-6, floor=4e-9)
+            assert ok, f"slot {slot} matrix {t} rows {r0}+ {k}: {worst:.3g}"
+    st.close()
