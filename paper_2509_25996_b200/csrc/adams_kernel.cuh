@@ -302,7 +302,15 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
         const bool need_prev = !(flags & kReselect) || (flags & kCountFlips);
         const uint32_t prev_keep = need_prev ? keep_from_meta_byte(u.prev_byte, bitmask) : 0u;
         uint32_t keep;
-        if (flags & kReselect) {
+        if ((flags & kReselect) && M == 4 && c.n_keep == 2) {       // uniform: 2:4 by the comparison network
+            select_2of4(ab, kept);
+            select_2of4(ab + 4, kept + 4);
+            keep = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) keep |= (kept[i] ? 1u : 0u) << i;
+            if (bitmask) u.meta_byte = keep;
+            else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+        } else if (flags & kReselect) {
             keep = select_by_rank<M>(ab, c.n_keep);     // uniform branch: all lanes shuffle
 #pragma unroll
             for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;

@@ -90,7 +90,7 @@ mask_stats_kernel(const __grid_constant__ StatsParams p, bool bitmask, cast_mask
             for (int i = 0; i < 8; ++i) {
                 const double m = (double)fabsf(x[i]);
                 total += m;
-                kept += ((keep >> i) & 1u) ? m : 0.0;
+                if ((keep >> i) & 1u) kept += m;
             }
         }
     }
