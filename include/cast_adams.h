@@ -107,6 +107,13 @@ enum cast_flags {
  *   N, M         keep N of every M consecutive columns; the kept set is chosen on the weights before
  *                this update, larger magnitude first, lower column first among equal magnitudes.
  *   lr           finite.  beta1, beta2 in [0, 1).  eps > 0.  l1_coeff (lambda of Eq. 7) finite.
+ *                Accuracy domain: the step is evaluated in fp32 (first-moment sums in fp64, approximate
+ *                square root and reciprocal with a relative error below ~5e-7 on the update term).  Its
+ *                results are within max(1e-6 relative, 1e-9 absolute) of an fp64 evaluation of Alg. 1 as
+ *                long as the per-step update |lr mu^ / (sqrt(v^) + eps)| stays below ~1e-3 (with
+ *                beta = 0.9/0.95 that is lr up to ~2e-4); for larger updates the error stays ~5e-7
+ *                RELATIVE TO THE UPDATE, which then exceeds the 1e-9 absolute floor for weights near
+ *                zero -- as it does for any fp32 evaluation, IEEE square root and division included.
  *   step         t >= 1;  total_steps  T >= t;  the decay weight is alpha_t = t/T.
  *   flags        OR of cast_flags.
  *   flip_count   device, one unsigned 64-bit counter the step ADDS to (the caller zeroes it); may be

@@ -125,17 +125,22 @@ class StreamedModelState:
         self.n_params = n_layers * self.slots[0].n_params
         self._done = [torch.cuda.Event() for _ in range(n_streams)]
 
-    def step(self, hyper: Hyper, flags: int, stream=None) -> None:
+    def step(self, hyper: Hyper, flags: int, stream=None, after_layer=None) -> None:
         """One AdamS iteration over all layers.  Work is ordered after what `stream` (default: the current
         stream) has queued so far, and `stream` waits for it at the end, so the caller can bracket steps with
-        events on that one stream."""
+        events on that one stream.  `after_layer(layer, slot_index, cuda_stream)`, if given, is called after
+        each layer's launch has been queued; what it queues on that stream runs between this visit of the slot
+        and the next one (used to copy a slot's state out between its visits)."""
         cur = stream if stream is not None else torch.cuda.current_stream(self.device)
         start = torch.cuda.Event()
         start.record(cur)
         for s in self.streams:
             s.wait_event(start)
         for layer in range(self.n_layers):
-            self.slots[layer % len(self.slots)].step(hyper, flags, self.streams[layer % len(self.streams)])
+            slot, side = layer % len(self.slots), self.streams[layer % len(self.streams)]
+            self.slots[slot].step(hyper, flags, side)
+            if after_layer is not None:
+                after_layer(layer, slot, side)
         for s, ev in zip(self.streams, self._done):
             ev.record(s)
             cur.wait_event(ev)

@@ -393,6 +393,39 @@ def test_reused_mask_is_decoded_and_flips_are_counted(bitmask):
     assert np.array_equal(bf16_bits_to_f32(reuse["w_fwd"]) != 0, np.tile(np.array([True, True, False, False]), 16)[None, :].repeat(4, 0))
 
 
+@pytest.mark.parametrize("bitmask", [True, False])
+def test_stored_mask_gates_the_decay_when_it_is_not_the_top_n(bitmask):
+    """Mask reuse (no reselection) with a stored mask that is NOT the magnitude top-2: every group of
+    (4, 3, 2, 1) * 0.01 stores the kept set {2, 3}, the two SMALLEST entries.  With alpha = 1, g = 0, m = 0,
+    v0 = lambda^2 the closed form of Eq. 7 says exactly which entries move: the ones outside the STORED set
+    (columns 0, 1) shrink by lr (lambda/bc1) / (lambda/sqrt(bc2) + eps) and feed lambda^2 into v; the stored
+    kept entries (columns 2, 3) do not move and their v only decays.  Had the decay been gated by a freshly
+    selected set (columns 0, 1 kept) the roles would be swapped."""
+    enc = orc.F_META_BITMASK if bitmask else 0
+    w0 = group_with_known_mask(1.0)
+    lam = float(np.float32(2e-3))
+    h = Hyper(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, l1_coeff=lam, step=20, total_steps=20)
+    lr, b1, b2, eps, _ = h.as_f32()
+    v0 = np.full_like(w0, np.float32(lam) ** 2)
+    field = 0b1100 if bitmask else (2 | 3 << 2)
+    stored = np.full((1, 1), sum(field << (4 * k) for k in range(8)), dtype=np.uint32)
+    out = run(w0, v=v0, N=2, M=4, hyper=h, flags=enc, meta_in=stored)
+    bc1, bc2 = 1 - b1 ** 20, 1 - b2 ** 20
+    v_decayed = b2 * float(v0[0, 0])
+    v_masked = v_decayed + (1 - b2) * lam * lam
+    step_size = lr * (lam / bc1) / (np.sqrt(v_masked / bc2) + eps)
+    outside = np.tile(np.array([True, True, False, False]), 8)[None, :]          # outside the stored set
+    np.testing.assert_allclose(out["w"], w0.astype(np.float64) - np.where(outside, step_size, 0.0), rtol=2e-7)
+    assert np.array_equal(out["w"][~outside], w0[~outside])
+    np.testing.assert_allclose(out["v"][outside], v_masked, rtol=2e-7)
+    np.testing.assert_allclose(out["v"][~outside], v_decayed, rtol=2e-7)
+    assert np.array_equal(out["meta"], stored)                                   # a reused mask is left as it is
+    assert np.array_equal(bf16_bits_to_f32(out["w_fwd"]) != 0, ~outside)         # and it prunes the emitted weight
+    # the freshly selected set on the same inputs moves the other half
+    fresh = run(w0, v=v0, N=2, M=4, hyper=h, flags=orc.F_RESELECT | enc)
+    assert np.array_equal(fresh["w"][outside], w0[outside]) and not np.any(fresh["w"][~outside] == w0[~outside])
+
+
 # --------------------------------------------------------------------------- numerics and long-run behaviour
 
 def test_fp32_order_stays_within_tolerance_of_fp64():
@@ -412,6 +445,43 @@ def test_fp32_order_stays_within_tolerance_of_fp64():
     da = bf16_bits_to_f32(a["w_fwd"]).astype(np.float64)
     db = bf16_bits_to_f32(b["w_fwd"])
     assert np.all(np.abs(da - db) <= np.abs(da) * 2.0 ** -7)
+
+
+def _refresh_schedule_worst_excess(lr):
+    """Steps t = 9, 10, 11 of a T = 12 run (mask refreshed and flips counted at t = 10, reused otherwise) on the
+    16 x 2048 seeded inputs of the GPU refresh-schedule test: worst |f32 - f64| / max(1e-6 |f64|, 1e-9) of w
+    over the three steps, each step of both builds starting from the fp64 build's previous state."""
+    from paper_2509_25996_b200 import workloads
+    from helpers import within_tol
+    rows, cols = 16, 2048
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=9, tensor_index=0, device="cpu", scale_mode="jitter")
+    w, m, v, sc = inp.w.numpy(), inp.m.numpy(), inp.v.numpy(), inp.scale.numpy()
+    meta = orc.adams_step(w, m, v, workloads.bf16_bits(inp.g), sc, 2, 4, Hyper(lr=0.0), orc.F_RESELECT)["meta"]
+    worst = 0.0
+    for t in (9, 10, 11):
+        flags = (orc.F_RESELECT | orc.F_COUNT_FLIPS) if t % 10 == 0 else 0
+        h = Hyper(lr=lr, l1_coeff=1e-3, step=t, total_steps=12)
+        gb = workloads.bf16_bits(workloads.gen_gradient(rows, cols, 9, 0, t))
+        a = orc.adams_step(w, m, v, gb, sc, 2, 4, h, flags, meta, "f64")
+        b = orc.adams_step(w, m, v, gb, sc, 2, 4, h, flags, meta, "f32")
+        assert np.array_equal(a["meta"], b["meta"])
+        for k in ("m", "v"):
+            assert within_tol(b[k], a[k])[0]
+        worst = max(worst, within_tol(b["w"], a["w"])[1])
+        w, m, v, meta = a["w"], a["m"], a["v"], a["meta"]
+    return worst
+
+
+def test_accuracy_domain_of_fp32_evaluation():
+    """The accepted error max(1e-6 |w|, 1e-9) has an absolute floor, so it bounds the per-step update for which
+    ANY fp32 evaluation of Alg. 1 can meet it: the update lr mu^/(sqrt(v^) + eps) carries a relative rounding
+    error of a few 2^-24, i.e. the floor is reached once the update is a few 1e-3.  With beta = 0.9 / 0.95 the
+    ratio mu^/sqrt(v^) is at most ~4.5, so lr = 5e-3 gives updates up to ~2e-2 and lr = 2e-4 up to ~1e-3.
+    The fp32 build of the oracle (plain IEEE operations in the written order) leaves the tolerance at the
+    first and stays well inside it at the second: the domain in which the tolerance is meaningful for an
+    fp32 implementation is per-step updates below ~1e-3, which every listed workload (lr = 1e-4) satisfies."""
+    assert _refresh_schedule_worst_excess(5e-3) > 1.5
+    assert _refresh_schedule_worst_excess(2e-4) < 0.5
 
 
 def test_masked_weights_shrink_as_alpha_ramps():
