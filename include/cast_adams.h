@@ -81,12 +81,37 @@ enum cast_flags {
                                        step applies the chain rule dL/dW = A (.) g itself and, where a scale_grad
                                        buffer is given, adds dL/dA[r, s] = sum_{c in segment s} g[r, c] W_{t-1}[r, c]
                                        to it                                                              */
-    CAST_F_EMIT_COMPRESSED = 1u << 5 /* emit only the kept entries of the pruned product (Alg. 2, final loop):
+    CAST_F_EMIT_COMPRESSED = 1u << 5, /* emit only the kept entries of the pruned product (Alg. 2, final loop):
                                        w_fwd_bf16 is then [rows][cols*N/M], the N kept values of each group in
                                        column order; with the metadata it is the whole pruned matrix, and a
                                        step writes 2 N/M instead of 2 bytes per parameter.  M <= 8 only; not
                                        together with CAST_F_EMIT_DENSE                                   */
+    CAST_F_MASK_STATS    = 1u << 7  /* the step also adds the mask statistics the paper monitors (App. C) to a
+                                       cast_mask_stats_t, from the registers it holds anyway: ||W_t (.) M_t||_1 and
+                                       ||W_t||_1 on the UPDATED weights with this step's kept set M_t, and
+                                       ||M_t - M_ref||_0 against the reference mask `meta_ref` of the matrix (the
+                                       initial mask for the initial flip rate i_t; 0 is added where meta_ref is
+                                       NULL).  Only cast_adams_step_stats / cast_plan_step_stats take this flag */
 };
+
+/*
+ * Accumulator of the mask statistics of App. C (cast_mask_stats, cast_plan_mask_stats and the steps that carry
+ * CAST_F_MASK_STATS add to it; the caller zeroes it):
+ *
+ *   mask_diff      += ||M - M_ref||_0   numerator of the flip rate r_t when M_ref is the previous mask, of the
+ *                                       initial flip rate i_t when it is the initial mask (0 without a reference)
+ *   kept_abs_sum   += ||W (.) M||_1     numerator of the sparse weight ratio S_t
+ *   total_abs_sum  += ||W||_1           its denominator
+ *
+ * The denominators of r_t and i_t are the parameter counts, which the caller knows.  Sums are formed in fp64
+ * (their last bits depend on the order in which CTAs add their parts).
+ */
+typedef struct cast_mask_stats {
+    unsigned long long mask_diff;
+    unsigned long long reserved_;     /* keeps the doubles 16-byte aligned; never written */
+    double kept_abs_sum;
+    double total_abs_sum;
+} cast_mask_stats_t;
 
 /*
  * cast_adams_step -- one AdamS iteration (Alg. 1 loop body, Eq. 6-8; Eq. 12 for the emitted weight)
@@ -141,6 +166,8 @@ typedef struct cast_tensor {
     int64_t rows, cols;
     float* scale_grad;       /* device, fp32 [rows][scale_groups], ADDED to by steps that carry
                                 CAST_F_GRAD_OF_SCALED (zero it before the step); may be NULL; needs `scale` */
+    const uint32_t* meta_ref;/* device, uint32 [rows*cols/32], same form as `meta`: the reference mask of
+                                CAST_F_MASK_STATS (never written); may be NULL                              */
 } cast_tensor_t;
 
 /* Hyper-parameters of one iteration (Alg. 1 inputs); ranges as in cast_adams_step. */
@@ -156,6 +183,17 @@ typedef struct cast_hyper {
  */
 CAST_API int cast_adams_step_ex(const cast_tensor_t* tensor, int N, int M, const cast_hyper_t* hyper,
                        unsigned long long* flip_count, cast_stream_t stream);
+
+/*
+ * cast_adams_step_stats -- cast_adams_step_ex that may carry CAST_F_MASK_STATS: the i_t and S_t sums of App. C come
+ * out of the step itself (the step holds |w_t|, the kept set and the stored metadata in registers), next to the
+ * flip count, instead of a second pass over the weights.
+ *   stats   device, 8-byte aligned, ADDED to (zero it before the first matrix of a model); required with the flag,
+ *           ignored without it.  Values: see cast_mask_stats_t; W is the weight after this update, M the kept set
+ *           of this step (selected now or reused), M_ref the matrix's `meta_ref`.
+ */
+CAST_API int cast_adams_step_stats(const cast_tensor_t* tensor, int N, int M, const cast_hyper_t* hyper,
+                          unsigned long long* flip_count, cast_mask_stats_t* stats, cast_stream_t stream);
 
 /*
  * cast_scale_adam_step -- the optimizer step of the scale matrix A of Eq. 12, which the paper learns jointly
@@ -206,6 +244,10 @@ CAST_API int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, in
                         void** plan_out);
 CAST_API int cast_plan_step(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
                    cast_stream_t stream);
+/* cast_plan_step that may carry CAST_F_MASK_STATS (see cast_adams_step_stats): the model-wide sums of App. C in the
+ * same launch as the step.  The reference masks are the `meta_ref` fields the plan was created with. */
+CAST_API int cast_plan_step_stats(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
+                         cast_mask_stats_t* stats, cast_stream_t stream);
 CAST_API int cast_plan_destroy(void* plan);
 
 /*
@@ -283,15 +325,8 @@ CAST_API int cast_prune_fold(const float* w, const float* scale, int scale_group
 CAST_API int cast_plan_prune_fold(void* plan, cast_bf16* const* out, uint32_t flags, cast_stream_t stream);
 
 /*
- * cast_mask_stats -- the mask statistics the paper monitors during training (App. C), for one matrix:
- *
- *   mask_diff      += ||M - M_ref||_0   numerator of the flip rate r_t when M_ref is the previous mask, of the
- *                                       initial flip rate i_t when it is the initial mask (0 when meta_ref is NULL)
- *   kept_abs_sum   += ||W (.) M||_1     numerator of the sparse weight ratio S_t
- *   total_abs_sum  += ||W||_1           its denominator
- *
- * The denominators of r_t and i_t are the parameter counts, which the caller knows.  Sums are formed in fp64
- * (their last bits depend on the order in which CTAs add their parts).
+ * cast_mask_stats -- the mask statistics the paper monitors during training (App. C), for one matrix, as a pass of
+ * its own over whatever (W, M, M_ref) the caller names (cast_mask_stats_t above says what is added).
  *
  *   w          device, fp32 [rows*cols]: the weights W.
  *   meta       device, uint32 [rows*cols/32]: the mask M in the metadata layout described at the top.
@@ -301,12 +336,6 @@ CAST_API int cast_plan_prune_fold(void* plan, cast_bf16* const* out, uint32_t fl
  *              call once per matrix to get the model-wide sums of App. C).
  * Asynchronous on `stream`.  Errors as cast_adams_step; nothing is launched on an error.
  */
-typedef struct cast_mask_stats {
-    unsigned long long mask_diff;
-    unsigned long long reserved_;     /* keeps the doubles 16-byte aligned; never written */
-    double kept_abs_sum;
-    double total_abs_sum;
-} cast_mask_stats_t;
 CAST_API int cast_mask_stats(const float* w, const uint32_t* meta, const uint32_t* meta_ref,
                     int64_t rows, int64_t cols, int M, uint32_t flags,
                     cast_mask_stats_t* stats, cast_stream_t stream);

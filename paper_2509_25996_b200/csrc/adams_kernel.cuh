@@ -14,9 +14,11 @@
 //
 // Instruction budget: at ~6.8 TB/s an SM retires ~0.85 parameters per clock, so the body has to stay
 // well under ~100 thread instructions per parameter or instruction issue (and, under the board's
-// power cap, the SM clock) becomes the limit.  Hence: flags are compile-time constants in the
-// common modes, the 2:4 selection is six comparisons and four 3-input predicate functions per group,
-// and the update uses the approximate reciprocal and square root units (error analysis below).
+// power cap, the SM clock) becomes the limit.  Hence: the flag word is a compile-time constant of the
+// kernel (one instantiation per valid combination of selection, metadata form, emission, flip counting,
+// scale gradient and statistics), the 2:4 selection is six comparisons and four 3-input predicate
+// functions per group, and the update uses the approximate reciprocal and square root units (error
+// analysis below).
 #pragma once
 
 #include <cuda_runtime.h>
@@ -27,7 +29,7 @@ namespace cast {
 constexpr int kThreads = 128;          // threads per CTA
 constexpr int kUnitElems = 8;          // parameters per thread
 constexpr int kTileUnits = kThreads;   // units per tile (1024 parameters)
-constexpr int kMinCtasPerSm = 7;       // register budget the kernels are compiled for (M <= 8)
+constexpr int kMinCtasPerSm = 7;       // register budget the kernels are compiled for
 
 // flag bits (values of the public header)
 constexpr uint32_t kReselect = 1u << 0;
@@ -37,32 +39,27 @@ constexpr uint32_t kVKeptFromG = 1u << 3;
 constexpr uint32_t kEmitDense = 1u << 4;
 constexpr uint32_t kEmitCompressed = 1u << 5;
 constexpr uint32_t kGradOfScaled = 1u << 6;
+constexpr uint32_t kMaskStats = 1u << 7;
 
-// Kernel modes: the flag word is a compile-time constant in the common cases.
-constexpr int kModeGeneric = 0;        // any flags, read from StepConsts at run time
-constexpr int kModeSelectIdx = 1;      // flags == kReselect, 2:4, index-form metadata
-constexpr int kModeSelectMask = 2;     // flags == kReselect | kMetaBitmask, any N:M
-constexpr int kModeSelectIdxPacked = 3;   // flags == kReselect | kEmitCompressed, 2:4, index-form metadata
-constexpr int kModeReuseIdx = 4;       // flags == 0: the stored 2:4 mask is reused (between the paper's refreshes)
-constexpr int kModeReuseIdxDense = 5;  // flags == kEmitDense: stored 2:4 mask, dense forward weight (Alg. 2's training step)
-constexpr int kModeSelectIdxFlips = 6;       // flags == kReselect | kCountFlips, 2:4, index-form metadata
-constexpr int kModeSelectMaskFlips = 7;      // flags == kReselect | kMetaBitmask | kCountFlips, any N:M
-constexpr int kModeSelectIdxFlipsDense = 8;  // flags == kReselect | kCountFlips | kEmitDense, 2:4: the refresh step of training
-constexpr int kModeReuseIdxDenseScaled = 9;        // flags == kEmitDense | kGradOfScaled: mode 5 with the gradient taken
-                                                   // through the scaling (the common step of training with a learned scale)
-constexpr int kModeSelectIdxFlipsDenseScaled = 10; // flags == mode 8 | kGradOfScaled: its refresh step
-constexpr int kModeCount = 11;
+// Every flag but kVKeptFromG is a template argument of the kernels; that one (the alternate reading of Eq. 8,
+// one select per parameter) is read from StepConsts at run time.
+constexpr uint32_t kCompileTimeFlags = kReselect | kCountFlips | kMetaBitmask | kEmitDense | kEmitCompressed |
+                                       kGradOfScaled | kMaskStats;
+constexpr uint32_t kFlagWords = 256;   // compile-time flag words live in [0, kFlagWords)
 
-// Modes whose kept set comes from the 2:4 comparison network (N = 2, M = 4, index-form metadata).
-__host__ __device__ constexpr bool mode_selects_2of4(int mode)
+// Which (M, two_four, flag word) combinations are instantiated.  `two_four` says N == 2 and M == 4: the kept set
+// comes from the comparison network, the metadata may be in index form and the compressed form is two byte
+// permutes.  The host normalises a flag word before it looks for its kernel: kCountFlips is dropped without
+// kReselect (a reused mask has no flips).
+__host__ __device__ constexpr bool step_kernel_exists(int M, bool two_four, uint32_t f)
 {
-    return mode == kModeSelectIdx || mode == kModeSelectIdxPacked || mode == kModeSelectIdxFlips || mode == kModeSelectIdxFlipsDense ||
-           mode == kModeSelectIdxFlipsDenseScaled;
-}
-// Modes that exist for M = 4 only.
-__host__ __device__ constexpr bool mode_is_2of4_only(int mode)
-{
-    return mode_selects_2of4(mode) || mode == kModeReuseIdx || mode == kModeReuseIdxDense || mode == kModeReuseIdxDenseScaled;
+    if (f & ~kCompileTimeFlags) return false;
+    if ((f & kCountFlips) && !(f & kReselect)) return false;
+    if ((f & kEmitDense) && (f & kEmitCompressed)) return false;
+    if ((f & kEmitCompressed) && M > kUnitElems) return false;
+    if (two_four && M != 4) return false;
+    if (!two_four && !(f & kMetaBitmask)) return false;      // index-form metadata is 2:4 only
+    return true;
 }
 
 // One matrix as the kernel sees it.
@@ -75,6 +72,7 @@ struct TensorDesc {
     uint32_t* meta;
     const float* scale;        // A[rows][n] or nullptr
     float* scale_grad;         // dL/dA[rows][n], added to, or nullptr
+    const uint8_t* meta_ref;   // reference mask of the statistics (same form as meta), or nullptr
     uint32_t n_units;          // rows * cols / 8
     uint32_t seg_magic;        // unit / seg_units == (uint64(unit) * seg_magic) >> seg_shift
     uint32_t seg_shift;
@@ -132,42 +130,24 @@ __device__ __forceinline__ void select_2of4(const uint32_t* a, bool* kept)
     kept[3] = at_least_two(!c03, !c13, !c23);
 }
 
-// General N:M: rank of a column = how many columns of its group come before it; kept iff rank < N.
-// Returns the keep mask of the unit (bit j = column j of the unit is kept).
+// General N:M, M <= 8 (the group lives in this thread): rank of a column = how many columns of its group come
+// before it; kept iff rank < N.  Returns the keep mask of the unit (bit j = column j of the unit is kept).
 template <int M>
 __device__ __forceinline__ uint32_t select_by_rank(const uint32_t (&a)[8], int n_keep)
 {
-    constexpr int G = (M <= 8) ? M : 8;      // columns of one group held by this thread
+    static_assert(M <= 8, "wider groups are shared by lanes: select_wide");
     int rank[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) rank[i] = 0;
 #pragma unroll
-    for (int base = 0; base < 8; base += G) {
+    for (int base = 0; base < 8; base += M) {
 #pragma unroll
-        for (int j = 0; j < G; ++j) {
+        for (int j = 0; j < M; ++j) {
 #pragma unroll
-            for (int k = j + 1; k < G; ++k) {
+            for (int k = j + 1; k < M; ++k) {
                 const bool j_first = a[base + j] >= a[base + k];
                 rank[base + k] += j_first ? 1 : 0;
                 rank[base + j] += j_first ? 0 : 1;
-            }
-        }
-    }
-    // columns of the same group held by neighbouring lanes (M = 16: 2 lanes, M = 32: 4 lanes)
-    if constexpr (M > 8) {
-        constexpr int L = M / 8;
-        const unsigned lane = threadIdx.x & 31u;
-#pragma unroll
-        for (int d = 1; d < L; ++d) {
-            const bool other_lower = ((lane ^ d) < lane);
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                const uint32_t ak = __shfl_xor_sync(0xFFFFFFFFu, a[k], d);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    const bool k_first = other_lower ? (ak >= a[j]) : (ak > a[j]);
-                    rank[j] += k_first ? 1 : 0;
-                }
             }
         }
     }
@@ -175,6 +155,107 @@ __device__ __forceinline__ uint32_t select_by_rank(const uint32_t (&a)[8], int n
 #pragma unroll
     for (int i = 0; i < 8; ++i) keep |= (rank[i] < n_keep ? 1u : 0u) << i;
     return keep;
+}
+
+// Groups of 16 or 32 columns are shared by L = 2 or 4 neighbouring lanes (8 columns each, lower lane = lower
+// columns).  The kept set is {|w| > tau} plus, among the columns with |w| == tau in column order, as many as
+// are still missing to N, where tau is the N-th largest magnitude of the group -- the same set as "rank < N"
+// under the order of Eq. 6 used everywhere else.  tau comes from a bitonic sort of the group's 31-bit keys
+// (minimum / maximum instructions only, no indices carried): each lane sorts its 8 keys with a 19-exchange
+// network, pairs of lanes merge (exchange against the partner's reversed run, then a local 12-exchange bitonic
+// merge), and for L = 4 the two sorted 16-runs merge the same way across lanes.  All lanes of the warp call this.
+__device__ __forceinline__ void exchange_desc(uint32_t& first, uint32_t& second)
+{
+    const uint32_t hi = max(first, second), lo = min(first, second);
+    first = hi;
+    second = lo;
+}
+__device__ __forceinline__ void sort8_desc(uint32_t (&s)[8])
+{
+    exchange_desc(s[0], s[1]); exchange_desc(s[2], s[3]); exchange_desc(s[4], s[5]); exchange_desc(s[6], s[7]);
+    exchange_desc(s[0], s[2]); exchange_desc(s[1], s[3]); exchange_desc(s[4], s[6]); exchange_desc(s[5], s[7]);
+    exchange_desc(s[1], s[2]); exchange_desc(s[5], s[6]); exchange_desc(s[0], s[4]); exchange_desc(s[3], s[7]);
+    exchange_desc(s[1], s[5]); exchange_desc(s[2], s[6]);
+    exchange_desc(s[1], s[4]); exchange_desc(s[3], s[6]);
+    exchange_desc(s[2], s[4]); exchange_desc(s[3], s[5]);
+    exchange_desc(s[3], s[4]);
+}
+__device__ __forceinline__ void bitonic_merge8_desc(uint32_t (&s)[8])
+{
+#pragma unroll
+    for (int d = 4; d > 0; d >>= 1)
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (!(i & d)) exchange_desc(s[i], s[i + d]);
+}
+// One cross-lane step of a bitonic merge: every key meets the key `REVERSED ? 7 - i : i` of lane ^ d; the lane
+// on the `upper` side keeps the smaller one, the other the larger one.
+template <bool REVERSED>
+__device__ __forceinline__ void exchange_lanes_desc(uint32_t (&s)[8], int d, bool upper)
+{
+    uint32_t r[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r[i] = __shfl_xor_sync(0xFFFFFFFFu, s[REVERSED ? 7 - i : i], d);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = upper ? min(s[i], r[i]) : max(s[i], r[i]);
+}
+
+template <int M>
+__device__ __forceinline__ uint32_t select_wide(const uint32_t (&a)[8], int n_keep)
+{
+    static_assert(M == 16 || M == 32, "groups of 16 or 32 columns");
+    constexpr unsigned L = M / 8;
+    const unsigned lane = threadIdx.x & 31u;
+    const unsigned pos = lane & (L - 1u);                  // this lane's place in its group
+    uint32_t s[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] = a[i];
+    sort8_desc(s);
+    exchange_lanes_desc<true>(s, 1, (pos & 1u) != 0);      // two sorted 8-runs -> upper / lower half of 16
+    bitonic_merge8_desc(s);
+    if constexpr (L == 4) {
+        exchange_lanes_desc<true>(s, 3, (pos & 2u) != 0);  // two sorted 16-runs -> upper / lower half of 32
+        exchange_lanes_desc<false>(s, 1, (pos & 1u) != 0);
+        bitonic_merge8_desc(s);
+    }
+    // the group's keys now stand in descending order across its lanes: place q is s[q & 7] of lane q >> 3
+    const int q = n_keep - 1;                              // uniform
+    uint32_t cand = s[0];
+#pragma unroll
+    for (int i = 1; i < 8; ++i) cand = ((q & 7) == i) ? s[i] : cand;
+    const uint32_t tau = __shfl_sync(0xFFFFFFFFu, cand, (int)(lane & ~(L - 1u)) + (q >> 3));
+    uint32_t gt = 0, eq = 0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        gt |= (a[i] > tau ? 1u : 0u) << i;
+        eq |= (a[i] == tau ? 1u : 0u) << i;
+    }
+    // columns above tau in the whole group, columns equal to tau in the lower lanes of the group
+    int above = __popc(gt);
+    const int equal_here = __popc(eq);
+    int equal_incl = equal_here;
+#pragma unroll
+    for (unsigned d = 1; d < L; d <<= 1) {
+        above += __shfl_xor_sync(0xFFFFFFFFu, above, (int)d);
+        const int up = __shfl_up_sync(0xFFFFFFFFu, equal_incl, d);
+        if (pos >= d) equal_incl += up;
+    }
+    int missing = n_keep - above - (equal_incl - equal_here);      // ties this lane may still keep, in column order
+    uint32_t keep = gt;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const bool e = (eq >> i) & 1u;
+        keep |= ((e && missing > 0) ? 1u : 0u) << i;
+        missing -= e ? 1 : 0;
+    }
+    return keep;
+}
+
+template <int M>
+__device__ __forceinline__ uint32_t select_top_n(const uint32_t (&a)[8], int n_keep)
+{
+    if constexpr (M <= 8) return select_by_rank<M>(a, n_keep);
+    else return select_wide<M>(a, n_keep);
 }
 
 // 2:4 index form: one nibble per group, lo | hi << 2 with lo < hi the positions of the kept pair.
@@ -221,11 +302,6 @@ __device__ __forceinline__ uint32_t kept_pair_2of4(uint32_t r01, uint32_t r23, u
 template <int M>
 __device__ __forceinline__ void store_kept_values(uint16_t* base, uint32_t unit, uint32_t keep, uint4 packed, int n_keep)
 {
-    if (M == 4 && n_keep == 2) {              // uniform: 4 values per unit, no shared memory needed
-        *reinterpret_cast<uint2*>(base + (size_t)unit * 4) =
-            make_uint2(kept_pair_2of4(packed.x, packed.y, keep & 0xFu), kept_pair_2of4(packed.z, packed.w, keep >> 4));
-        return;
-    }
     __shared__ __align__(16) uint16_t s_comp[kThreads * 8];
     uint16_t* mine = s_comp + threadIdx.x * 8;
     const uint32_t hw[4] = {packed.x, packed.y, packed.z, packed.w};
@@ -247,29 +323,44 @@ struct UnitRegs {
     float w[8], m[8], v[8];
     uint4 g;               // 8 bf16 gradients in; 8 bf16 forward weights out
     uint32_t prev_byte;    // metadata byte of the unit before the step (when it is read)
+    uint32_t ref_byte;     // byte of the statistics' reference mask (when there is one)
     uint32_t meta_byte;    // metadata byte after the step
-    uint32_t keep;         // keep mask of the unit (bit j = column j kept); not set by the 2:4 comparison-network modes
+    uint32_t keep;         // keep mask of the unit (bit j = column j kept), where the configuration needs it as bits
 };
 
-template <int MODE>
-__device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
-{
-    if constexpr (MODE == kModeSelectIdx) return kReselect;
-    else if constexpr (MODE == kModeSelectIdxPacked) return kReselect | kEmitCompressed;
-    else if constexpr (MODE == kModeSelectMask) return kReselect | kMetaBitmask;
-    else if constexpr (MODE == kModeReuseIdx) return 0u;
-    else if constexpr (MODE == kModeReuseIdxDense) return kEmitDense;
-    else if constexpr (MODE == kModeSelectIdxFlips) return kReselect | kCountFlips;
-    else if constexpr (MODE == kModeSelectMaskFlips) return kReselect | kMetaBitmask | kCountFlips;
-    else if constexpr (MODE == kModeSelectIdxFlipsDense) return kReselect | kCountFlips | kEmitDense;
-    else if constexpr (MODE == kModeReuseIdxDenseScaled) return kEmitDense | kGradOfScaled;
-    else if constexpr (MODE == kModeSelectIdxFlipsDenseScaled) return kReselect | kCountFlips | kEmitDense | kGradOfScaled;
-    else return c.flags;
-}
+// What one CTA adds to the caller's counters: flips (App. C, numerator of r_t) and the mask statistics
+// (App. C: ||M_t - M_ref||_0, ||W_t (.) M_t||_1, ||W_t||_1 on the updated weights).
+struct UnitSums {
+    uint32_t flips = 0;
+    uint32_t mask_diff = 0;
+    double kept_abs = 0.0, total_abs = 0.0;
+};
+
+// Device view of the statistics accumulator (layout of cast_mask_stats_t in the public header).
+struct MaskStats {
+    unsigned long long mask_diff;
+    unsigned long long reserved_;
+    double kept_abs_sum;
+    double total_abs_sum;
+};
+
+// Compile-time view of a flag word.
+template <int M, uint32_t F, bool TF>
+struct StepCfg {
+    static_assert(step_kernel_exists(M, TF, F), "no such kernel");
+    static constexpr bool reselect = (F & kReselect) != 0;
+    static constexpr bool count_flips = (F & kCountFlips) != 0;
+    static constexpr bool bitmask = (F & kMetaBitmask) != 0;
+    static constexpr bool dense = (F & kEmitDense) != 0;
+    static constexpr bool compressed = (F & kEmitCompressed) != 0;
+    static constexpr bool of_scaled = (F & kGradOfScaled) != 0;
+    static constexpr bool stats = (F & kMaskStats) != 0;
+    static constexpr bool network = TF && reselect;               // kept set from the 2:4 comparison network
+    static constexpr bool need_prev = !reselect || count_flips;   // the stored metadata is read
+};
 
 // Arithmetic of one unit, registers only (and warp shuffles for M > 8: every lane of the warp must
-// call this, lanes without data pass zeros).  `a` is the unit's scale A[r, segment].  Returns the
-// number of flipped mask bits of the unit (App. C: ||M_t - M_{t-1}||_0; 0 unless flips are counted).
+// call this, lanes without data pass zeros).  `a` is the unit's scale A[r, segment].
 //
 // Precision.  The first moment and the decayed first moment are sums of terms of opposite sign and
 // like size (beta1 m against (1 - beta1) g, (1 - alpha) mu against alpha lambda), so they are formed
@@ -279,71 +370,63 @@ __device__ __forceinline__ uint32_t mode_flags(const StepConsts& c)
 // approximate square root and reciprocal: its relative error is below ~5e-7 (2^-23 each, plus five
 // roundings of 2^-24), i.e. below 2.5e-10 absolute for updates up to 5e-4, which is under both the
 // fp32 spacing of typical weights (1.9e-9 at 0.02) and the 1e-9 floor of the accepted error.
-template <int M, int MODE>
-__device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& c, float a, float& gw_sum)
+template <int M, uint32_t F, bool TF>
+__device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, float a, bool has_ref, float& gw_sum, UnitSums& sums)
 {
-    static_assert(!mode_is_2of4_only(MODE) || M == 4, "index-form metadata is 2:4 only");
-    const uint32_t flags = mode_flags<MODE>(c);
-    const bool bitmask = (flags & kMetaBitmask) != 0;
+    using Cfg = StepCfg<M, F, TF>;
     uint32_t ab[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) ab[i] = abs_bits(u.w[i]);
 
     bool kept[8];
-    uint32_t flips = 0;
-    if constexpr (mode_selects_2of4(MODE)) {
+    uint32_t keep = 0;                  // as bits, where some consumer below wants bits
+    if constexpr (Cfg::network) {
         select_2of4(ab, kept);
         select_2of4(ab + 4, kept + 4);
-        u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
-        if (flags & kCountFlips)                        // both masks as index bytes: decode and compare
-            flips = (uint32_t)__popc(keep_from_meta_byte(u.meta_byte, false) ^ keep_from_meta_byte(u.prev_byte, false));
-    } else {
-        // `flags` is a compile-time constant in every mode but the generic one: the branches below fold away
-        const bool need_prev = !(flags & kReselect) || (flags & kCountFlips);
-        const uint32_t prev_keep = need_prev ? keep_from_meta_byte(u.prev_byte, bitmask) : 0u;
-        uint32_t keep;
-        if ((flags & kReselect) && M == 4 && c.n_keep == 2) {       // uniform: 2:4 by the comparison network
-            select_2of4(ab, kept);
-            select_2of4(ab + 4, kept + 4);
-            keep = 0;
+        constexpr bool want_bits = Cfg::bitmask || Cfg::stats;
+        if constexpr (want_bits) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) keep |= (kept[i] ? 1u : 0u) << i;
-            if (bitmask) u.meta_byte = keep;
-            else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
-        } else if (flags & kReselect) {
-            keep = select_by_rank<M>(ab, c.n_keep);     // uniform branch: all lanes shuffle
-#pragma unroll
-            for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
-            if (bitmask) u.meta_byte = keep;
-            else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+        }
+        if constexpr (Cfg::bitmask) u.meta_byte = keep;
+        else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
+        if constexpr (Cfg::count_flips) {
+            if constexpr (Cfg::bitmask) sums.flips = (uint32_t)__popc(keep ^ u.prev_byte);
+            else sums.flips = (uint32_t)__popc(keep_from_meta_byte(u.meta_byte, false) ^ keep_from_meta_byte(u.prev_byte, false));
+        }
+    } else {
+        if constexpr (Cfg::reselect) {
+            keep = select_top_n<M>(ab, c.n_keep);              // all lanes shuffle for M > 8
+            u.meta_byte = keep;                                 // only 2:4 has an index form
+            if constexpr (Cfg::count_flips) sums.flips = (uint32_t)__popc(keep ^ u.prev_byte);
         } else {
-            keep = prev_keep;                           // the stored mask, as it is
-#pragma unroll
-            for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+            keep = keep_from_meta_byte(u.prev_byte, Cfg::bitmask);   // the stored mask, as it is
             u.meta_byte = u.prev_byte;
         }
-        u.keep = keep;
-        if (flags & kCountFlips) flips = (uint32_t)__popc(keep ^ prev_keep);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
+    }
+    u.keep = keep;
+    if constexpr (Cfg::stats) {
+        if (has_ref) sums.mask_diff = (uint32_t)__popc(keep ^ keep_from_meta_byte(u.ref_byte, Cfg::bitmask));
     }
 
     const uint32_t gw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
-    const bool v_from_g = (flags & kVKeptFromG) != 0;
-    const bool dense = (flags & kEmitDense) != 0;
+    const bool v_from_g = (c.flags & kVKeptFromG) != 0;
     const int sign_hi = __double2hiint(c.c_sign), sign_lo = __double2loint(c.c_sign);
     // With kGradOfScaled the gradient is taken with respect to W_scale = Diag(A) W (Eq. 12): the chain rule
     // gives dL/dW = A g (formed exactly in fp64) and dL/dA = sum of g W over the row segment, whose part
     // for this unit is returned in gw_sum (fp32 chain of 8 fused multiply-adds on the weights before the update).
-    const bool of_scaled = (flags & kGradOfScaled) != 0;
-    const double omb1_g = of_scaled ? c.omb1 * (double)a : c.omb1;
+    const double omb1_g = Cfg::of_scaled ? c.omb1 * (double)a : c.omb1;
     gw_sum = 0.0f;
     float fwd[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         float g32 = __uint_as_float((i & 1) ? (gw[i >> 1] & 0xFFFF0000u) : (gw[i >> 1] << 16));
-        if (of_scaled) gw_sum = fmaf(g32, u.w[i], gw_sum);
+        if constexpr (Cfg::of_scaled) gw_sum = fmaf(g32, u.w[i], gw_sum);
         // first moment, stored undecayed (Alg. 1)
         const double mu = fma(c.beta1, (double)u.m[i], omb1_g * (double)g32);
-        if (of_scaled) g32 *= a;                 // only the alternate reading of v below still uses g itself
+        if constexpr (Cfg::of_scaled) g32 *= a;      // only the alternate reading of v below still uses g itself
         const float mu_f = (float)mu;
         u.m[i] = mu_f;
         // proportional L1 decay outside the kept set (Eq. 7): alpha lambda Sign(w), Sign(+-0) = 0
@@ -358,37 +441,42 @@ __device__ __forceinline__ uint32_t compute_unit(UnitRegs& u, const StepConsts& 
         // bias-corrected update (Alg. 1): w - (lr / bc1) mu~ / (sqrt(v / bc2) + eps)
         const float wn = u.w[i] - update_term(mu_t, vn, c);
         u.w[i] = wn;
+        if constexpr (Cfg::stats) {                  // |w_t| converts exactly; fp64 sums
+            const double mag = (double)fabsf(wn);
+            sums.total_abs += mag;
+            if (kept[i]) sums.kept_abs += mag;
+        }
         // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for
-        fwd[i] = (kept[i] || dense) ? a * wn : 0.0f;
+        fwd[i] = (kept[i] || Cfg::dense) ? a * wn : 0.0f;
     }
     u.g.x = pack_bf16x2(fwd[0], fwd[1]);
     u.g.y = pack_bf16x2(fwd[2], fwd[3]);
     u.g.z = pack_bf16x2(fwd[4], fwd[5]);
     u.g.w = pack_bf16x2(fwd[6], fwd[7]);
-    return flips;
 }
 
 // The whole per-unit body: loads, arithmetic, stores.
 // `active` is false for threads past the end of the matrix; they take part in the shuffles only.
-template <int M, int MODE>
-__device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const StepConsts& c,
-                                                 uint32_t unit, bool active)
+template <int M, uint32_t F, bool TF>
+__device__ __forceinline__ void process_unit(const TensorDesc& t, const StepConsts& c, uint32_t unit, bool active, UnitSums& sums)
 {
+    using Cfg = StepCfg<M, F, TF>;
     UnitRegs u;
     u.g = make_uint4(0, 0, 0, 0);
     u.prev_byte = 0;
+    u.ref_byte = 0;
     const size_t e = (size_t)unit * kUnitElems;
-    const uint32_t flags = mode_flags<MODE>(c);
-    const bool need_prev = ((flags & kReselect) == 0) || (flags & kCountFlips);
     float a = 1.0f;
     uint32_t seg = 0;
+    const bool has_ref = Cfg::stats && t.meta_ref != nullptr;      // uniform over the CTA
 
     if (active) {
         const float4 w0 = ld_f4(t.w + e), w1 = ld_f4(t.w + e + 4);
         const float4 m0 = ld_f4(t.m + e), m1 = ld_f4(t.m + e + 4);
         const float4 v0 = ld_f4(t.v + e), v1 = ld_f4(t.v + e + 4);
         u.g = *reinterpret_cast<const uint4*>(t.g + e);
-        if (need_prev) u.prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[unit];
+        if constexpr (Cfg::need_prev) u.prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[unit];
+        if (has_ref) u.ref_byte = t.meta_ref[unit];
         if (t.scale != nullptr) {
             seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
             a = __ldg(t.scale + seg);
@@ -402,9 +490,10 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
     }
 
     float gw_sum;
-    const uint32_t flips = compute_unit<M, MODE>(u, c, a, gw_sum);
-    {
-        if ((flags & kGradOfScaled) && t.scale_grad != nullptr) {     // uniform over the CTA: all lanes shuffle
+    UnitSums mine;
+    compute_unit<M, F, TF>(u, c, a, has_ref, gw_sum, mine);
+    if constexpr (Cfg::of_scaled) {
+        if (t.scale_grad != nullptr) {                              // uniform over the CTA: all lanes shuffle
             // Sum gw_sum over the lanes of the warp that share a row segment (segments are runs of consecutive
             // lanes), then one atomic per run.  Lanes without data carry a segment of their own and add nothing.
             const unsigned lane = threadIdx.x & 31u;
@@ -428,22 +517,23 @@ __device__ __forceinline__ uint32_t process_unit(const TensorDesc& t, const Step
         st_f4(t.m + e + 4, make_float4(u.m[4], u.m[5], u.m[6], u.m[7]));
         st_f4(t.v + e, make_float4(u.v[0], u.v[1], u.v[2], u.v[3]));
         st_f4(t.v + e + 4, make_float4(u.v[4], u.v[5], u.v[6], u.v[7]));
-        bool compressed = false;
-        if constexpr (M <= 8) compressed = (flags & kEmitCompressed) != 0;
-        if constexpr (MODE == kModeSelectIdxPacked) {
+        if constexpr (!Cfg::compressed) {
+            *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
+        } else if constexpr (TF && !Cfg::bitmask) {
             // the index-form metadata byte holds the kept positions of both groups: lo | hi << 2 per nibble
             const uint32_t mb = u.meta_byte;
             *reinterpret_cast<uint2*>(t.w_fwd + (size_t)unit * 4) =
                 make_uint2(kept_pair_by_index(u.g.x, u.g.y, mb & 3u, (mb >> 2) & 3u),
                            kept_pair_by_index(u.g.z, u.g.w, (mb >> 4) & 3u, mb >> 6));
-        } else if (!compressed) {
-            *reinterpret_cast<uint4*>(t.w_fwd + e) = u.g;
+        } else if constexpr (TF) {
+            *reinterpret_cast<uint2*>(t.w_fwd + (size_t)unit * 4) =
+                make_uint2(kept_pair_2of4(u.g.x, u.g.y, u.meta_byte & 0xFu), kept_pair_2of4(u.g.z, u.g.w, u.meta_byte >> 4));
         } else {
             store_kept_values<M>(t.w_fwd, unit, u.keep, u.g, c.n_keep);
         }
-        if (flags & kReselect) reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;   // else unchanged
+        if constexpr (Cfg::reselect) reinterpret_cast<uint8_t*>(t.meta)[unit] = (uint8_t)u.meta_byte;   // else unchanged
+        sums = mine;
     }
-    return active ? flips : 0u;
 }
 
 // Tables of one multi-tensor launch, passed by value in kernel parameter space (constant bank): a CTA
@@ -462,49 +552,78 @@ struct MultiParams {
     uint32_t tile_start[kMaxLaunchTensors + 1];
     TensorDesc desc[kMaxLaunchTensors];
 };
-static_assert(sizeof(MultiParams) + sizeof(StepConsts) + 16 <= 32764, "kernel parameters are limited to 32764 bytes");
+static_assert(sizeof(MultiParams) + sizeof(StepConsts) + 32 <= 32764, "kernel parameters are limited to 32764 bytes");
 
-// Flips of the CTA added to the caller's counter (one atomic per CTA that saw any).
-__device__ __forceinline__ void add_flips(uint32_t flips, unsigned long long* flip_count)
+// What the CTA counted, added to the caller's counters: one atomic per counter per CTA.
+template <bool FLIPS, bool STATS>
+__device__ __forceinline__ void add_sums(UnitSums x, unsigned long long* flip_count, MaskStats* stats)
 {
-    flips = __reduce_add_sync(0xFFFFFFFFu, flips);
-    __shared__ uint32_t warp_sums[kThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_sums[threadIdx.x >> 5] = flips;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned long long total = 0;
+    if constexpr (FLIPS || STATS) {
+        __shared__ uint32_t s_flips[kThreads / 32], s_diff[kThreads / 32];
+        __shared__ double s_kept[kThreads / 32], s_total[kThreads / 32];
+        const int warp = threadIdx.x >> 5;
+        const bool lead = (threadIdx.x & 31) == 0;
+        if constexpr (FLIPS) {
+            const uint32_t f = __reduce_add_sync(0xFFFFFFFFu, x.flips);
+            if (lead) s_flips[warp] = f;
+        }
+        if constexpr (STATS) {
+            const uint32_t d = __reduce_add_sync(0xFFFFFFFFu, x.mask_diff);
+            double k = x.kept_abs, t = x.total_abs;
 #pragma unroll
-        for (int i = 0; i < kThreads / 32; ++i) total += warp_sums[i];
-        if (total) atomicAdd(flip_count, total);
+            for (int o = 16; o > 0; o >>= 1) {
+                k += __shfl_down_sync(0xFFFFFFFFu, k, o);
+                t += __shfl_down_sync(0xFFFFFFFFu, t, o);
+            }
+            if (lead) { s_diff[warp] = d; s_kept[warp] = k; s_total[warp] = t; }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            if constexpr (FLIPS) {
+                unsigned long long total = 0;
+#pragma unroll
+                for (int i = 0; i < kThreads / 32; ++i) total += s_flips[i];
+                if (total) atomicAdd(flip_count, total);
+            }
+            if constexpr (STATS) {
+                unsigned long long d = 0;
+                double k = 0.0, t = 0.0;
+#pragma unroll
+                for (int i = 0; i < kThreads / 32; ++i) { d += s_diff[i]; k += s_kept[i]; t += s_total[i]; }
+                if (d) atomicAdd(&stats->mask_diff, d);
+                atomicAdd(&stats->kept_abs_sum, k);
+                atomicAdd(&stats->total_abs_sum, t);
+            }
+        }
     }
 }
 
-#define CAST_LAUNCH_BOUNDS(M) __launch_bounds__(kThreads, ((M) <= 8) ? kMinCtasPerSm : 4)
-
 // One matrix: CTA b handles tile b.
-template <int M, int MODE>
-__global__ void CAST_LAUNCH_BOUNDS(M)
+template <int M, uint32_t F, bool TF>
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 adams_nm_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c,
-                unsigned long long* __restrict__ flip_count)
+                unsigned long long* __restrict__ flip_count, MaskStats* __restrict__ stats)
 {
     const uint32_t unit = blockIdx.x * kTileUnits + threadIdx.x;
-    const uint32_t flips = process_unit<M, MODE>(t, c, unit, unit < t.n_units);
-    if (mode_flags<MODE>(c) & kCountFlips) add_flips(flips, flip_count);
+    UnitSums sums;
+    process_unit<M, F, TF>(t, c, unit, unit < t.n_units, sums);
+    add_sums<StepCfg<M, F, TF>::count_flips, StepCfg<M, F, TF>::stats>(sums, flip_count, stats);
 }
 
 // Up to kMaxLaunchTensors matrices in one grid: CTA b handles tile b of the concatenated index space.
-template <int M, int MODE>
-__global__ void CAST_LAUNCH_BOUNDS(M)
+template <int M, uint32_t F, bool TF>
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 adams_nm_multi_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
-                      unsigned long long* __restrict__ flip_count)
+                      unsigned long long* __restrict__ flip_count, MaskStats* __restrict__ stats)
 {
     const uint32_t tile = blockIdx.x;
     uint32_t k = p.hint[tile >> p.hint_shift];
     while (tile >= p.tile_start[k + 1]) ++k;
     const TensorDesc& t = p.desc[k];
     const uint32_t unit = (tile - p.tile_start[k]) * kTileUnits + threadIdx.x;
-    const uint32_t flips = process_unit<M, MODE>(t, c, unit, unit < t.n_units);
-    if (mode_flags<MODE>(c) & kCountFlips) add_flips(flips, flip_count);
+    UnitSums sums;
+    process_unit<M, F, TF>(t, c, unit, unit < t.n_units, sums);
+    add_sums<StepCfg<M, F, TF>::count_flips, StepCfg<M, F, TF>::stats>(sums, flip_count, stats);
 }
 
 }  // namespace cast

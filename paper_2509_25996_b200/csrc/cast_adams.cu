@@ -29,7 +29,7 @@ int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count)
     if (!(flags & CAST_F_META_BITMASK) && !(N == 2 && M == 4)) return CAST_ERR_NM;
     const uint32_t known = CAST_F_RESELECT | CAST_F_COUNT_FLIPS | CAST_F_META_BITMASK |
                            CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE | CAST_F_EMIT_COMPRESSED |
-                           CAST_F_GRAD_OF_SCALED;
+                           CAST_F_GRAD_OF_SCALED | CAST_F_MASK_STATS;
     if (flags & ~known) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && (flags & CAST_F_EMIT_DENSE)) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && M > kUnitElems) return CAST_ERR_NM;
@@ -144,12 +144,14 @@ static void fast_div(uint32_t d, uint32_t* magic, uint32_t* shift)
 }
 
 TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
-                     const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad)
+                     const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad,
+                     const uint32_t* meta_ref)
 {
     TensorDesc d;
     std::memset(&d, 0, sizeof d);
     d.w = w; d.m = m; d.v = v; d.g = g; d.w_fwd = w_fwd; d.meta = meta; d.scale = scale;
     d.scale_grad = scale ? scale_grad : nullptr;
+    d.meta_ref = reinterpret_cast<const uint8_t*>(meta_ref);
     d.n_units = (uint32_t)((uint64_t)rows * (uint64_t)cols / kUnitElems);
     if (scale) {
         const uint32_t seg_units = (uint32_t)(cols / scale_groups / kUnitElems);
@@ -161,101 +163,57 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
 // ---------------------------------------------------------------------------------------------
 // launches
 
-namespace {
+// The kernels are instantiated in step_inst.cu, compiled once per (M, two_four, statistics) with every valid
+// compile-time flag word of that slice; each such object exports one launcher.
+#define CAST_DECLARE_STEP_LAUNCHER(M, TF, S) int launch_step_m##M##_tf##TF##_s##S(uint32_t flag_word, const StepLaunch& a);
+CAST_DECLARE_STEP_LAUNCHER(2, 0, 0) CAST_DECLARE_STEP_LAUNCHER(2, 0, 1)
+CAST_DECLARE_STEP_LAUNCHER(4, 0, 0) CAST_DECLARE_STEP_LAUNCHER(4, 0, 1)
+CAST_DECLARE_STEP_LAUNCHER(4, 1, 0) CAST_DECLARE_STEP_LAUNCHER(4, 1, 1)
+CAST_DECLARE_STEP_LAUNCHER(8, 0, 0) CAST_DECLARE_STEP_LAUNCHER(8, 0, 1)
+CAST_DECLARE_STEP_LAUNCHER(16, 0, 0) CAST_DECLARE_STEP_LAUNCHER(16, 0, 1)
+CAST_DECLARE_STEP_LAUNCHER(32, 0, 0) CAST_DECLARE_STEP_LAUNCHER(32, 0, 1)
+#undef CAST_DECLARE_STEP_LAUNCHER
 
-// The flag word is a compile-time constant of the kernel in the common cases.
-int mode_of(const StepConsts& c, int M)
+uint32_t kernel_flag_word(uint32_t flags)
 {
-    const bool two_four = M == 4 && c.n_keep == 2;
-    switch (c.flags) {
-        case kReselect:                                return two_four ? kModeSelectIdx : kModeGeneric;
-        case kReselect | kEmitCompressed:              return two_four ? kModeSelectIdxPacked : kModeGeneric;
-        case 0u:                                       return two_four ? kModeReuseIdx : kModeGeneric;
-        case kEmitDense:                               return two_four ? kModeReuseIdxDense : kModeGeneric;
-        case kReselect | kCountFlips:                  return two_four ? kModeSelectIdxFlips : kModeGeneric;
-        case kReselect | kCountFlips | kEmitDense:     return two_four ? kModeSelectIdxFlipsDense : kModeGeneric;
-        case kEmitDense | kGradOfScaled:               return two_four ? kModeReuseIdxDenseScaled : kModeGeneric;
-        case kReselect | kCountFlips | kEmitDense | kGradOfScaled:
-                                                       return two_four ? kModeSelectIdxFlipsDenseScaled : kModeGeneric;
-        case kReselect | kMetaBitmask:                 return kModeSelectMask;
-        case kReselect | kMetaBitmask | kCountFlips:   return kModeSelectMaskFlips;
-    }
-    return kModeGeneric;
+    uint32_t f = flags & kCompileTimeFlags;
+    if (!(f & kReselect)) f &= ~kCountFlips;       // a reused mask has no flips: the counter gets nothing added
+    return f;
 }
 
-template <int M, int MODE>
-int launch_single_t(const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+int launch_step(const StepLaunch& a, int M)
 {
-    const uint32_t tiles = tiles_of(d);
-    if (tiles == 0) return CAST_OK;
-    if (tiles > kMaxTiles) return CAST_ERR_SHAPE;
-    // one CTA per tile: the hardware scheduler hands tiles out in address order
-    adams_nm_kernel<M, MODE><<<tiles, kThreads, 0, stream>>>(d, c, flip_count);
-    CAST_CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return CAST_OK;
-}
-
-template <int M, int MODE>
-int launch_multi_t(const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
-{
-    const uint32_t tiles = p.tile_start[p.n_tensors];
-    if (tiles == 0) return CAST_OK;
-    adams_nm_multi_kernel<M, MODE><<<tiles, kThreads, 0, stream>>>(p, c, flip_count);
-    CAST_CUDA_TRY(cudaGetLastError());
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return CAST_OK;
-}
-
-// Walks the mode list at compile time: instantiates the kernel of every mode that exists for this M.
-template <int M, int MODE = 0>
-int launch_single_m(int mode, const TensorDesc& d, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
-{
-    if constexpr (MODE >= kModeCount) {
-        return CAST_ERR_NM;
-    } else {
-        if constexpr (M == 4 || !mode_is_2of4_only(MODE))
-            if (mode == MODE) return launch_single_t<M, MODE>(d, c, flip_count, stream);
-        return launch_single_m<M, MODE + 1>(mode, d, c, flip_count, stream);
-    }
-}
-
-template <int M, int MODE = 0>
-int launch_multi_m(int mode, const MultiParams& p, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
-{
-    if constexpr (MODE >= kModeCount) {
-        return CAST_ERR_NM;
-    } else {
-        if constexpr (M == 4 || !mode_is_2of4_only(MODE))
-            if (mode == MODE) return launch_multi_t<M, MODE>(p, c, flip_count, stream);
-        return launch_multi_m<M, MODE + 1>(mode, p, c, flip_count, stream);
-    }
-}
-
-}  // namespace
-
-int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
-{
+    const uint32_t f = kernel_flag_word(a.c->flags);
+    const bool two_four = M == 4 && a.c->n_keep == 2;
+    const bool st = (f & kMaskStats) != 0;
+    if (!step_kernel_exists(M, two_four, f)) return CAST_ERR_NM;
+    if (a.single ? tiles_of(*a.single) == 0 : a.multi->tile_start[a.multi->n_tensors] == 0) return CAST_OK;
+    if (a.single && tiles_of(*a.single) > kMaxTiles) return CAST_ERR_SHAPE;
+    int rc = CAST_ERR_NM;
     switch (M) {
-        case 2:  return launch_single_m<2>(mode_of(c, 2), d, c, flip_count, stream);
-        case 4:  return launch_single_m<4>(mode_of(c, 4), d, c, flip_count, stream);
-        case 8:  return launch_single_m<8>(mode_of(c, 8), d, c, flip_count, stream);
-        case 16: return launch_single_m<16>(mode_of(c, 16), d, c, flip_count, stream);
-        case 32: return launch_single_m<32>(mode_of(c, 32), d, c, flip_count, stream);
+        case 2:  rc = st ? launch_step_m2_tf0_s1(f, a) : launch_step_m2_tf0_s0(f, a); break;
+        case 4:  rc = two_four ? (st ? launch_step_m4_tf1_s1(f, a) : launch_step_m4_tf1_s0(f, a))
+                               : (st ? launch_step_m4_tf0_s1(f, a) : launch_step_m4_tf0_s0(f, a)); break;
+        case 8:  rc = st ? launch_step_m8_tf0_s1(f, a) : launch_step_m8_tf0_s0(f, a); break;
+        case 16: rc = st ? launch_step_m16_tf0_s1(f, a) : launch_step_m16_tf0_s0(f, a); break;
+        case 32: rc = st ? launch_step_m32_tf0_s1(f, a) : launch_step_m32_tf0_s0(f, a); break;
     }
-    return CAST_ERR_NM;
+    if (rc == CAST_OK) g_launches.fetch_add(1, std::memory_order_relaxed);
+    return rc;
 }
 
-int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
+int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
+                  cast_mask_stats_t* stats)
 {
-    switch (M) {
-        case 2:  return launch_multi_m<2>(mode_of(c, 2), p, c, flip_count, stream);
-        case 4:  return launch_multi_m<4>(mode_of(c, 4), p, c, flip_count, stream);
-        case 8:  return launch_multi_m<8>(mode_of(c, 8), p, c, flip_count, stream);
-        case 16: return launch_multi_m<16>(mode_of(c, 16), p, c, flip_count, stream);
-        case 32: return launch_multi_m<32>(mode_of(c, 32), p, c, flip_count, stream);
-    }
-    return CAST_ERR_NM;
+    const StepLaunch a = {&d, nullptr, &c, flip_count, reinterpret_cast<MaskStats*>(stats), stream};
+    return launch_step(a, M);
+}
+
+int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
+                 cast_mask_stats_t* stats)
+{
+    const StepLaunch a = {nullptr, &p, &c, flip_count, reinterpret_cast<MaskStats*>(stats), stream};
+    return launch_step(a, M);
 }
 
 void fill_hint_table(uint32_t n_tensors, const uint32_t* tile_start, uint16_t* hint, uint32_t* hint_shift)
@@ -345,6 +303,7 @@ extern "C" int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
 {
     int rc;
     if ((rc = check_nm_flags(N, M, flags, flip_count)) != CAST_OK) return rc;
+    if (flags & CAST_F_MASK_STATS) return CAST_ERR_NULL;      // this signature has no accumulator: cast_adams_step_stats
     StepConsts c;
     if ((rc = make_step_consts(lr, beta1, beta2, eps, l1_coeff, step, total_steps, N, flags, &c)) != CAST_OK) return rc;
     if (!w || !m || !v || !g || !w_fwd_bf16 || !meta) return CAST_ERR_NULL;
@@ -369,12 +328,45 @@ int check_tensor_scale_grad(const cast_tensor_t& t, int N, int M, uint32_t fwd_f
 }
 }  // namespace
 
+namespace {
+// The accumulator of CAST_F_MASK_STATS: required with the flag, 8-byte aligned device memory.
+int check_stats_ptr(uint32_t flags, const cast_mask_stats_t* stats)
+{
+    if (!(flags & CAST_F_MASK_STATS)) return CAST_OK;
+    if (!stats) return CAST_ERR_NULL;
+    if ((uintptr_t)stats & 7u) return CAST_ERR_ALIGN;
+    const void* p[1] = {stats};
+    return check_device_memory(p, 1);
+}
+// The optional reference mask of one matrix: 16-byte aligned device memory that the step does not write.
+int check_meta_ref(const cast_tensor_t& t)
+{
+    if (!t.meta_ref) return CAST_OK;
+    if ((uintptr_t)t.meta_ref & 15u) return CAST_ERR_ALIGN;
+    const uint64_t P = (uint64_t)t.rows * (uint64_t)t.cols;
+    const uintptr_t lo = (uintptr_t)t.meta_ref, hi = lo + P / 8;
+    const void* written[5] = {t.w, t.m, t.v, t.w_fwd, t.meta};
+    const uint64_t bytes[5] = {4 * P, 4 * P, 4 * P, 2 * P, P / 8};
+    for (int i = 0; i < 5; ++i)
+        if (lo < (uintptr_t)written[i] + bytes[i] && (uintptr_t)written[i] < hi) return CAST_ERR_ALIAS;
+    const void* p[1] = {t.meta_ref};
+    return check_device_memory(p, 1);
+}
+}  // namespace
+
 extern "C" int cast_adams_step_ex(const cast_tensor_t* t, int N, int M, const cast_hyper_t* h,
                                   unsigned long long* flip_count, cast_stream_t stream)
+{
+    return cast_adams_step_stats(t, N, M, h, flip_count, nullptr, stream);
+}
+
+extern "C" int cast_adams_step_stats(const cast_tensor_t* t, int N, int M, const cast_hyper_t* h,
+                                     unsigned long long* flip_count, cast_mask_stats_t* stats, cast_stream_t stream)
 {
     if (!t || !h) return CAST_ERR_NULL;
     int rc;
     if ((rc = check_nm_flags(N, M, h->flags, flip_count)) != CAST_OK) return rc;
+    if ((rc = check_stats_ptr(h->flags, stats)) != CAST_OK) return rc;
     StepConsts c;
     if ((rc = make_step_consts(h->lr, h->beta1, h->beta2, h->eps, h->l1_coeff, h->step, h->total_steps, N, h->flags, &c)) != CAST_OK) return rc;
     if (!t->w || !t->m || !t->v || !t->g || !t->w_fwd || !t->meta) return CAST_ERR_NULL;
@@ -384,9 +376,10 @@ extern "C" int cast_adams_step_ex(const cast_tensor_t* t, int N, int M, const ca
     const void* ptrs[8] = {t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, (h->flags & CAST_F_COUNT_FLIPS) ? flip_count : nullptr};
     if ((rc = check_device_memory(ptrs, 8)) != CAST_OK) return rc;
     if ((rc = check_tensor_scale_grad(*t, N, M, h->flags)) != CAST_OK) return rc;
+    if ((rc = check_meta_ref(*t)) != CAST_OK) return rc;
     const TensorDesc d = make_desc(t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, t->scale_groups, t->rows, t->cols,
-                                   t->scale_grad);
-    return launch_single(d, M, c, flip_count, (cudaStream_t)stream);
+                                   t->scale_grad, t->meta_ref);
+    return launch_single(d, M, c, flip_count, (cudaStream_t)stream, (h->flags & CAST_F_MASK_STATS) ? stats : nullptr);
 }
 
 extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out)
@@ -418,6 +411,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
         const void* ptrs[7] = {t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale};
         if ((rc = check_device_memory(ptrs, 7)) != CAST_OK) return rc;
         if ((rc = check_tensor_scale_grad(t, N, M, plan_flags)) != CAST_OK) return rc;
+        if ((rc = check_meta_ref(t)) != CAST_OK) return rc;
     }
 
     Plan* p = new (std::nothrow) Plan;
@@ -435,7 +429,8 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
             uint64_t tiles = 0;
             while (i < n_tensors && mp.n_tensors < (uint32_t)kMaxLaunchTensors) {
                 const cast_tensor_t& t = tensors[i];
-                const TensorDesc d = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols, t.scale_grad);
+                const TensorDesc d = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols, t.scale_grad,
+                                               t.meta_ref);
                 if (tiles + tiles_of(d) > kMaxTiles) break;      // a single matrix always fits (rows*cols < 2^31)
                 mp.desc[mp.n_tensors] = d;
                 mp.tile_start[mp.n_tensors] = (uint32_t)tiles;
@@ -459,11 +454,18 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
 
 extern "C" int cast_plan_step(void* plan, const cast_hyper_t* h, unsigned long long* flip_count, cast_stream_t stream)
 {
+    return cast_plan_step_stats(plan, h, flip_count, nullptr, stream);
+}
+
+extern "C" int cast_plan_step_stats(void* plan, const cast_hyper_t* h, unsigned long long* flip_count,
+                                    cast_mask_stats_t* stats, cast_stream_t stream)
+{
     Plan* p = (Plan*)plan;
     if (!p || p->magic != kPlanMagic) return CAST_ERR_PLAN;
     if (!h) return CAST_ERR_NULL;
     int rc;
     if ((rc = check_nm_flags(p->N, p->M, h->flags, flip_count)) != CAST_OK) return rc;
+    if ((rc = check_stats_ptr(h->flags, stats)) != CAST_OK) return rc;
     if ((h->flags & CAST_F_EMIT_COMPRESSED) != p->plan_flags) return CAST_ERR_PLAN;
     StepConsts c;
     if ((rc = make_step_consts(h->lr, h->beta1, h->beta2, h->eps, h->l1_coeff, h->step, h->total_steps,
@@ -476,7 +478,8 @@ extern "C" int cast_plan_step(void* plan, const cast_hyper_t* h, unsigned long l
         if ((rc = check_device_memory(fp, 1)) != CAST_OK) return rc;
     }
     for (const MultiParams& mp : p->launches)
-        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream)) != CAST_OK) return rc;
+        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream,
+                               (h->flags & CAST_F_MASK_STATS) ? stats : nullptr)) != CAST_OK) return rc;
     return CAST_OK;
 }
 

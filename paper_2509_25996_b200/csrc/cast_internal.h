@@ -49,7 +49,8 @@ int check_device_memory(const void* const* ptrs, int n);
 
 // Kernel-side description of one (already validated) matrix.
 TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
-                     const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad = nullptr);
+                     const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad = nullptr,
+                     const uint32_t* meta_ref = nullptr);
 
 // The optional scale-gradient buffer of one matrix: needs a scale, 16-byte alignment, device memory, no overlap
 // with the matrix's other buffers (checked by address only).
@@ -58,10 +59,20 @@ int check_scale_grad(const float* scale_grad, const float* scale, int scale_grou
 
 inline uint32_t tiles_of(const TensorDesc& d) { return (d.n_units + kTileUnits - 1) / kTileUnits; }
 
-// Launch over one matrix or over a table of matrices (both passed by value as kernel parameters).
+// One launch of the step: over one matrix (`single`) or over a table of matrices (`multi`), both passed by value
+// as kernel parameters.  The kernel is picked by M, N and the compile-time part of c->flags.
+struct StepLaunch {
+    const TensorDesc* single;
+    const MultiParams* multi;
+    const StepConsts* c;
+    unsigned long long* flip_count;
+    MaskStats* stats;
+    cudaStream_t stream;
+};
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count,
-                  cudaStream_t stream);
-int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
+                  cudaStream_t stream, cast_mask_stats_t* stats = nullptr);
+int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
+                 cast_mask_stats_t* stats = nullptr);
 
 // Fill the tile-to-matrix hint table (kHintEntries entries) of a launch whose tile_start[0..n_tensors] is set:
 // hint[b] = the matrix that holds tile b << *hint_shift.

@@ -75,7 +75,7 @@ prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t fl
             select_2of4(ab, kept);
             select_2of4(ab + 4, kept + 4);
         } else {
-            if (flags & kReselect) keep = select_by_rank<M>(ab, n_keep);          // uniform branch: all lanes shuffle
+            if (flags & kReselect) keep = select_top_n<M>(ab, n_keep);           // uniform branch: all lanes shuffle
             else keep = keep_from_meta_byte(stored[j], bitmask);
 #pragma unroll
             for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
