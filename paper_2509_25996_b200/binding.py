@@ -34,9 +34,11 @@ CAST_F_V_KEPT_FROM_G = 1 << 3
 CAST_F_EMIT_DENSE = 1 << 4
 CAST_F_EMIT_COMPRESSED = 1 << 5
 CAST_F_GRAD_OF_SCALED = 1 << 6
+CAST_F_MASK_STATS = 1 << 7
 
 EXPORTS = (
-    "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_scale_adam_step", "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_destroy",
+    "cast_adams_step", "cast_adams_step_ex", "cast_adams_step_stats", "cast_scale_adam_step", "cast_plan_scale_adam_step",
+    "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_step_stats", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
@@ -56,6 +58,7 @@ class cast_tensor_t(ctypes.Structure):
         ("scale", ctypes.c_void_p), ("scale_groups", ctypes.c_int32),
         ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
         ("scale_grad", ctypes.c_void_p),
+        ("meta_ref", ctypes.c_void_p),
     ]
 
 
@@ -95,6 +98,9 @@ def load_library() -> ctypes.CDLL:
     lib.cast_adams_step_ex.restype = ctypes.c_int
     lib.cast_adams_step_ex.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.POINTER(cast_hyper_t),
                                        ctypes.c_void_p, ctypes.c_void_p]
+    lib.cast_adams_step_stats.restype = ctypes.c_int
+    lib.cast_adams_step_stats.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.POINTER(cast_hyper_t),
+                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.cast_scale_adam_step.restype = ctypes.c_int
     lib.cast_scale_adam_step.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_float,
                                                                  ctypes.c_float, ctypes.c_int64, ctypes.c_int, ctypes.c_void_p]
@@ -110,6 +116,8 @@ def load_library() -> ctypes.CDLL:
                                         ctypes.POINTER(ctypes.c_void_p)]
     lib.cast_plan_step.restype = ctypes.c_int
     lib.cast_plan_step.argtypes = [ctypes.c_void_p, ctypes.POINTER(cast_hyper_t), ctypes.c_void_p, ctypes.c_void_p]
+    lib.cast_plan_step_stats.restype = ctypes.c_int
+    lib.cast_plan_step_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(cast_hyper_t), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.cast_plan_destroy.restype = ctypes.c_int
     lib.cast_plan_destroy.argtypes = [ctypes.c_void_p]
     lib.cast_host_ctx_create.restype = ctypes.c_int
@@ -201,9 +209,9 @@ def cast_plan_scale_adam_step(plan, m_as, v_as, lr, beta1, beta2, eps, step, cle
                                                     _stream(stream))
 
 
-def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols, scale_grad=None) -> cast_tensor_t:
+def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols, scale_grad=None, meta_ref=None) -> cast_tensor_t:
     return cast_tensor_t(_ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd), _ptr(meta), _ptr(scale),
-                         int(scale_groups), int(rows), int(cols), _ptr(scale_grad))
+                         int(scale_groups), int(rows), int(cols), _ptr(scale_grad), _ptr(meta_ref))
 
 
 def cast_adams_step_ex(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: Optional[cast_hyper_t],
@@ -211,6 +219,14 @@ def cast_adams_step_ex(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: O
     t = ctypes.byref(tensor) if tensor is not None else None
     h = ctypes.byref(hyper) if hyper is not None else None
     return load_library().cast_adams_step_ex(t, int(N), int(M), h, _ptr(flip_count), _stream(stream))
+
+
+def cast_adams_step_stats(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: Optional[cast_hyper_t],
+                          flip_count=None, stats=None, stream=None) -> int:
+    """`stats`: device buffer of sizeof(cast_mask_stats_t) = 32 bytes that a step with CAST_F_MASK_STATS adds to."""
+    t = ctypes.byref(tensor) if tensor is not None else None
+    h = ctypes.byref(hyper) if hyper is not None else None
+    return load_library().cast_adams_step_stats(t, int(N), int(M), h, _ptr(flip_count), _ptr(stats), _stream(stream))
 
 
 def cast_scale_adam_step(a, m_a, v_a, grad, n, lr, beta1, beta2, eps, step, clear_grad=True, stream=None) -> int:
@@ -243,6 +259,11 @@ def make_hyper(lr, beta1, beta2, eps, l1_coeff, step, total_steps, flags) -> cas
 def cast_plan_step(plan, hyper: Optional[cast_hyper_t], flip_count=None, stream=None) -> int:
     h = ctypes.byref(hyper) if hyper is not None else None
     return load_library().cast_plan_step(plan, h, _ptr(flip_count), _stream(stream))
+
+
+def cast_plan_step_stats(plan, hyper: Optional[cast_hyper_t], flip_count=None, stats=None, stream=None) -> int:
+    h = ctypes.byref(hyper) if hyper is not None else None
+    return load_library().cast_plan_step_stats(plan, h, _ptr(flip_count), _ptr(stats), _stream(stream))
 
 
 def cast_plan_destroy(plan) -> int:

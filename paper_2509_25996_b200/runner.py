@@ -5,6 +5,7 @@ every arithmetic step runs in the CUDA library.
 """
 from __future__ import annotations
 
+import ctypes
 from dataclasses import dataclass
 from typing import List, Optional, Sequence, Tuple
 
@@ -28,6 +29,7 @@ class MatrixState:
     scale_grad: Optional[torch.Tensor] = None      # fp32 [rows, n]; with a learned scale
     scale_m: Optional[torch.Tensor] = None         # Adam moments of the scale
     scale_v: Optional[torch.Tensor] = None
+    meta_ref: Optional[torch.Tensor] = None        # int32 [rows, cols/32]; reference mask of the App. C statistics
 
 
 @dataclass
@@ -46,11 +48,14 @@ class DeviceModelState:
 
     def __init__(self, shapes: Sequence[Tuple[int, int]], N: int = 2, M: int = 4, seed: int = 0,
                  device="cuda:0", scale_mode: str = "ones", first_tensor_index: int = 0, compressed: bool = False,
-                 learned_scale: bool = False):
+                 learned_scale: bool = False, reference_masks: bool = False):
         """compressed: the forward-weight buffers hold only the kept entries ([rows, cols*N/M]); every step of
         this state then carries CAST_F_EMIT_COMPRESSED.
         learned_scale: every matrix gets a scale-gradient buffer (filled by steps that carry
-        CAST_F_GRAD_OF_SCALED) and Adam moments for its scale; scale_step() then trains the scales."""
+        CAST_F_GRAD_OF_SCALED) and Adam moments for its scale; scale_step() then trains the scales.
+        reference_masks: every matrix gets a second metadata buffer (zeros until the caller fills it, e.g. with
+        the initial mask), against which steps that carry CAST_F_MASK_STATS count ||M_t - M_ref||_0; the sums
+        land in self.stats."""
         self.device = torch.device(device)
         self.N, self.M = N, M
         self.compressed = compressed
@@ -70,10 +75,14 @@ class DeviceModelState:
                 mat.scale_grad = torch.zeros_like(inp.scale)
                 mat.scale_m = torch.zeros_like(inp.scale)
                 mat.scale_v = torch.zeros_like(inp.scale)
+            if reference_masks:
+                self.mats[-1].meta_ref = torch.zeros_like(self.mats[-1].meta)
         self.n_params = sum(s.rows * s.cols for s in self.mats)
         self.flips = torch.zeros(1, dtype=torch.int64, device=self.device)
+        self.stats = torch.zeros(ctypes.sizeof(B.cast_mask_stats_t), dtype=torch.uint8, device=self.device)
         tensors = [B.make_tensor(s.w, s.m, s.v, s.g, s.w_fwd, s.meta, s.scale,
-                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad) for s in self.mats]
+                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad, s.meta_ref)
+                   for s in self.mats]
         rc, self.plan = B.cast_plan_create_ex(tensors, N, M, B.CAST_F_EMIT_COMPRESSED if compressed else 0)
         B.check(rc)
 
@@ -84,7 +93,15 @@ class DeviceModelState:
         h = B.make_hyper(hyper.lr, hyper.beta1, hyper.beta2, hyper.eps, hyper.l1_coeff,
                          hyper.step, hyper.total_steps, flags)
         s = stream if stream is not None else torch.cuda.current_stream(self.device)
-        B.check(B.cast_plan_step(self.plan, h, self.flips if flags & B.CAST_F_COUNT_FLIPS else None, s))
+        flips = self.flips if flags & B.CAST_F_COUNT_FLIPS else None
+        if flags & B.CAST_F_MASK_STATS:
+            B.check(B.cast_plan_step_stats(self.plan, h, flips, self.stats, s))
+        else:
+            B.check(B.cast_plan_step(self.plan, h, flips, s))
+
+    def read_stats(self) -> "B.cast_mask_stats_t":
+        """Host copy of the statistics accumulator (synchronises)."""
+        return B.cast_mask_stats_t.from_buffer_copy(self.stats.cpu().numpy().tobytes())
 
     def scale_step(self, lr: float, hyper: Hyper, stream=None) -> None:
         """Adam step of every scale matrix from the accumulated scale gradients (which it clears), one launch."""
