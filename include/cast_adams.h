@@ -91,7 +91,8 @@ enum cast_flags {
                                        ||W_t||_1 on the UPDATED weights with this step's kept set M_t, and
                                        ||M_t - M_ref||_0 against the reference mask `meta_ref` of the matrix (the
                                        initial mask for the initial flip rate i_t; 0 is added where meta_ref is
-                                       NULL).  Only cast_adams_step_stats / cast_plan_step_stats take this flag */
+                                       NULL).  Only cast_plan_step_stats takes this flag, on a plan created
+                                       with it (other entry points answer CAST_ERR_PLAN)                  */
 };
 
 /*
@@ -185,17 +186,6 @@ CAST_API int cast_adams_step_ex(const cast_tensor_t* tensor, int N, int M, const
                        unsigned long long* flip_count, cast_stream_t stream);
 
 /*
- * cast_adams_step_stats -- cast_adams_step_ex that may carry CAST_F_MASK_STATS: the i_t and S_t sums of App. C come
- * out of the step itself (the step holds |w_t|, the kept set and the stored metadata in registers), next to the
- * flip count, instead of a second pass over the weights.
- *   stats   device, 8-byte aligned, ADDED to (zero it before the first matrix of a model); required with the flag,
- *           ignored without it.  Values: see cast_mask_stats_t; W is the weight after this update, M the kept set
- *           of this step (selected now or reused), M_ref the matrix's `meta_ref`.
- */
-CAST_API int cast_adams_step_stats(const cast_tensor_t* tensor, int N, int M, const cast_hyper_t* hyper,
-                          unsigned long long* flip_count, cast_mask_stats_t* stats, cast_stream_t stream);
-
-/*
  * cast_scale_adam_step -- the optimizer step of the scale matrix A of Eq. 12, which the paper learns jointly
  * with the weights (Sec. 4.2) without naming its optimizer: plain Adam with bias correction (Alg. 1 without
  * its mask and decay lines), element-wise over `n` = rows * scale_groups entries, in fp64 internally.
@@ -228,7 +218,7 @@ CAST_API int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* con
  * cast_plan_create  validates `n_tensors` descriptors (host array, copied) and returns an opaque handle
  *                   in *plan_out.  The plan is host memory only: it holds the launch tables, which travel
  *                   to the device as kernel parameters at every step, and allocates nothing on the
- *                   device.  All matrices share N:M.  The buffers named by the descriptors stay owned by
+ *                   device (but see CAST_F_MASK_STATS under cast_plan_create_ex).  All matrices share N:M.  The buffers named by the descriptors stay owned by
  *                   the caller and must outlive the plan's use.
  * cast_plan_step    launches one grid over all matrices on `stream` (ceil(n_tensors / 320) grids for
  *                   larger lists); arguments as cast_adams_step.  The plan may be stepped any number of
@@ -237,15 +227,29 @@ CAST_API int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* con
  * cast_plan_destroy frees the handle (no device work).
  */
 CAST_API int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out);
-/* As cast_plan_create, for matrices whose w_fwd buffers have the compressed size: plan_flags is
- * CAST_F_EMIT_COMPRESSED (or 0 = cast_plan_create).  Every step of such a plan must carry that flag, and a step
- * of an ordinary plan must not (CAST_ERR_PLAN otherwise): the buffer sizes are fixed when the plan is made. */
+/* As cast_plan_create, with plan_flags = OR of
+ *   CAST_F_EMIT_COMPRESSED  the w_fwd buffers have the compressed size.  Every step of such a plan must carry that
+ *                           flag, and a step of an ordinary plan must not (CAST_ERR_PLAN otherwise): the buffer
+ *                           sizes are fixed when the plan is made;
+ *   CAST_F_MASK_STATS       the plan may take steps with the statistics epilogue (cast_plan_step_stats); this is
+ *                           the one case in which a plan allocates device memory (32 KB).
+ * 0 = cast_plan_create. */
 CAST_API int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, int N, int M, uint32_t plan_flags,
                         void** plan_out);
 CAST_API int cast_plan_step(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
                    cast_stream_t stream);
-/* cast_plan_step that may carry CAST_F_MASK_STATS (see cast_adams_step_stats): the model-wide sums of App. C in the
- * same launch as the step.  The reference masks are the `meta_ref` fields the plan was created with. */
+/*
+ * cast_plan_step_stats -- cast_plan_step that may carry CAST_F_MASK_STATS: the i_t and S_t sums of App. C come out
+ * of the step itself (it holds |w_t|, the kept set and the stored metadata in registers), next to the flip count,
+ * instead of a second pass over the weights (cast_plan_mask_stats, 4.25 B per parameter).
+ *   stats   device, 8-byte aligned, ADDED to (the caller zeroes it); required with the flag, ignored without it.
+ *           Values: see cast_mask_stats_t; W is the weight after this update, M the kept set of this step
+ *           (selected now or reused), M_ref the `meta_ref` of each matrix as given when the plan was created.
+ * The plan must have been created with CAST_F_MASK_STATS among its plan_flags (CAST_ERR_PLAN otherwise): such a
+ * plan owns 32 KB of device memory (1024 partial accumulators that the step's CTAs add to, so that their atomics
+ * do not queue on one address), allocated by cast_plan_create_ex and freed by cast_plan_destroy.  A step with the
+ * flag launches one more, one-CTA kernel that folds the partial sums into `stats` and clears them.
+ */
 CAST_API int cast_plan_step_stats(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
                          cast_mask_stats_t* stats, cast_stream_t stream);
 CAST_API int cast_plan_destroy(void* plan);

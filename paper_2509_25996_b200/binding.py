@@ -37,7 +37,7 @@ CAST_F_GRAD_OF_SCALED = 1 << 6
 CAST_F_MASK_STATS = 1 << 7
 
 EXPORTS = (
-    "cast_adams_step", "cast_adams_step_ex", "cast_adams_step_stats", "cast_scale_adam_step", "cast_plan_scale_adam_step",
+    "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_scale_adam_step",
     "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_step_stats", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
@@ -98,9 +98,6 @@ def load_library() -> ctypes.CDLL:
     lib.cast_adams_step_ex.restype = ctypes.c_int
     lib.cast_adams_step_ex.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.POINTER(cast_hyper_t),
                                        ctypes.c_void_p, ctypes.c_void_p]
-    lib.cast_adams_step_stats.restype = ctypes.c_int
-    lib.cast_adams_step_stats.argtypes = [ctypes.POINTER(cast_tensor_t), ctypes.c_int, ctypes.c_int, ctypes.POINTER(cast_hyper_t),
-                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
     lib.cast_scale_adam_step.restype = ctypes.c_int
     lib.cast_scale_adam_step.argtypes = [ctypes.c_void_p] * 4 + [ctypes.c_int64, ctypes.c_float, ctypes.c_float, ctypes.c_float,
                                                                  ctypes.c_float, ctypes.c_int64, ctypes.c_int, ctypes.c_void_p]
@@ -221,14 +218,6 @@ def cast_adams_step_ex(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: O
     return load_library().cast_adams_step_ex(t, int(N), int(M), h, _ptr(flip_count), _stream(stream))
 
 
-def cast_adams_step_stats(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: Optional[cast_hyper_t],
-                          flip_count=None, stats=None, stream=None) -> int:
-    """`stats`: device buffer of sizeof(cast_mask_stats_t) = 32 bytes that a step with CAST_F_MASK_STATS adds to."""
-    t = ctypes.byref(tensor) if tensor is not None else None
-    h = ctypes.byref(hyper) if hyper is not None else None
-    return load_library().cast_adams_step_stats(t, int(N), int(M), h, _ptr(flip_count), _ptr(stats), _stream(stream))
-
-
 def cast_scale_adam_step(a, m_a, v_a, grad, n, lr, beta1, beta2, eps, step, clear_grad=True, stream=None) -> int:
     return load_library().cast_scale_adam_step(_ptr(a), _ptr(m_a), _ptr(v_a), _ptr(grad), int(n), lr, beta1, beta2, eps,
                                                int(step), 1 if clear_grad else 0, _stream(stream))
@@ -244,7 +233,7 @@ def cast_plan_create(tensors: Sequence[cast_tensor_t], N: int, M: int):
 
 
 def cast_plan_create_ex(tensors: Sequence[cast_tensor_t], N: int, M: int, plan_flags: int):
-    """Returns (status, plan handle or None); plan_flags: CAST_F_EMIT_COMPRESSED or 0."""
+    """Returns (status, plan handle or None); plan_flags: OR of CAST_F_EMIT_COMPRESSED, CAST_F_MASK_STATS, or 0."""
     n = len(tensors)
     arr = (cast_tensor_t * max(n, 1))(*tensors)
     out = ctypes.c_void_p(None)
@@ -262,6 +251,7 @@ def cast_plan_step(plan, hyper: Optional[cast_hyper_t], flip_count=None, stream=
 
 
 def cast_plan_step_stats(plan, hyper: Optional[cast_hyper_t], flip_count=None, stats=None, stream=None) -> int:
+    """`stats`: device buffer of sizeof(cast_mask_stats_t) = 32 bytes that a step with CAST_F_MASK_STATS adds to."""
     h = ctypes.byref(hyper) if hyper is not None else None
     return load_library().cast_plan_step_stats(plan, h, _ptr(flip_count), _ptr(stats), _stream(stream))
 

@@ -202,17 +202,16 @@ int launch_step(const StepLaunch& a, int M)
     return rc;
 }
 
-int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
-                  cast_mask_stats_t* stats)
+int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    const StepLaunch a = {&d, nullptr, &c, flip_count, reinterpret_cast<MaskStats*>(stats), stream};
+    const StepLaunch a = {&d, nullptr, &c, flip_count, nullptr, stream};
     return launch_step(a, M);
 }
 
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
-                 cast_mask_stats_t* stats)
+                 MaskStats* stat_slots)
 {
-    const StepLaunch a = {nullptr, &p, &c, flip_count, reinterpret_cast<MaskStats*>(stats), stream};
+    const StepLaunch a = {nullptr, &p, &c, flip_count, stat_slots, stream};
     return launch_step(a, M);
 }
 
@@ -243,9 +242,46 @@ struct Plan {
     int device;
     int N, M;
     int n_tensors;
-    uint32_t plan_flags;                 // CAST_F_EMIT_COMPRESSED or 0: fixes the size of the w_fwd buffers
+    uint32_t plan_flags;                 // CAST_F_EMIT_COMPRESSED fixes the size of the w_fwd buffers; CAST_F_MASK_STATS
+                                         // says the plan owns the statistics slots
+    MaskStats* stat_slots;               // device, kStatSlots accumulators (zero between steps), or nullptr
     std::vector<MultiParams> launches;   // one table per launch of up to kMaxLaunchTensors matrices
 };
+
+// Adds the sum of the slots to the caller's accumulator and clears them (one CTA of kStatSlots threads).
+__global__ void __launch_bounds__(kStatSlots)
+fold_stat_slots_kernel(MaskStats* __restrict__ slots, MaskStats* __restrict__ out)
+{
+    MaskStats mine = slots[threadIdx.x];
+    slots[threadIdx.x] = MaskStats{0ull, 0ull, 0.0, 0.0};
+    unsigned long long d = mine.mask_diff;
+    double k = mine.kept_abs_sum, t = mine.total_abs_sum;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        d += __shfl_down_sync(0xFFFFFFFFu, d, o);
+        k += __shfl_down_sync(0xFFFFFFFFu, k, o);
+        t += __shfl_down_sync(0xFFFFFFFFu, t, o);
+    }
+    __shared__ unsigned long long s_d[kStatSlots / 32];
+    __shared__ double s_k[kStatSlots / 32], s_t[kStatSlots / 32];
+    if ((threadIdx.x & 31) == 0) { s_d[threadIdx.x >> 5] = d; s_k[threadIdx.x >> 5] = k; s_t[threadIdx.x >> 5] = t; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        d = s_d[threadIdx.x]; k = s_k[threadIdx.x]; t = s_t[threadIdx.x];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            d += __shfl_down_sync(0xFFFFFFFFu, d, o);
+            k += __shfl_down_sync(0xFFFFFFFFu, k, o);
+            t += __shfl_down_sync(0xFFFFFFFFu, t, o);
+        }
+        if (threadIdx.x == 0) {
+            atomicAdd(&out->mask_diff, d);
+            atomicAdd(&out->kept_abs_sum, k);
+            atomicAdd(&out->total_abs_sum, t);
+        }
+    }
+}
+static_assert(kStatSlots == 1024, "the fold kernel is one CTA with one thread per slot");
 }  // namespace
 
 int plan_tensor_count(const void* plan)
@@ -303,7 +339,7 @@ extern "C" int cast_adams_step(float* w, float* m, float* v, const cast_bf16* g,
 {
     int rc;
     if ((rc = check_nm_flags(N, M, flags, flip_count)) != CAST_OK) return rc;
-    if (flags & CAST_F_MASK_STATS) return CAST_ERR_NULL;      // this signature has no accumulator: cast_adams_step_stats
+    if (flags & CAST_F_MASK_STATS) return CAST_ERR_PLAN;      // the statistics epilogue needs a plan (cast_plan_step_stats)
     StepConsts c;
     if ((rc = make_step_consts(lr, beta1, beta2, eps, l1_coeff, step, total_steps, N, flags, &c)) != CAST_OK) return rc;
     if (!w || !m || !v || !g || !w_fwd_bf16 || !meta) return CAST_ERR_NULL;
@@ -357,16 +393,10 @@ int check_meta_ref(const cast_tensor_t& t)
 extern "C" int cast_adams_step_ex(const cast_tensor_t* t, int N, int M, const cast_hyper_t* h,
                                   unsigned long long* flip_count, cast_stream_t stream)
 {
-    return cast_adams_step_stats(t, N, M, h, flip_count, nullptr, stream);
-}
-
-extern "C" int cast_adams_step_stats(const cast_tensor_t* t, int N, int M, const cast_hyper_t* h,
-                                     unsigned long long* flip_count, cast_mask_stats_t* stats, cast_stream_t stream)
-{
     if (!t || !h) return CAST_ERR_NULL;
     int rc;
     if ((rc = check_nm_flags(N, M, h->flags, flip_count)) != CAST_OK) return rc;
-    if ((rc = check_stats_ptr(h->flags, stats)) != CAST_OK) return rc;
+    if (h->flags & CAST_F_MASK_STATS) return CAST_ERR_PLAN;     // the statistics epilogue needs a plan (cast_plan_step_stats)
     StepConsts c;
     if ((rc = make_step_consts(h->lr, h->beta1, h->beta2, h->eps, h->l1_coeff, h->step, h->total_steps, N, h->flags, &c)) != CAST_OK) return rc;
     if (!t->w || !t->m || !t->v || !t->g || !t->w_fwd || !t->meta) return CAST_ERR_NULL;
@@ -379,7 +409,7 @@ extern "C" int cast_adams_step_stats(const cast_tensor_t* t, int N, int M, const
     if ((rc = check_meta_ref(*t)) != CAST_OK) return rc;
     const TensorDesc d = make_desc(t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, t->scale_groups, t->rows, t->cols,
                                    t->scale_grad, t->meta_ref);
-    return launch_single(d, M, c, flip_count, (cudaStream_t)stream, (h->flags & CAST_F_MASK_STATS) ? stats : nullptr);
+    return launch_single(d, M, c, flip_count, (cudaStream_t)stream);
 }
 
 extern "C" int cast_plan_create(const cast_tensor_t* tensors, int n_tensors, int N, int M, void** plan_out)
@@ -395,30 +425,41 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
     if (!tensors) return CAST_ERR_NULL;
     if (n_tensors < 1) return CAST_ERR_SHAPE;
     int rc;
-    if (plan_flags & ~(uint32_t)CAST_F_EMIT_COMPRESSED) return CAST_ERR_HYPER;
+    if (plan_flags & ~(uint32_t)(CAST_F_EMIT_COMPRESSED | CAST_F_MASK_STATS)) return CAST_ERR_HYPER;
+    const uint32_t fwd_flags = plan_flags & CAST_F_EMIT_COMPRESSED;
     // the encoding flag is a per-step choice; here only N:M itself (and the compressed form's M <= 8) is checked
-    if ((rc = check_nm_flags(N, M, CAST_F_META_BITMASK | plan_flags, nullptr)) != CAST_OK) return rc;
+    if ((rc = check_nm_flags(N, M, CAST_F_META_BITMASK | fwd_flags, nullptr)) != CAST_OK) return rc;
 
     for (int i = 0; i < n_tensors; ++i) {
         const cast_tensor_t& t = tensors[i];
         if (!t.w || !t.m || !t.v || !t.g || !t.w_fwd || !t.meta) return CAST_ERR_NULL;
         if ((rc = check_shape(t.rows, t.cols, M, t.scale != nullptr, t.scale_groups)) != CAST_OK) return rc;
         if ((rc = check_pointers(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols,
-                                 fwd_elems_of(t.rows, t.cols, N, M, plan_flags))) != CAST_OK) return rc;
+                                 fwd_elems_of(t.rows, t.cols, N, M, fwd_flags))) != CAST_OK) return rc;
     }
     for (int i = 0; i < n_tensors; ++i) {
         const cast_tensor_t& t = tensors[i];
         const void* ptrs[7] = {t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale};
         if ((rc = check_device_memory(ptrs, 7)) != CAST_OK) return rc;
-        if ((rc = check_tensor_scale_grad(t, N, M, plan_flags)) != CAST_OK) return rc;
+        if ((rc = check_tensor_scale_grad(t, N, M, fwd_flags)) != CAST_OK) return rc;
         if ((rc = check_meta_ref(t)) != CAST_OK) return rc;
     }
 
     Plan* p = new (std::nothrow) Plan;
     if (!p) return CAST_ERR_PLAN;
     p->magic = 0;
+    p->stat_slots = nullptr;
     cudaError_t e = cudaGetDevice(&p->device);
-    if (e != cudaSuccess) { delete p; return cuda_failed(e); }
+    if (e == cudaSuccess && (plan_flags & CAST_F_MASK_STATS)) {
+        e = cudaMalloc(&p->stat_slots, sizeof(MaskStats) * kStatSlots);
+        if (e == cudaSuccess) e = cudaMemset(p->stat_slots, 0, sizeof(MaskStats) * kStatSlots);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();      // the slots are zero before any stream can use them
+    }
+    if (e != cudaSuccess) {
+        if (p->stat_slots) cudaFree(p->stat_slots);
+        delete p;
+        return cuda_failed(e);
+    }
     // cut the list into launches: at most kMaxLaunchTensors matrices and kMaxTiles tiles each
     try {
         int i = 0;
@@ -442,6 +483,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
             fill_hints(&mp);
         }
     } catch (const std::bad_alloc&) {
+        if (p->stat_slots) cudaFree(p->stat_slots);
         delete p;
         return CAST_ERR_PLAN;
     }
@@ -466,7 +508,9 @@ extern "C" int cast_plan_step_stats(void* plan, const cast_hyper_t* h, unsigned 
     int rc;
     if ((rc = check_nm_flags(p->N, p->M, h->flags, flip_count)) != CAST_OK) return rc;
     if ((rc = check_stats_ptr(h->flags, stats)) != CAST_OK) return rc;
-    if ((h->flags & CAST_F_EMIT_COMPRESSED) != p->plan_flags) return CAST_ERR_PLAN;
+    if ((h->flags & CAST_F_EMIT_COMPRESSED) != (p->plan_flags & CAST_F_EMIT_COMPRESSED)) return CAST_ERR_PLAN;
+    const bool with_stats = (h->flags & CAST_F_MASK_STATS) != 0;
+    if (with_stats && !p->stat_slots) return CAST_ERR_PLAN;      // the plan was not created for statistics
     StepConsts c;
     if ((rc = make_step_consts(h->lr, h->beta1, h->beta2, h->eps, h->l1_coeff, h->step, h->total_steps,
                                p->N, h->flags, &c)) != CAST_OK) return rc;
@@ -478,8 +522,16 @@ extern "C" int cast_plan_step_stats(void* plan, const cast_hyper_t* h, unsigned 
         if ((rc = check_device_memory(fp, 1)) != CAST_OK) return rc;
     }
     for (const MultiParams& mp : p->launches)
-        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream,
-                               (h->flags & CAST_F_MASK_STATS) ? stats : nullptr)) != CAST_OK) return rc;
+        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream, with_stats ? p->stat_slots : nullptr)) != CAST_OK) {
+            // what the launches so far left in the slots must not reach a later step
+            if (with_stats) (void)cudaMemsetAsync(p->stat_slots, 0, sizeof(MaskStats) * kStatSlots, (cudaStream_t)stream);
+            return rc;
+        }
+    if (with_stats) {
+        fold_stat_slots_kernel<<<1, kStatSlots, 0, (cudaStream_t)stream>>>(p->stat_slots, reinterpret_cast<MaskStats*>(stats));
+        CAST_CUDA_TRY(cudaGetLastError());
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+    }
     return CAST_OK;
 }
 
@@ -488,8 +540,13 @@ extern "C" int cast_plan_destroy(void* plan)
     Plan* p = (Plan*)plan;
     if (!p || p->magic != kPlanMagic) return CAST_ERR_PLAN;
     p->magic = 0;
+    int rc = CAST_OK;
+    if (p->stat_slots) {
+        const cudaError_t e = cudaFree(p->stat_slots);
+        if (e != cudaSuccess) rc = cuda_failed(e);
+    }
     delete p;
-    return CAST_OK;
+    return rc;
 }
 
 extern "C" const char* cast_strerror(int status)

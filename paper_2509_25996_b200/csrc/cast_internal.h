@@ -66,13 +66,12 @@ struct StepLaunch {
     const MultiParams* multi;
     const StepConsts* c;
     unsigned long long* flip_count;
-    MaskStats* stats;
+    MaskStats* stats;                 // the plan's kStatSlots accumulators, or nullptr
     cudaStream_t stream;
 };
-int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count,
-                  cudaStream_t stream, cast_mask_stats_t* stats = nullptr);
+int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
-                 cast_mask_stats_t* stats = nullptr);
+                 MaskStats* stat_slots = nullptr);
 
 // Fill the tile-to-matrix hint table (kHintEntries entries) of a launch whose tile_start[0..n_tensors] is set:
 // hint[b] = the matrix that holds tile b << *hint_shift.

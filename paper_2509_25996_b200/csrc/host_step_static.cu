@@ -72,7 +72,7 @@ extern "C" int cast_host_step_static(float* w, float* m, float* v, const cast_bf
 {
     int rc;
     if ((rc = check_nm_flags(N, M, flags, flip_count)) != CAST_OK) return rc;
-    if (flags & CAST_F_MASK_STATS) return CAST_ERR_NULL;      // no accumulator in this signature
+    if (flags & CAST_F_MASK_STATS) return CAST_ERR_PLAN;      // the statistics epilogue needs a plan
     StepConsts k;
     if ((rc = make_step_consts(lr, beta1, beta2, eps, l1_coeff, step, total_steps, N, flags, &k)) != CAST_OK) return rc;
     if (!w || !m || !v || !g || !w_fwd_bf16 || !meta) return CAST_ERR_NULL;

@@ -28,7 +28,8 @@ int launch_word(const StepLaunch& a)
 {
     if (a.single) {
         // one CTA per tile: the hardware scheduler hands tiles out in address order
-        adams_nm_kernel<kM, F, kTwoFour><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.stats);
+        if constexpr (kStats) return CAST_ERR_NM;      // the statistics epilogue exists for plans only
+        else adams_nm_kernel<kM, F, kTwoFour><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.stats);
     } else {
         adams_nm_multi_kernel<kM, F, kTwoFour><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(
             *a.multi, *a.c, a.flip_count, a.stats);

@@ -55,7 +55,7 @@ class DeviceModelState:
         CAST_F_GRAD_OF_SCALED) and Adam moments for its scale; scale_step() then trains the scales.
         reference_masks: every matrix gets a second metadata buffer (zeros until the caller fills it, e.g. with
         the initial mask), against which steps that carry CAST_F_MASK_STATS count ||M_t - M_ref||_0; the sums
-        land in self.stats."""
+        land in self.stats (the plan is created with CAST_F_MASK_STATS)."""
         self.device = torch.device(device)
         self.N, self.M = N, M
         self.compressed = compressed
@@ -83,7 +83,8 @@ class DeviceModelState:
         tensors = [B.make_tensor(s.w, s.m, s.v, s.g, s.w_fwd, s.meta, s.scale,
                                  1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad, s.meta_ref)
                    for s in self.mats]
-        rc, self.plan = B.cast_plan_create_ex(tensors, N, M, B.CAST_F_EMIT_COMPRESSED if compressed else 0)
+        rc, self.plan = B.cast_plan_create_ex(tensors, N, M, (B.CAST_F_EMIT_COMPRESSED if compressed else 0) |
+                                              (B.CAST_F_MASK_STATS if reference_masks else 0))
         B.check(rc)
 
     def step(self, hyper: Hyper, flags: int, stream=None) -> None:

@@ -33,20 +33,23 @@ def read_stats(buf):
 
 
 def step_with_stats(inp, N, M, h, flags, meta_in, meta_ref):
-    """One fused step through cast_adams_step_stats on guarded buffers; returns (outputs, statistics)."""
-    st = U.to_device(inp, DEV, meta_in)
+    """One fused step of a one-matrix plan on guarded buffers; returns (outputs, statistics)."""
+    st = U.to_device(inp, DEV, meta_in, inp.w.numel() * N // M if flags & B.CAST_F_EMIT_COMPRESSED else None)
     d_ref = None if meta_ref is None else torch.from_numpy(np.ascontiguousarray(meta_ref).view(np.int32).reshape(-1)).to(DEV)
     flips = torch.zeros(1, dtype=torch.int64, device=DEV) if flags & FL else None
     stats = torch.zeros(ctypes.sizeof(B.cast_mask_stats_t), dtype=torch.uint8, device=DEV)
     lr, b1, b2, eps, lam = h.as_f32()
     t = B.make_tensor(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale,
                       1 if st.scale is None else st.scale.shape[1], st.rows, st.cols, None, d_ref)
+    rc, plan = B.cast_plan_create_ex([t], N, M, ST | (flags & B.CAST_F_EMIT_COMPRESSED))
+    cast.check(rc)
     before = cast.cast_kernel_launch_count()
-    cast.check(cast.cast_adams_step_stats(t, N, M, B.make_hyper(lr, b1, b2, eps, lam, h.step, h.total_steps, flags), flips, stats,
-                                          torch.cuda.current_stream()))
+    hy = B.make_hyper(lr, b1, b2, eps, lam, h.step, h.total_steps, flags)
+    cast.check(cast.cast_plan_step_stats(plan, hy, flips, stats, torch.cuda.current_stream()))
     torch.cuda.synchronize()
-    assert cast.cast_kernel_launch_count() == before + 1          # the statistics cost no second launch
+    assert cast.cast_kernel_launch_count() == before + 2          # the step and the one-CTA fold of the partial sums
     assert st.all_intact()
+    cast.check(cast.cast_plan_destroy(plan))
     return U.device_outputs(st, flips), read_stats(stats)
 
 
@@ -123,7 +126,7 @@ def test_plan_step_with_statistics_accumulates_over_matrices():
     fused.step(h, RS | FL | DN | ST)
     plain.step(h, RS | FL | DN)
     torch.cuda.synchronize()
-    assert cast.cast_kernel_launch_count() == launches + 2
+    assert cast.cast_kernel_launch_count() == launches + 3       # two steps and one fold
     got = fused.read_stats()
     oh = Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
     want = dict(flips=0, kept_abs=0.0, total_abs=0.0)
@@ -144,19 +147,45 @@ def test_plan_step_with_statistics_accumulates_over_matrices():
     fused.close()
 
 
-def test_statistics_flag_needs_its_accumulator():
+def test_statistics_flag_needs_a_plan_made_for_it_and_an_accumulator():
     inp = workloads.gen_tensor_inputs(4, 64, seed=3, device="cpu", scale_mode="none")
     st = U.to_device(inp, DEV)
     before = cast.cast_kernel_launch_count()
     rc = cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, None, 1, 4, 64, 2, 4,
                               1e-4, 0.9, 0.95, 1e-8, 1e-3, 1, 10, RS | ST, None, None)
-    assert rc == B.CAST_ERR_NULL
+    assert rc == B.CAST_ERR_PLAN
     t = B.make_tensor(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, None, 1, 4, 64)
     hy = B.make_hyper(1e-4, 0.9, 0.95, 1e-8, 1e-3, 1, 10, RS | ST)
-    assert cast.cast_adams_step_stats(t, 2, 4, hy, None, None, None) == B.CAST_ERR_NULL
-    assert cast.cast_adams_step_ex(t, 2, 4, hy, None, None) == B.CAST_ERR_NULL
+    assert cast.cast_adams_step_ex(t, 2, 4, hy, None, None) == B.CAST_ERR_PLAN
     stats = torch.zeros(40, dtype=torch.uint8, device=DEV)
-    assert cast.cast_adams_step_stats(t, 2, 4, hy, None, stats[4:36], None) == B.CAST_ERR_ALIGN
+    rc, ordinary = B.cast_plan_create([t], 2, 4)
+    cast.check(rc)
+    assert cast.cast_plan_step_stats(ordinary, hy, None, stats[:32], None) == B.CAST_ERR_PLAN     # not created for statistics
+    assert cast.cast_plan_step(ordinary, hy, None, None) == B.CAST_ERR_NULL                        # no accumulator
+    cast.check(cast.cast_plan_destroy(ordinary))
+    rc, plan = B.cast_plan_create_ex([t], 2, 4, ST)
+    cast.check(rc)
+    assert cast.cast_plan_step_stats(plan, hy, None, None, None) == B.CAST_ERR_NULL
+    assert cast.cast_plan_step_stats(plan, hy, None, stats[4:36], None) == B.CAST_ERR_ALIGN
+    cast.check(cast.cast_plan_destroy(plan))
     bad_ref = B.make_tensor(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, None, 1, 4, 64, None, st.meta.view)
-    assert cast.cast_adams_step_stats(bad_ref, 2, 4, hy, None, stats[:32], None) == B.CAST_ERR_ALIAS
+    rc, none = B.cast_plan_create_ex([bad_ref], 2, 4, ST)
+    assert rc == B.CAST_ERR_ALIAS and none is None
     assert cast.cast_kernel_launch_count() == before
+
+
+def test_two_steps_of_one_plan_leave_no_partial_sums_behind():
+    """The partial accumulators of the plan are cleared by every step: a second step adds exactly its own sums."""
+    shapes = [(16, 512), (5, 96)]
+    st = DeviceModelState(shapes, 2, 4, seed=8, device=DEV, scale_mode="jitter", reference_masks=True)
+    h = RunHyper(total_steps=30000)
+    st.step(h, RS | ST)
+    first = st.read_stats()
+    st.stats.zero_()
+    h.step += 1
+    st.step(h, ST)                                    # stored mask, same weights' successors
+    second = st.read_stats()
+    mag = sum(float(m.w.double().abs().sum().item()) for m in st.mats)
+    assert second.total_abs_sum == pytest.approx(mag, rel=1e-12)
+    assert first.total_abs_sum != second.total_abs_sum
+    st.close()
