@@ -5,7 +5,7 @@ library loads on a machine without a driver (calls then return CAST_ERR_CUDA).
 
 Every .cu file becomes one object; csrc/step_inst.cu, which instantiates the step kernels,
 is compiled once per slice (group size M, 2:4 or general N:M, with or without the statistics
-epilogue) so that the few hundred instantiations compile in parallel.  Objects live in
+epilogue, literal or alternate reading of Eq. 8) so that the few hundred instantiations compile in parallel.  Objects live in
 paper_2509_25996_b200/_build/ and are rebuilt only when a source or header is newer.
 """
 from __future__ import annotations
@@ -32,8 +32,8 @@ NVCC_FLAGS = [
 ]
 LINK_FLAGS = ["--cudart", "static", "-shared", "-gencode", "arch=compute_100a,code=sm_100a"]
 
-# slices of the step kernels: (M, two_four, statistics); 2:4 exists for M = 4 only
-STEP_SLICES = [(m, tf, s) for m in (2, 4, 8, 16, 32) for tf in ((0, 1) if m == 4 else (0,)) for s in (0, 1)]
+# slices of the step kernels: (M, two_four, statistics, alternate reading of Eq. 8); 2:4 exists for M = 4 only
+STEP_SLICES = [(m, tf, s, v) for m in (2, 4, 8, 16, 32) for tf in ((0, 1) if m == 4 else (0,)) for s in (0, 1) for v in (0, 1)]
 
 
 def _nvcc() -> str:
@@ -58,9 +58,9 @@ def _jobs():
     for src in sources():
         base = os.path.splitext(os.path.basename(src))[0]
         if base == "step_inst":
-            for m, tf, s in STEP_SLICES:
-                jobs.append((os.path.join(OBJ_DIR, f"step_inst_m{m}_tf{tf}_s{s}.o"), src,
-                             [f"-DCAST_INST_M={m}", f"-DCAST_INST_TF={tf}", f"-DCAST_INST_STATS={s}"]))
+            for m, tf, s, v in STEP_SLICES:
+                jobs.append((os.path.join(OBJ_DIR, f"step_inst_m{m}_tf{tf}_s{s}_v{v}.o"), src,
+                             [f"-DCAST_INST_M={m}", f"-DCAST_INST_TF={tf}", f"-DCAST_INST_STATS={s}", f"-DCAST_INST_V={v}"]))
         else:
             jobs.append((os.path.join(OBJ_DIR, base + ".o"), src, []))
     return jobs

@@ -41,9 +41,9 @@ constexpr uint32_t kEmitCompressed = 1u << 5;
 constexpr uint32_t kGradOfScaled = 1u << 6;
 constexpr uint32_t kMaskStats = 1u << 7;
 
-// Every flag but kVKeptFromG is a template argument of the kernels; that one (the alternate reading of Eq. 8,
-// one select per parameter) is read from StepConsts at run time.
-constexpr uint32_t kCompileTimeFlags = kReselect | kCountFlips | kMetaBitmask | kEmitDense | kEmitCompressed |
+// Every flag is a template argument of the kernels (even the alternate reading of Eq. 8, one select per parameter,
+// cost 1.4 % of the headline step when it was read at run time).
+constexpr uint32_t kCompileTimeFlags = kReselect | kCountFlips | kMetaBitmask | kVKeptFromG | kEmitDense | kEmitCompressed |
                                        kGradOfScaled | kMaskStats;
 constexpr uint32_t kFlagWords = 256;   // compile-time flag words live in [0, kFlagWords)
 
@@ -360,6 +360,7 @@ struct StepCfg {
     static constexpr bool compressed = (F & kEmitCompressed) != 0;
     static constexpr bool of_scaled = (F & kGradOfScaled) != 0;
     static constexpr bool stats = (F & kMaskStats) != 0;
+    static constexpr bool v_from_g = (F & kVKeptFromG) != 0;
     static constexpr bool network = TF && reselect;               // kept set from the 2:4 comparison network
     static constexpr bool need_prev = !reselect || count_flips;   // the stored metadata is read
 };
@@ -397,7 +398,9 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
         else u.meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);
         if constexpr (Cfg::count_flips) {
             if constexpr (Cfg::bitmask) sums.flips = (uint32_t)__popc(keep ^ u.prev_byte);
-            else if (u.meta_byte != u.prev_byte)      // equal index bytes are equal masks: most units, most steps
+            // equal index bytes are equal masks (most units, most steps): the decode is skipped there -- except in the
+            // kernels that also carry the scale gradient, where the branch costs registers (spills; measured slower)
+            else if (Cfg::of_scaled || u.meta_byte != u.prev_byte)
                 sums.flips = (uint32_t)__popc(keep_from_meta_byte(u.meta_byte, false) ^ keep_from_meta_byte(u.prev_byte, false));
         }
     } else {
@@ -418,7 +421,6 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
     }
 
     const uint32_t gw[4] = {u.g.x, u.g.y, u.g.z, u.g.w};
-    const bool v_from_g = (c.flags & kVKeptFromG) != 0;
     const int sign_hi = __double2hiint(c.c_sign), sign_lo = __double2loint(c.c_sign);
     // With kGradOfScaled the gradient is taken with respect to W_scale = Diag(A) W (Eq. 12): the chain rule
     // gives dL/dW = A g (formed exactly in fp64) and dL/dA = sum of g W over the row segment, whose part
@@ -432,7 +434,7 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
         if constexpr (Cfg::of_scaled) gw_sum = fmaf(g32, u.w[i], gw_sum);
         // first moment, stored undecayed (Alg. 1)
         const double mu = fma(c.beta1, (double)u.m[i], omb1_g * (double)g32);
-        if constexpr (Cfg::of_scaled) g32 *= a;      // only the alternate reading of v below still uses g itself
+        if constexpr (Cfg::of_scaled && Cfg::v_from_g) g32 *= a;      // the alternate reading of v below uses dL/dW itself
         const float mu_f = (float)mu;
         u.m[i] = mu_f;
         // proportional L1 decay outside the kept set (Eq. 7): alpha lambda Sign(w), Sign(+-0) = 0
@@ -441,7 +443,7 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
                                                  w_zero ? 0 : sign_lo);
         const float mu_t = kept[i] ? mu_f : (float)fma(c.c_mu, mu, sgn_term);
         // second moment from the decayed first moment (Eq. 8)
-        const float src = (v_from_g && kept[i]) ? g32 : mu_t;
+        const float src = (Cfg::v_from_g && kept[i]) ? g32 : mu_t;
         const float vn = fmaf(c.beta2, u.v[i], (c.omb2 * src) * src);
         u.v[i] = vn;
         // bias-corrected update (Alg. 1): w - (lr / bc1) mu~ / (sqrt(v / bc2) + eps)

@@ -163,16 +163,19 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
 // ---------------------------------------------------------------------------------------------
 // launches
 
-// The kernels are instantiated in step_inst.cu, compiled once per (M, two_four, statistics) with every valid
-// compile-time flag word of that slice; each such object exports one launcher.
-#define CAST_DECLARE_STEP_LAUNCHER(M, TF, S) int launch_step_m##M##_tf##TF##_s##S(uint32_t flag_word, const StepLaunch& a);
-CAST_DECLARE_STEP_LAUNCHER(2, 0, 0) CAST_DECLARE_STEP_LAUNCHER(2, 0, 1)
-CAST_DECLARE_STEP_LAUNCHER(4, 0, 0) CAST_DECLARE_STEP_LAUNCHER(4, 0, 1)
-CAST_DECLARE_STEP_LAUNCHER(4, 1, 0) CAST_DECLARE_STEP_LAUNCHER(4, 1, 1)
-CAST_DECLARE_STEP_LAUNCHER(8, 0, 0) CAST_DECLARE_STEP_LAUNCHER(8, 0, 1)
-CAST_DECLARE_STEP_LAUNCHER(16, 0, 0) CAST_DECLARE_STEP_LAUNCHER(16, 0, 1)
-CAST_DECLARE_STEP_LAUNCHER(32, 0, 0) CAST_DECLARE_STEP_LAUNCHER(32, 0, 1)
-#undef CAST_DECLARE_STEP_LAUNCHER
+// The kernels are instantiated in step_inst.cu, compiled once per slice (M, two_four, statistics, reading of
+// Eq. 8) with every valid compile-time flag word of that slice; each such object exports one launcher.
+using StepLauncher = int (*)(uint32_t flag_word, const StepLaunch& a);
+#define CAST_SLICE(M, TF, S, V) int launch_step_m##M##_tf##TF##_s##S##_v##V(uint32_t flag_word, const StepLaunch& a);
+#define CAST_SLICES_OF(M, TF) CAST_SLICE(M, TF, 0, 0) CAST_SLICE(M, TF, 0, 1) CAST_SLICE(M, TF, 1, 0) CAST_SLICE(M, TF, 1, 1)
+CAST_SLICES_OF(2, 0) CAST_SLICES_OF(4, 0) CAST_SLICES_OF(4, 1) CAST_SLICES_OF(8, 0) CAST_SLICES_OF(16, 0) CAST_SLICES_OF(32, 0)
+#undef CAST_SLICE
+#define CAST_SLICE(M, TF, S, V) launch_step_m##M##_tf##TF##_s##S##_v##V,
+// indexed [group size: 2, 4, 4 as 2:4, 8, 16, 32][statistics * 2 + alternate reading]
+static const StepLauncher kStepLaunchers[6][4] = {
+    {CAST_SLICES_OF(2, 0)}, {CAST_SLICES_OF(4, 0)}, {CAST_SLICES_OF(4, 1)}, {CAST_SLICES_OF(8, 0)}, {CAST_SLICES_OF(16, 0)}, {CAST_SLICES_OF(32, 0)}};
+#undef CAST_SLICE
+#undef CAST_SLICES_OF
 
 uint32_t kernel_flag_word(uint32_t flags)
 {
@@ -189,15 +192,16 @@ int launch_step(const StepLaunch& a, int M)
     if (!step_kernel_exists(M, two_four, f)) return CAST_ERR_NM;
     if (a.single ? tiles_of(*a.single) == 0 : a.multi->tile_start[a.multi->n_tensors] == 0) return CAST_OK;
     if (a.single && tiles_of(*a.single) > kMaxTiles) return CAST_ERR_SHAPE;
-    int rc = CAST_ERR_NM;
+    int row = -1;
     switch (M) {
-        case 2:  rc = st ? launch_step_m2_tf0_s1(f, a) : launch_step_m2_tf0_s0(f, a); break;
-        case 4:  rc = two_four ? (st ? launch_step_m4_tf1_s1(f, a) : launch_step_m4_tf1_s0(f, a))
-                               : (st ? launch_step_m4_tf0_s1(f, a) : launch_step_m4_tf0_s0(f, a)); break;
-        case 8:  rc = st ? launch_step_m8_tf0_s1(f, a) : launch_step_m8_tf0_s0(f, a); break;
-        case 16: rc = st ? launch_step_m16_tf0_s1(f, a) : launch_step_m16_tf0_s0(f, a); break;
-        case 32: rc = st ? launch_step_m32_tf0_s1(f, a) : launch_step_m32_tf0_s0(f, a); break;
+        case 2:  row = 0; break;
+        case 4:  row = two_four ? 2 : 1; break;
+        case 8:  row = 3; break;
+        case 16: row = 4; break;
+        case 32: row = 5; break;
     }
+    if (row < 0) return CAST_ERR_NM;
+    const int rc = kStepLaunchers[row][(st ? 2 : 0) + ((f & kVKeptFromG) ? 1 : 0)](f, a);
     if (rc == CAST_OK) g_launches.fetch_add(1, std::memory_order_relaxed);
     return rc;
 }

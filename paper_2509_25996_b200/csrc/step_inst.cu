@@ -1,7 +1,8 @@
 // Instantiations of the AdamS step kernels.  This file is compiled once per slice (group size M, 2:4 or not,
-// with or without the statistics epilogue; see build_ext.py), each time with every valid compile-time flag word
-// of the slice, so that no combination of flags is decided inside a kernel and the compilation runs in parallel.
-// Every object exports one function, launch_step_m<M>_tf<0|1>_s<0|1>(flag_word, launch).
+// with or without the statistics epilogue, literal or alternate reading of Eq. 8; see build_ext.py), each time with
+// every valid compile-time flag word of the slice, so that no combination of flags is decided inside a kernel and
+// the compilation runs in parallel.  Every object exports one function,
+// launch_step_m<M>_tf<0|1>_s<0|1>_v<0|1>(flag_word, launch).
 #include <utility>
 
 #include "cast_internal.h"
@@ -10,11 +11,12 @@
 #define CAST_INST_M 4
 #define CAST_INST_TF 1
 #define CAST_INST_STATS 0
+#define CAST_INST_V 0
 #endif
 
-#define CAST_CAT_(a, b, c, d, e, f) a##b##c##d##e##f
-#define CAST_CAT(a, b, c, d, e, f) CAST_CAT_(a, b, c, d, e, f)
-#define CAST_INST_FN CAST_CAT(launch_step_m, CAST_INST_M, _tf, CAST_INST_TF, _s, CAST_INST_STATS)
+#define CAST_CAT_(a, b, c, d, e, f, g, h) a##b##c##d##e##f##g##h
+#define CAST_CAT(a, b, c, d, e, f, g, h) CAST_CAT_(a, b, c, d, e, f, g, h)
+#define CAST_INST_FN CAST_CAT(launch_step_m, CAST_INST_M, _tf, CAST_INST_TF, _s, CAST_INST_STATS, _v, CAST_INST_V)
 
 namespace cast {
 namespace {
@@ -22,6 +24,7 @@ namespace {
 constexpr int kM = CAST_INST_M;
 constexpr bool kTwoFour = CAST_INST_TF != 0;
 constexpr bool kStats = CAST_INST_STATS != 0;
+constexpr bool kAltV = CAST_INST_V != 0;
 
 template <uint32_t F>
 int launch_word(const StepLaunch& a)
@@ -42,7 +45,7 @@ int launch_word(const StepLaunch& a)
 template <uint32_t F>
 bool try_word(uint32_t flag_word, const StepLaunch& a, int& rc)
 {
-    if constexpr (((F & kMaskStats) != 0) == kStats && step_kernel_exists(kM, kTwoFour, F)) {
+    if constexpr (((F & kMaskStats) != 0) == kStats && ((F & kVKeptFromG) != 0) == kAltV && step_kernel_exists(kM, kTwoFour, F)) {
         if (flag_word == F) {
             rc = launch_word<F>(a);
             return true;
