@@ -29,11 +29,13 @@ BYTES_PER_PARAM = 28.125          # 14 read (w, m, v fp32 + g bf16) + 14 written
 BYTES_PER_PARAM_FLIPS = 28.25     # + 1/8 previous metadata read
 NOMINAL_HBM_GBS = 8000.0          # the nominal peak the target fraction is quoted against
 FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
-# dram__bytes_read.sum + dram__bytes_write.sum per parameter of adams_nm_multi_kernel<4, 1>, from the ncu
-# capture of one LLaMA2-7B layer (202,375,168 parameters) summarised under profiles/; every byte is touched
-# once, so the traffic of a launch is this figure times its parameter count.  Set to None when the kernel
-# changes until the counters are taken again.
-NCU_DRAM_BYTES_PER_PARAM = 27.863
+# dram__bytes_read.sum + dram__bytes_write.sum per parameter of the headline kernel, from the ncu capture of one
+# LLaMA2-7B layer (202,375,168 parameters) summarised under profiles/ (which names the kernel the counters were
+# taken on); every byte is touched once, so the traffic of a launch is this figure times its parameter count.
+# None until the counters have been taken on the kernel as it stands; reported only for the workload and
+# configuration they were taken on (the 2:4 headline over LLaMA2-7B shapes).
+NCU_DRAM_BYTES_PER_PARAM = None
+NCU_KERNEL = "adams_nm_multi_kernel<4, 1u, true>"
 
 METRIC = "AdamS 2:4 step params/s"
 
@@ -64,6 +66,10 @@ def parse_args():
     p.add_argument("--op", choices=["step", "mask_stats", "prune_fold", "kd_loss"], default="step",
                    help="step: the AdamS step (the headline metric); mask_stats: the App. C statistics pass; prune_fold: the "
                         "final pruning of Alg. 2; kd_loss: the distillation loss of Eq. 13 with its gradient")
+    p.add_argument("--configs", choices=["all", "none"], default="all",
+                   help="all (default, 1 GPU, headline workload only): after the headline line's own measurements, also time the "
+                        "other listed workloads (one matrix, the d=768 decoder, the streamed 13B shapes, 4:8 and 1:4 with the "
+                        "L1-coefficient sweep and flip counts) and report them in the `configs` array of the same JSON line")
     p.add_argument("--tokens", type=int, default=16384, help="kd_loss: tokens per step")
     p.add_argument("--vocab", type=int, default=32000, help="kd_loss: vocabulary size (LLaMA2: 32000)")
     return p.parse_args()
@@ -214,6 +220,301 @@ def reference_arm(args):
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+def _gbs(params, bytes_per_param, ms):
+    return params * bytes_per_param / (ms * 1e-3) / 1e9
+
+
+def _rows(mat, r0, n, fields):
+    """Host copies of `n` rows of some buffers of one matrix (numpy; bf16 as raw bits; metadata as uint32)."""
+    import numpy as np
+    from paper_2509_25996_b200 import workloads
+    out = {}
+    for k in fields:
+        t = getattr(mat, k)[r0:r0 + n]
+        if k in ("g", "w_fwd"):
+            out[k] = workloads.bf16_bits(t)
+        elif k == "meta":
+            out[k] = t.cpu().numpy().view(np.uint32)
+        else:
+            out[k] = t.cpu().numpy()
+    return out
+
+
+def _rows_match_oracle(before, after, N, M, hyper, flags, cols):
+    """One oracle step (fp64 build) from `before` compared with `after` at the stated tolerances."""
+    import numpy as np
+    from oracle import adams_oracle as orc
+    oh = orc.Hyper(lr=hyper.lr, beta1=hyper.beta1, beta2=hyper.beta2, eps=hyper.eps, l1_coeff=hyper.l1_coeff,
+                   step=hyper.step, total_steps=hyper.total_steps)
+    ref = orc.adams_step(before["w"], before["m"], before["v"], before["g"], before.get("scale"), N, M, oh, flags, before.get("meta"))
+    ok = True
+    for k in ("w", "m", "v"):
+        r = ref[k].astype(np.float64).reshape(-1)
+        g_ = after[k].astype(np.float64).reshape(-1)
+        ok &= bool(np.all(np.abs(g_ - r) <= np.maximum(1e-6 * np.abs(r), 1e-9)))
+    ok &= bool(np.array_equal(ref["meta"].reshape(-1), after["meta"].reshape(-1)))
+    d = np.abs((ref["w_fwd"].reshape(-1).astype(np.int32) & 0x7FFF) - (after["w_fwd"].reshape(-1).astype(np.int32) & 0x7FFF))
+    ok &= bool(d.max() <= 1)
+    return ok, int(ref["flips"])
+
+
+def extra_configs(args, dev, stream, state_7b, sampler, peak):
+    """The listed workloads other than the headline, timed in the same process (1 GPU): the 4:8 / 1:4 sweep of the L1
+    coefficient with flip counts on the LLaMA2-7B set, the streamed LLaMA2-13B shapes, the one-matrix case with its
+    launch floors, and the d = 768 decoder.  `state_7b` is the headline's resident state (reused, then freed here).
+    Every entry carries a sampled parity check against the CPU oracle."""
+    import gc
+    import numpy as np
+    import torch
+    import paper_2509_25996_b200 as cast
+    from paper_2509_25996_b200 import binding as B
+    from paper_2509_25996_b200 import workloads
+    from paper_2509_25996_b200.runner import DeviceModelState, StreamedModelState, Hyper
+    from oracle import adams_oracle as orc
+
+    out = []
+    RS, BM, FL = B.CAST_F_RESELECT, B.CAST_F_META_BITMASK, B.CAST_F_COUNT_FLIPS
+    sample_rows = 8
+
+    def entry(config, wl, nm, ms, bpp, t0, t1, **more):
+        gbs = _gbs(wl.n_params, bpp, ms)
+        e = {"config": config, "workload": wl.name, "nm": nm, "params": wl.n_params, "matrices": len(wl.shapes),
+             "ms_per_step": ms, "value": wl.n_params / (ms * 1e-3), "unit": "params/s", "bytes_per_param": bpp,
+             "hbm_gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8tbs": gbs / NOMINAL_HBM_GBS,
+             "clocks": sampler.summary(t0, t1) if sampler is not None else None}
+        e.update(more)
+        return e
+
+    def timed(fn, steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize(dev)
+        a.record(stream)
+        for _ in range(steps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize(dev)
+        return a.elapsed_time(b) / steps
+
+    # ---- config 5: the 7B set under 4:8 and 1:4, L1 coefficient swept, flips per step (App. C: r_t = flips / parameters)
+    wl7 = workloads.workload("llama2_7b")
+    picks = sorted({0, len(wl7.shapes) // 2, len(wl7.shapes) - 1})
+    for N, M in ((4, 8), (1, 4)):
+        state_7b.set_nm(N, M)
+        for lam in (0.0, 1e-4, 1e-3, 1e-2):
+            t0 = time.time()
+            state_7b.reset()
+            h = Hyper(l1_coeff=lam, step=1000, total_steps=wl7.total_steps)
+            flags = RS | BM | FL
+            state_7b.step(h, flags, stream)                        # establishes M_1 (there is no earlier mask)
+            h.step += 1
+            times, flips, parity_ok = [], [], True
+            for k in range(2):                                     # two consecutive iterations, a fresh gradient each
+                state_7b.fresh_gradients(h.step)
+                before = {t: _rows(state_7b.mats[t], 0, sample_rows, ("w", "m", "v", "g", "scale", "meta")) for t in picks} if k == 0 else {}
+                state_7b.flips.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+                state_7b.step(h, flags, stream)
+                b.record(stream)
+                torch.cuda.synchronize(dev)
+                times.append(a.elapsed_time(b))
+                flips.append(int(state_7b.flips.item()))
+                for t, bef in before.items():
+                    aft = _rows(state_7b.mats[t], 0, sample_rows, ("w", "m", "v", "w_fwd", "meta"))
+                    ok, _ = _rows_match_oracle(bef, aft, N, M, h, orc.F_RESELECT | orc.F_META_BITMASK | orc.F_COUNT_FLIPS,
+                                               state_7b.mats[t].cols)
+                    parity_ok &= ok
+                h.step += 1
+            ms = sum(times) / len(times)
+            out.append(entry(5, wl7, f"{N}:{M}", ms, BYTES_PER_PARAM_FLIPS, t0, time.time(), l1_coeff=lam, steps=len(times),
+                             ms_each_step=times, flips_per_step=flips, flip_rate_r_t=[f / wl7.n_params for f in flips],
+                             l2="inputs far larger than L2, no flush",
+                             note="state drawn afresh per (N:M, lambda); step 1000 establishes the mask, steps 1001 and 1002 "
+                                  "(fresh seeded gradients) are timed one by one and counted",
+                             parity={"ok": bool(parity_ok), "sample": f"first {sample_rows} rows of matrices {picks} at step 1001, "
+                                                                      "incl. metadata against the stored previous mask"}))
+    state_7b.close()
+    del state_7b
+    gc.collect()
+    torch.cuda.empty_cache()
+
+    # ---- config 4: LLaMA2-13B shapes, 40 per-layer calls on 2 streams over 10 resident layer slots
+    wl13 = workloads.workload("llama2_13b")
+    n_layers = len(wl13.shapes) // wl13.layer_matrices
+    st = StreamedModelState(wl13.shapes[:wl13.layer_matrices], n_layers, wl13.resident_layers, 2, 2, 4, seed=args.seed, device=dev,
+                            scale_mode="ones")
+    h = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl13.total_steps)
+    mats0 = st.slots[0].mats
+    picks13 = (0, 4, 6)
+    before = {t: _rows(mats0[t], 0, sample_rows, ("w", "m", "v", "g", "scale")) for t in picks13}
+    after = {}
+
+    def grab(layer, slot, side):
+        if layer == 0:
+            with torch.cuda.stream(side):                          # after slot 0's first visit, before its second
+                for t in picks13:
+                    after[t] = {k: getattr(mats0[t], k)[:sample_rows].clone() for k in ("w", "m", "v", "w_fwd", "meta")}
+
+    st.step(h, RS, stream, after_layer=grab)
+    torch.cuda.synchronize(dev)
+    parity_ok = True
+    for t in picks13:
+        aft = {k: (workloads.bf16_bits(v) if k == "w_fwd" else v.cpu().numpy().view(np.uint32) if k == "meta" else v.cpu().numpy())
+               for k, v in after[t].items()}
+        ok, _ = _rows_match_oracle(before[t], aft, 2, 4, h, orc.F_RESELECT, mats0[t].cols)
+        parity_ok &= ok
+    h.step += 1
+
+    def pass13():
+        st.step(h, RS, stream)
+        h.step += 1
+
+    for _ in range(3):
+        pass13()
+    t0 = time.time()
+    launches0 = cast.cast_kernel_launch_count()
+    ms = timed(pass13, 20)
+    out.append(entry(4, wl13, "2:4", ms, BYTES_PER_PARAM, t0, time.time(), steps=20,
+                     launches_per_step=(cast.cast_kernel_launch_count() - launches0) // 20, resident_layers=wl13.resident_layers,
+                     streams=2, l2="inputs far larger than L2, no flush", traffic=None,
+                     parity={"ok": bool(parity_ok), "sample": f"first {sample_rows} rows of matrices {list(picks13)} of slot 0 after its "
+                                                              "first visit, copied out on the slot's stream before the second"}))
+    st.close()
+    del st, mats0, after
+    gc.collect()
+    torch.cuda.empty_cache()
+
+    # ---- config 2: the d = 768 decoder, 72 matrices in one launch
+    wl2 = workloads.workload("decoder_d768_12l")
+    s2 = DeviceModelState(wl2.shapes, 2, 4, seed=args.seed, device=dev, scale_mode="ones")
+    h = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl2.total_steps)
+    picks2 = sorted({0, len(wl2.shapes) // 2, len(wl2.shapes) - 1})
+    before = {t: _rows(s2.mats[t], 0, sample_rows, ("w", "m", "v", "g", "scale")) for t in picks2}
+    s2.step(h, RS, stream)
+    torch.cuda.synchronize(dev)
+    parity_ok = True
+    for t in picks2:
+        ok, _ = _rows_match_oracle(before[t], _rows(s2.mats[t], 0, sample_rows, ("w", "m", "v", "w_fwd", "meta")), 2, 4, h,
+                                   orc.F_RESELECT, s2.mats[t].cols)
+        parity_ok &= ok
+    h.step += 1
+
+    def step2():
+        s2.step(h, RS, stream)
+        h.step += 1
+
+    for _ in range(5):
+        step2()
+    t0 = time.time()
+    ms = timed(step2, 200)
+    out.append(entry(2, wl2, "2:4", ms, BYTES_PER_PARAM, t0, time.time(), steps=200, launches_per_step=1,
+                     l2="1.37 GB of state per step, far larger than L2, no flush",
+                     parity={"ok": bool(parity_ok), "sample": f"first {sample_rows} rows of matrices {picks2} after the first step"}))
+    s2.close()
+    del s2
+
+    # ---- config 1: one 3072 x 768 matrix (38 MB of state: fits the L2), cold and warm, with the launch floors beside it
+    wl1 = workloads.workload("opt125m_fc2")
+    rows, cols = wl1.shapes[0]
+    s1 = DeviceModelState(wl1.shapes, 2, 4, seed=args.seed, device=dev, scale_mode="ones")
+    m1 = s1.mats[0]
+    h = Hyper(l1_coeff=args.l1_coeff, step=1000, total_steps=wl1.total_steps)
+    before = _rows(m1, 0, sample_rows, ("w", "m", "v", "g", "scale"))
+    s1.step(h, RS, stream)
+    torch.cuda.synchronize(dev)
+    parity_ok, _ = _rows_match_oracle(before, _rows(m1, 0, sample_rows, ("w", "m", "v", "w_fwd", "meta")), 2, 4, h, orc.F_RESELECT, cols)
+    h.step += 1
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    tiles = (rows * cols + 1023) // 1024
+
+    def single_step():
+        cast.check(cast.cast_adams_step(m1.w, m1.m, m1.v, m1.g, m1.w_fwd, m1.meta, m1.scale, m1.scale.shape[1], rows, cols, 2, 4,
+                                        h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps, RS, None, stream))
+
+    def plan_step():
+        s1.step(h, RS, stream)
+
+    def cold(fn, n=50):
+        """Median and mean device time of fn() with the L2 flushed by a 512 MB write before each call."""
+        pairs = []
+        for _ in range(n):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            fn()
+            b.record(stream)
+            pairs.append((a, b))
+        torch.cuda.synchronize(dev)
+        ts = [a.elapsed_time(b) for a, b in pairs]
+        return statistics.median(ts), sum(ts) / len(ts)
+
+    def host_cost(fn, n=300):
+        """Host time of one call (the launch is asynchronous; the queue is drained before and after)."""
+        torch.cuda.synchronize(dev)
+        t = time.perf_counter()
+        for _ in range(n):
+            fn()
+        dt = time.perf_counter() - t
+        torch.cuda.synchronize(dev)
+        return 1e6 * dt / n
+
+    for fn in (single_step, plan_step):
+        for _ in range(5):
+            fn()
+    t0 = time.time()
+    cold_plan_med, cold_plan = cold(plan_step)
+    cold_single_med, cold_single = cold(single_step)
+    empty_med, _ = cold(lambda: cast.check(cast.cast_probe_launch(tiles, stream)))
+    stream_med, _ = cold(lambda: cast.check(cast.cast_probe_stream(m1.w, m1.m, m1.v, m1.g, m1.w_fwd, m1.meta, rows * cols, stream)))
+    warm_single = timed(single_step, 200)
+    warm_plan = timed(plan_step, 200)
+    host_single = host_cost(single_step)
+    host_plan = host_cost(plan_step)
+    algorithmic_us = 1e6 * wl1.n_params * BYTES_PER_PARAM / (peak * 1e9)
+    out.append(entry(1, wl1, "2:4", cold_single, BYTES_PER_PARAM, t0, time.time(), steps=50,
+                     l2="L2 flushed by a 512 MB write before every step, steps timed one by one (mean; median beside it)",
+                     cold_us={"cast_adams_step": 1e3 * cold_single, "cast_adams_step_median": 1e3 * cold_single_med,
+                              "cast_plan_step": 1e3 * cold_plan, "cast_plan_step_median": 1e3 * cold_plan_med},
+                     warm_l2_us={"cast_adams_step": 1e3 * warm_single, "cast_plan_step": 1e3 * warm_plan,
+                                 "note": "back to back without the flush: the state stays in L2, not an HBM figure"},
+                     floors_us={"algorithmic_bytes_at_measured_peak": algorithmic_us,
+                                "empty_grid_same_ctas_cold": 1e3 * empty_med,
+                                "loads_and_stores_only_same_shape_cold": 1e3 * stream_med,
+                                "note": f"cast_probe_launch({tiles}) and cast_probe_stream over the same buffers, same flush, medians of 50"},
+                     host_us_per_call={"cast_adams_step": host_single, "cast_plan_step": host_plan,
+                                       "note": "host time of the asynchronous call (argument checks, pointer attribute queries, launch)"},
+                     parity={"ok": bool(parity_ok), "sample": f"first {sample_rows} rows after the first step"}))
+    s1.close()
+    del s1, flush
+    torch.cuda.empty_cache()
+    out.sort(key=lambda e: (e["config"], e["nm"], e.get("l1_coeff", 0.0)))
+    return out
+
+
+def pcie_ceiling(dev, mb=256, reps=6):
+    """Concurrent host->device and device->host copies of page-locked buffers on two streams: GB/s each way."""
+    import torch
+    n = mb << 20
+    h_in = torch.empty(n, dtype=torch.uint8).pin_memory()
+    h_out = torch.empty(n, dtype=torch.uint8).pin_memory()
+    d_in = torch.empty(n, dtype=torch.uint8, device=dev)
+    d_out = torch.zeros(n, dtype=torch.uint8, device=dev)
+    s_up, s_down = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+    best = None
+    for i in range(reps + 1):
+        torch.cuda.synchronize(dev)
+        t = time.perf_counter()
+        with torch.cuda.stream(s_up):
+            d_in.copy_(h_in, non_blocking=True)
+        with torch.cuda.stream(s_down):
+            h_out.copy_(d_out, non_blocking=True)
+        torch.cuda.synchronize(dev)
+        dt = time.perf_counter() - t
+        if i and (best is None or dt < best):
+            best = dt
+    return n / best / 1e9
 
 
 def cuda_arm(args):
@@ -371,8 +672,7 @@ def cuda_arm(args):
     clocks = None
     if sampler is not None:
         time.sleep(0.15)
-        sampler.stop()
-        clocks = sampler.summary(t_wall0, t_wall1)
+        clocks = sampler.summary(t_wall0, t_wall1)       # the sampler keeps running for the other configurations
 
     ms_per_step = ms / args.steps
     # launches of the step kernel per step: one per resident-layer call, else one per 320 matrices
@@ -415,9 +715,16 @@ def cuda_arm(args):
         dt = replicas.max_over_ranks(time.perf_counter() - t0, dev)
         cast.check(cast.cast_host_ctx_destroy(ctx))
         scale_bytes = sum(h["scale"].numel() * 4 for h in host)
+        ceiling = pcie_ceiling(dev)
+        h2d_gbs = (n_e2e * 14 + scale_bytes) * args.e2e_steps / dt / 1e9
+        d2h_gbs = n_e2e * 14.125 * args.e2e_steps / dt / 1e9
         e2e = {"value": world * n_e2e * args.e2e_steps / dt, "unit": "params/s",
                "h2d_bytes_per_step": int(n_e2e * 14 + scale_bytes), "d2h_bytes_per_step": int(n_e2e * 14.125),
                "ms_per_step": 1e3 * dt / args.e2e_steps,
+               "h2d_gbs": h2d_gbs, "d2h_gbs": d2h_gbs,
+               "pcie_ceiling_gbs_each_way": ceiling, "frac_of_pcie_ceiling": max(h2d_gbs, d2h_gbs) / ceiling,
+               "pcie_ceiling_how": "concurrent host->device and device->host copies of 256 MB page-locked buffers on two streams, "
+                                   "best of 6, measured in this run",
                "workload": f"first {len(shapes)} matrices of {wl.name} ({n_e2e} parameters) held in page-locked host memory, "
                            f"staged in 16 Mi-parameter blocks through 3 device slots",
                "steps": args.e2e_steps}
@@ -429,6 +736,26 @@ def cuda_arm(args):
             dist.barrier()
             dist.destroy_process_group()
         return
+
+    # host copies for the CPU baseline leg (taken before the device state is reused or freed below)
+    cpu_arrays, cpu_n = [], 0
+    if args.cpu_baseline and world == 1:
+        for i, sm in enumerate(mats):
+            if cpu_n and cpu_n + sm.rows * sm.cols > 210_000_000:
+                break
+            cpu_arrays.append(dict(w=sm.w.cpu().numpy(), m=sm.m.cpu().numpy(), v=sm.v.cpu().numpy(), g=workloads.bf16_bits(sm.g),
+                                   scale=sm.scale.cpu().numpy(), rows=sm.rows, cols=sm.cols))
+            cpu_n += sm.rows * sm.cols
+
+    # ---- the other listed workloads (1 GPU, default headline only): reported in `configs`
+    configs = None
+    headline_default = (wl.name == "llama2_7b" and (N, M) == (2, 4) and args.emit == "pruned" and args.schedule == "every-step"
+                        and not args.count_flips and not args.learned_scale)
+    if args.configs == "all" and world == 1 and headline_default:
+        configs = extra_configs(args, dev, stream, state, sampler, peak)
+        del state, mats
+    if sampler is not None:
+        sampler.stop()
 
     # ---- CPU baseline leg (rank 0, N = 1 only): the oracle as it stands on the host cores, plus parity of the sample
     cpu_baseline = None
@@ -454,13 +781,7 @@ def cuda_arm(args):
             ok &= bool(d.max() <= 1)
         parity = {"ok": ok, "sample": f"first {sample_rows} rows of matrices {picks} after the first step"}
         # timing sample: whole matrices from the front of the workload, about 2e8 parameters (one LLaMA2-7B layer)
-        arrays, n = [], 0
-        for i, s in enumerate(mats):
-            if n and n + s.rows * s.cols > 210_000_000:
-                break
-            arrays.append(dict(w=s.w.cpu().numpy(), m=s.m.cpu().numpy(), v=s.v.cpu().numpy(), g=workloads.bf16_bits(s.g),
-                               scale=s.scale.cpu().numpy(), rows=s.rows, cols=s.cols))
-            n += s.rows * s.cols
+        arrays, n = cpu_arrays, cpu_n
         threads = host_threads()
         oh.step = hyper.step
         time_oracle(arrays[:1], N, M, oh, o_flags, threads)                 # warm-up pass
@@ -494,13 +815,15 @@ def cuda_arm(args):
                      "note": "same steps back to back without the flush: the state stays in L2, not an HBM figure"}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}>",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}u, {'true' if (N, M) == (2, 4) else 'false'}>",
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": step_launches,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,
-                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None or args.emit != "pruned" or args.count_flips or (N, M) != (2, 4) or args.schedule != "every-step"
-                                 else NCU_DRAM_BYTES_PER_PARAM * wl.n_params / step_launches)},
-        "cpu_baseline": cpu_baseline, "parity": parity,
+                     "traffic": (None if NCU_DRAM_BYTES_PER_PARAM is None or not headline_default
+                                 else NCU_DRAM_BYTES_PER_PARAM * wl.n_params / step_launches),
+                     "traffic_from": (None if NCU_DRAM_BYTES_PER_PARAM is None or not headline_default else
+                                      f"ncu dram bytes per parameter of {NCU_KERNEL} on one LLaMA2-7B layer (profiles/), scaled by the parameter count")},
+        "cpu_baseline": cpu_baseline, "parity": parity, "configs": configs,
     }
     if world > 1:
         dist.barrier()

@@ -387,6 +387,22 @@ CAST_API int cast_host_step_static(float* w, float* m, float* v, const cast_bf16
                    uint32_t flags, unsigned long long* flip_count,
                    cast_stream_t stream);
 
+/*
+ * Measurement aids.  Neither computes anything of the method (the paper has no counterpart); a benchmark puts their
+ * times beside a measured step.
+ *
+ * cast_probe_launch   launches an empty grid of n_ctas CTAs of 128 threads on `stream`: the cost of launching and
+ *                     draining as many CTAs as a step over 1024 * n_ctas parameters has.
+ * cast_probe_stream   performs the loads and stores of one AdamS step over n_params parameters (device buffers
+ *                     sized as in cast_adams_step, n_params % 32 == 0, < 2^31) in the step's own launch shape and
+ *                     access pattern, with no arithmetic between them: w, m, v come back with their signs flipped,
+ *                     w_fwd receives the gradient's bits, meta is overwritten.  Its rate is the ceiling of a
+ *                     28.125-byte-per-parameter step of this shape on the device at hand.
+ */
+CAST_API int cast_probe_launch(int64_t n_ctas, cast_stream_t stream);
+CAST_API int cast_probe_stream(float* w, float* m, float* v, const cast_bf16* g, cast_bf16* w_fwd, uint32_t* meta,
+                      int64_t n_params, cast_stream_t stream);
+
 /* Static description of a status code (never NULL). */
 CAST_API const char* cast_strerror(int status);
 

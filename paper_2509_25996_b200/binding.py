@@ -41,6 +41,7 @@ EXPORTS = (
     "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_step_stats", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
+    "cast_probe_launch", "cast_probe_stream",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
 )
 
@@ -136,6 +137,10 @@ def load_library() -> ctypes.CDLL:
     lib.cast_plan_mask_stats.restype = ctypes.c_int
     lib.cast_plan_mask_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_uint32, ctypes.c_void_p,
                                          ctypes.c_void_p]
+    lib.cast_probe_launch.restype = ctypes.c_int
+    lib.cast_probe_launch.argtypes = [ctypes.c_int64, ctypes.c_void_p]
+    lib.cast_probe_stream.restype = ctypes.c_int
+    lib.cast_probe_stream.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int64, ctypes.c_void_p]
     lib.cast_host_ctx_sync.restype = ctypes.c_int
     lib.cast_host_ctx_sync.argtypes = [ctypes.c_void_p]
     lib.cast_host_ctx_destroy.restype = ctypes.c_int
@@ -168,6 +173,15 @@ def _stream(stream) -> Optional[int]:
     if isinstance(stream, int):
         return stream
     return stream.cuda_stream          # torch.cuda.Stream
+
+
+def kernel_flag_word(flags: int) -> int:
+    """The template argument that names the step kernel a flag word runs (flip counting is dropped where the mask
+    is reused: nothing can flip).  Names only; the library picks the kernel itself."""
+    f = int(flags) & 0xFF
+    if not f & CAST_F_RESELECT:
+        f &= ~CAST_F_COUNT_FLIPS
+    return f
 
 
 def cast_strerror(status: int) -> str:
@@ -321,6 +335,15 @@ def cast_plan_mask_stats(plan, meta_refs, flags, stats, stream=None) -> int:
     if meta_refs is not None:
         arr = (ctypes.c_void_p * len(meta_refs))(*[_ptr(r) for r in meta_refs])
     return load_library().cast_plan_mask_stats(plan, arr, int(flags), _ptr(stats), _stream(stream))
+
+
+def cast_probe_launch(n_ctas, stream=None) -> int:
+    return load_library().cast_probe_launch(int(n_ctas), _stream(stream))
+
+
+def cast_probe_stream(w, m, v, g, w_fwd, meta, n_params, stream=None) -> int:
+    return load_library().cast_probe_stream(_ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd), _ptr(meta), int(n_params),
+                                            _stream(stream))
 
 
 def cast_host_ctx_sync(ctx) -> int:

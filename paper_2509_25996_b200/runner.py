@@ -59,6 +59,9 @@ class DeviceModelState:
         self.device = torch.device(device)
         self.N, self.M = N, M
         self.compressed = compressed
+        self.seed, self.scale_mode, self.first_tensor_index = seed, scale_mode, first_tensor_index
+        self.reference_masks = reference_masks
+        self.plan = None
         self.mats: List[MatrixState] = []
         for i, (rows, cols) in enumerate(shapes):
             inp = workloads.gen_tensor_inputs(rows, cols, seed=seed, tensor_index=first_tensor_index + i,
@@ -80,12 +83,40 @@ class DeviceModelState:
         self.n_params = sum(s.rows * s.cols for s in self.mats)
         self.flips = torch.zeros(1, dtype=torch.int64, device=self.device)
         self.stats = torch.zeros(ctypes.sizeof(B.cast_mask_stats_t), dtype=torch.uint8, device=self.device)
+        self._make_plan()
+
+    def _make_plan(self) -> None:
         tensors = [B.make_tensor(s.w, s.m, s.v, s.g, s.w_fwd, s.meta, s.scale,
                                  1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad, s.meta_ref)
                    for s in self.mats]
-        rc, self.plan = B.cast_plan_create_ex(tensors, N, M, (B.CAST_F_EMIT_COMPRESSED if compressed else 0) |
-                                              (B.CAST_F_MASK_STATS if reference_masks else 0))
+        rc, self.plan = B.cast_plan_create_ex(tensors, self.N, self.M, (B.CAST_F_EMIT_COMPRESSED if self.compressed else 0) |
+                                              (B.CAST_F_MASK_STATS if self.reference_masks else 0))
         B.check(rc)
+
+    def set_nm(self, N: int, M: int) -> None:
+        """Another N:M pattern over the same buffers (a new plan; the state itself is not touched)."""
+        if self.compressed:
+            raise ValueError("the compressed forward-weight buffers are sized for one N:M")
+        self.close()
+        self.N, self.M = N, M
+        self._make_plan()
+
+    def reset(self) -> None:
+        """Draws the initial state again, from the same seeds, into the existing buffers (metadata zeroed)."""
+        for i, s in enumerate(self.mats):
+            inp = workloads.gen_tensor_inputs(s.rows, s.cols, seed=self.seed, tensor_index=self.first_tensor_index + i,
+                                              device=self.device, scale_mode=self.scale_mode)
+            s.w.copy_(inp.w); s.m.copy_(inp.m); s.v.copy_(inp.v); s.g.copy_(inp.g)
+            if s.scale is not None:
+                s.scale.copy_(inp.scale)
+            s.meta.zero_()
+            del inp
+        self.flips.zero_()
+
+    def fresh_gradients(self, step: int) -> None:
+        """A new seeded gradient for every matrix (what backpropagation would deliver at iteration `step`)."""
+        for i, s in enumerate(self.mats):
+            s.g.copy_(workloads.gen_gradient(s.rows, s.cols, self.seed, self.first_tensor_index + i, step, device=self.device))
 
     def step(self, hyper: Hyper, flags: int, stream=None) -> None:
         """One AdamS iteration over every matrix (asynchronous on `stream` or the current stream)."""
