@@ -32,10 +32,10 @@ FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
 # dram__bytes_read.sum + dram__bytes_write.sum per parameter of the headline kernel, from the ncu capture of one
 # LLaMA2-7B layer (202,375,168 parameters) summarised under profiles/ (which names the kernel the counters were
 # taken on); every byte is touched once, so the traffic of a launch is this figure times its parameter count.
-# None until the counters have been taken on the kernel as it stands; reported only for the workload and
+# Set to None when that kernel changes, until the counters are taken again; reported only for the workload and
 # configuration they were taken on (the 2:4 headline over LLaMA2-7B shapes).
-NCU_DRAM_BYTES_PER_PARAM = None
-NCU_KERNEL = "adams_nm_multi_kernel<4, 1u, true>"
+NCU_DRAM_BYTES_PER_PARAM = 27.849
+NCU_KERNEL = "adams_nm_multi_kernel<4, 1, 1>"
 
 METRIC = "AdamS 2:4 step params/s"
 
@@ -815,7 +815,7 @@ def cuda_arm(args):
                      "note": "same steps back to back without the flush: the state stays in L2, not an HBM figure"}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}u, {'true' if (N, M) == (2, 4) else 'false'}>",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}, {1 if (N, M) == (2, 4) else 0}>",
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": step_launches,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,
