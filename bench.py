@@ -989,18 +989,24 @@ def kd_arm(args):
     def one_pass():
         cast.check(cast.cast_kd_loss(student, teacher, labels, loss, grad, T, V, eta, 1.0 / T, stream))
 
+    sampler = ClockSampler("GPU-" + str(torch.cuda.get_device_properties(dev).uuid))
     for _ in range(args.warmup):
         one_pass()
     torch.cuda.synchronize(dev)
     launches0 = cast.cast_kernel_launch_count()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.profiler.start()
+    t_wall0 = time.time()
     ev0.record(stream)
     for _ in range(args.steps):
         one_pass()
     ev1.record(stream)
     torch.cuda.synchronize(dev)
+    t_wall1 = time.time()
     torch.cuda.profiler.stop()
+    time.sleep(0.15)
+    sampler.stop()
+    clocks = sampler.summary(t_wall0, t_wall1)
     ms = ev0.elapsed_time(ev1) / args.steps
     launches = cast.cast_kernel_launch_count() - launches0
     from oracle import adams_oracle as orc
@@ -1011,19 +1017,24 @@ def kd_arm(args):
     ok = bool(np.all(np.abs(got - ref_loss) <= 2e-5 + 1e-5 * np.abs(ref_loss)))
     gbs = T * V * 6.0 / (ms * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
+    # The op needs four exponentials per logit on the special-function unit (16 lanes per SM and clock): at the SM
+    # clock of this run (median of the samples taken during the timed region; the maximum clock if the region was too
+    # short to be sampled) that is the same order as the HBM bound, so the fraction is taken against the lower of the two.
+    sms = torch.cuda.get_device_properties(dev).multi_processor_count
+    clock_mhz = clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") and clocks["samples"] >= 3 else 1965.0
+    xu_logits = sms * 16 * clock_mhz * 1e6 / 4.0
+    hbm_logits = peak * 1e9 / 6.0
+    logits_s = T * V / (ms * 1e-3)
     print(json.dumps({
         "metric": "distillation loss + gradient (Eq. 13) tokens/s", "value": T / (ms * 1e-3), "unit": "tokens/s", "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{T} tokens x {V} logits", "eta": eta, "l2": "inputs far larger than L2, no flush"},
-        "gpu_launches": int(launches),
+        "gpu_launches": int(launches), "clocks": clocks,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak, "peak_kind": f"of {peak_kind}",
                      "kernel": "kd_loss_kernel", "bytes_per_logit": 6.0, "launches_per_step": 1, "traffic": None},
-        # the op needs four exponentials per logit on the special-function unit (16 lanes per SM and clock): at the
-        # maximum SM clock that is the same order as the HBM bound, so both are reported
-        "xu_roofline": {"bound": "alu", "unit": "logits/s", "achieved": T * V / (ms * 1e-3),
-                        "peak": torch.cuda.get_device_properties(dev).multi_processor_count * 16 * 1.965e9 / 4.0,
-                        "frac": (T * V / (ms * 1e-3)) / (torch.cuda.get_device_properties(dev).multi_processor_count * 16 * 1.965e9 / 4.0),
-                        "peak_kind": "derived: SMs x 16 ex2 per clock x 1.965 GHz / 4 ex2 per logit"},
+        "xu_roofline": {"bound": "alu", "unit": "logits/s", "achieved": logits_s, "peak": xu_logits, "frac": logits_s / xu_logits,
+                        "peak_kind": f"derived: {sms} SMs x 16 ex2 per clock x {clock_mhz:.0f} MHz / 4 ex2 per logit"},
+        "frac_of_lower_bound": logits_s / min(xu_logits, hbm_logits),
         "mean_loss": float(loss.double().mean().item()),
         "parity": {"ok": ok, "sample": f"losses of the first {rows} tokens against the CPU oracle"}}), flush=True)
 

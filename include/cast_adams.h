@@ -267,7 +267,10 @@ CAST_API int cast_plan_destroy(void* plan);
  *                       memory makes the copies asynchronous; pageable memory works and is slower).
  *                       flip_count is a host counter that is added to.  The call returns when all work
  *                       is queued; results are valid after cast_host_ctx_sync.  A matrix whose rows are
- *                       longer than max_block_params is rejected with CAST_ERR_PLAN.
+ *                       longer than max_block_params is rejected with CAST_ERR_PLAN.  If a CUDA call fails
+ *                       part-way (CAST_ERR_CUDA), the call first waits for every copy it has already queued
+ *                       and then returns: nothing touches the host buffers afterwards, but they may hold a
+ *                       partly updated state.
  * cast_host_ctx_sync    waits for everything queued through the context and folds the flip counts.
  * cast_host_ctx_destroy waits, then frees streams and buffers.
  */
@@ -364,12 +367,21 @@ CAST_API int cast_plan_mask_stats(void* plan, const uint32_t* const* meta_ref, u
  * process uses the library, until the process exits), and the call allocates and frees nothing, on the
  * device or through any other library.
  *
+ *   When the memory is taken: the CUDA runtime loads device code lazily by default, so the image that holds the
+ *   staging area is placed in device memory by the FIRST call on each device, not when the library is opened.
+ *   That first call needs about 16.6 MiB of free device memory (it fails with CAST_ERR_CUDA otherwise) and may
+ *   synchronise the device.  Make it once per device at start-up -- any small matrix will do -- before the
+ *   framework's allocator takes the memory and outside any stream capture; or run the process with
+ *   CUDA_MODULE_LOADING=EAGER, which moves the loading to context creation.  Later calls leave the amount of
+ *   free device memory exactly as they find it.
+ *
  *   Arguments as cast_host_step (every data pointer is a HOST pointer; flip_count is a host counter that
  *   is added to), plus `stream`, on which the copies and the kernel are queued.
  *   Limit: rows * cols <= CAST_STATIC_MAX_PARAMS; a larger matrix is refused with CAST_ERR_PLAN (the
  *   staging area is too small) and nothing is queued.  Cut larger matrices into blocks of whole rows.
  *   The call is synchronous: it returns after `stream` has finished the step, with the results in the
- *   host buffers.
+ *   host buffers.  This also holds when a CUDA call fails part-way (CAST_ERR_CUDA): the stream is drained
+ *   before the error is returned, and the host buffers may then hold a partly updated state.
  *   The first call on each device looks up the device address of the staging area (with that device
  *   current); make that first call outside any stream capture.
  *   All calls of a process on one device share the one staging area, which keeps the contents the

@@ -58,7 +58,10 @@ int sync_ctx(HostCtx* c)
         CAST_CUDA_TRY(cudaMemcpy(c->h_flips, c->d_flips, sizeof(unsigned long long) * (size_t)c->n_flip_pending,
                                  cudaMemcpyDeviceToHost));
         for (int i = 0; i < c->n_flip_pending; ++i) *c->flip_dst[i] += c->h_flips[i];
-        CAST_CUDA_TRY(cudaMemset(c->d_flips, 0, sizeof(unsigned long long) * (size_t)c->n_flip_pending));
+        // cleared on a slot stream and waited for: the slot streams do not order against the legacy default stream,
+        // so a plain cudaMemset could still be pending when the next counting step starts
+        CAST_CUDA_TRY(cudaMemsetAsync(c->d_flips, 0, sizeof(unsigned long long) * (size_t)c->n_flip_pending, c->slot[0].stream));
+        CAST_CUDA_TRY(cudaStreamSynchronize(c->slot[0].stream));
         c->n_flip_pending = 0;
     }
     return CAST_OK;
@@ -113,6 +116,7 @@ extern "C" int cast_host_ctx_create(int64_t max_block_params, int n_slots, void*
     }
     if (e == cudaSuccess) e = cudaMalloc(&c->d_flips, sizeof(unsigned long long) * kFlipCounters);
     if (e == cudaSuccess) e = cudaMemset(c->d_flips, 0, sizeof(unsigned long long) * kFlipCounters);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();      // the counters are zero before any slot stream can add to them
     if (e == cudaSuccess) e = cudaMallocHost(&c->h_flips, sizeof(unsigned long long) * kFlipCounters);
     if (e != cudaSuccess) {
         free_ctx(c);
@@ -158,31 +162,42 @@ extern "C" int cast_host_step(void* ctx,
     }
     const bool need_prev = !(flags & CAST_F_RESELECT) || (flags & CAST_F_COUNT_FLIPS);
     const int64_t rows_per_block = c->max_block / cols;
-    for (int64_t r0 = 0; r0 < rows; r0 += rows_per_block) {
-        const int64_t nr = (rows - r0 < rows_per_block) ? rows - r0 : rows_per_block;
-        const size_t P = (size_t)nr * (size_t)cols, off = (size_t)r0 * (size_t)cols;
-        Slot& s = c->slot[c->next_slot];
-        c->next_slot = (c->next_slot + 1) % c->n_slots;
-        CAST_CUDA_TRY(cudaMemcpyAsync(s.w, w + off, 4 * P, cudaMemcpyHostToDevice, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(s.m, m + off, 4 * P, cudaMemcpyHostToDevice, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(s.v, v + off, 4 * P, cudaMemcpyHostToDevice, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(s.g, g + off, 2 * P, cudaMemcpyHostToDevice, s.stream));
-        if (need_prev)
-            CAST_CUDA_TRY(cudaMemcpyAsync(s.meta, meta + off / 32, P / 8, cudaMemcpyHostToDevice, s.stream));
-        if (scale)
-            CAST_CUDA_TRY(cudaMemcpyAsync(s.scale, scale + (size_t)r0 * (size_t)scale_groups,
-                                          4 * (size_t)nr * (size_t)scale_groups, cudaMemcpyHostToDevice, s.stream));
-        const TensorDesc d = make_desc(s.w, s.m, s.v, s.g, s.fwd, s.meta, scale ? s.scale : nullptr, scale_groups, nr, cols);
-        if ((rc = launch_single(d, M, k, d_flip, s.stream)) != CAST_OK) return rc;
-        CAST_CUDA_TRY(cudaMemcpyAsync(w + off, s.w, 4 * P, cudaMemcpyDeviceToHost, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(m + off, s.m, 4 * P, cudaMemcpyDeviceToHost, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(v + off, s.v, 4 * P, cudaMemcpyDeviceToHost, s.stream));
-        const size_t fwd_scale_n = (flags & CAST_F_EMIT_COMPRESSED) ? (size_t)N : 1, fwd_scale_m = (flags & CAST_F_EMIT_COMPRESSED) ? (size_t)M : 1;
-        CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16 + off / fwd_scale_m * fwd_scale_n, s.fwd, 2 * (P / fwd_scale_m * fwd_scale_n),
-                                      cudaMemcpyDeviceToHost, s.stream));
-        CAST_CUDA_TRY(cudaMemcpyAsync(meta + off / 32, s.meta, P / 8, cudaMemcpyDeviceToHost, s.stream));
+    auto queue_all = [&]() -> int {
+        for (int64_t r0 = 0; r0 < rows; r0 += rows_per_block) {
+            const int64_t nr = (rows - r0 < rows_per_block) ? rows - r0 : rows_per_block;
+            const size_t P = (size_t)nr * (size_t)cols, off = (size_t)r0 * (size_t)cols;
+            Slot& s = c->slot[c->next_slot];
+            c->next_slot = (c->next_slot + 1) % c->n_slots;
+            CAST_CUDA_TRY(cudaMemcpyAsync(s.w, w + off, 4 * P, cudaMemcpyHostToDevice, s.stream));
+            CAST_CUDA_TRY(cudaMemcpyAsync(s.m, m + off, 4 * P, cudaMemcpyHostToDevice, s.stream));
+            CAST_CUDA_TRY(cudaMemcpyAsync(s.v, v + off, 4 * P, cudaMemcpyHostToDevice, s.stream));
+            CAST_CUDA_TRY(cudaMemcpyAsync(s.g, g + off, 2 * P, cudaMemcpyHostToDevice, s.stream));
+            if (need_prev)
+                CAST_CUDA_TRY(cudaMemcpyAsync(s.meta, meta + off / 32, P / 8, cudaMemcpyHostToDevice, s.stream));
+            if (scale)
+                CAST_CUDA_TRY(cudaMemcpyAsync(s.scale, scale + (size_t)r0 * (size_t)scale_groups,
+                                              4 * (size_t)nr * (size_t)scale_groups, cudaMemcpyHostToDevice, s.stream));
+            const TensorDesc d = make_desc(s.w, s.m, s.v, s.g, s.fwd, s.meta, scale ? s.scale : nullptr, scale_groups, nr, cols);
+            const int launch_rc = launch_single(d, M, k, d_flip, s.stream);
+            if (launch_rc != CAST_OK) return launch_rc;
+            CAST_CUDA_TRY(cudaMemcpyAsync(w + off, s.w, 4 * P, cudaMemcpyDeviceToHost, s.stream));
+            CAST_CUDA_TRY(cudaMemcpyAsync(m + off, s.m, 4 * P, cudaMemcpyDeviceToHost, s.stream));
+            CAST_CUDA_TRY(cudaMemcpyAsync(v + off, s.v, 4 * P, cudaMemcpyDeviceToHost, s.stream));
+            const size_t fwd_scale_n = (flags & CAST_F_EMIT_COMPRESSED) ? (size_t)N : 1, fwd_scale_m = (flags & CAST_F_EMIT_COMPRESSED) ? (size_t)M : 1;
+            CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16 + off / fwd_scale_m * fwd_scale_n, s.fwd, 2 * (P / fwd_scale_m * fwd_scale_n),
+                                          cudaMemcpyDeviceToHost, s.stream));
+            CAST_CUDA_TRY(cudaMemcpyAsync(meta + off / 32, s.meta, P / 8, cudaMemcpyDeviceToHost, s.stream));
+        }
+        return CAST_OK;
+    };
+    rc = queue_all();
+    if (rc != CAST_OK) {
+        // a call failed part-way: wait for the copies already queued, so that nothing is still reading or writing the
+        // caller's host buffers when the error comes back (the state in them may be partly updated)
+        for (int i = 0; i < c->n_slots; ++i) (void)cudaStreamSynchronize(c->slot[i].stream);
+        (void)cudaGetLastError();
     }
-    return CAST_OK;
+    return rc;
 }
 
 extern "C" int cast_host_ctx_sync(void* ctx)

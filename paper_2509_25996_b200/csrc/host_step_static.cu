@@ -6,9 +6,17 @@
 // (a further cudaMalloc fails or forces the pool to shrink), a step that runs where the implicit
 // device-wide synchronisation of cudaMalloc / cudaFree is not acceptable, or a process that is simply
 // not allowed to grow its device footprint after start-up.  For them the staging area below is a
-// file-scope __device__ array: it is reserved when the library is loaded on a GPU (every GPU that
-// loads the library holds these ~16.6 MiB until the process exits) and nothing is ever allocated or
-// freed by this entry point, by CUDA on its behalf, or by any other library.
+// file-scope __device__ array: it belongs to the library image, every GPU on which the process uses
+// it holds these ~16.6 MiB until the process exits, and this entry point calls no allocation or
+// release routine of CUDA or of any other library.
+//
+// When the memory is actually taken.  The CUDA runtime loads a library's device code lazily by
+// default: the image that holds the array is placed in device memory by the FIRST call of this
+// entry point on a device (its cudaGetSymbolAddress), not when the shared library is opened.  That
+// first call therefore needs ~16.6 MiB of free device memory and may synchronise the device: make
+// it once per device at start-up, before a framework allocator takes the memory and outside any
+// stream capture (or run the process with CUDA_MODULE_LOADING=EAGER, which moves the loading to
+// context creation).  Every later call finds the address cached and touches no memory management.
 //
 // The array's name is only a host-side handle here: its device address is looked up once per device
 // with cudaGetSymbolAddress (with that device current) and that address is what kernels and copies get.
@@ -103,25 +111,34 @@ extern "C" int cast_host_step_static(float* w, float* m, float* v, const cast_bf
     const size_t P = (size_t)rows * (size_t)cols;
     const bool count = (flags & CAST_F_COUNT_FLIPS) != 0;
     const bool need_prev = !(flags & CAST_F_RESELECT) || count;
-    CAST_CUDA_TRY(cudaMemcpyAsync(d_w, w, 4 * P, cudaMemcpyHostToDevice, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(d_m, m, 4 * P, cudaMemcpyHostToDevice, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(d_v, v, 4 * P, cudaMemcpyHostToDevice, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(d_g, g, 2 * P, cudaMemcpyHostToDevice, s));
-    if (need_prev) CAST_CUDA_TRY(cudaMemcpyAsync(d_meta, meta, P / 8, cudaMemcpyHostToDevice, s));
-    if (scale)
-        CAST_CUDA_TRY(cudaMemcpyAsync(d_scale, scale, 4 * (size_t)rows * (size_t)scale_groups, cudaMemcpyHostToDevice, s));
-    // the area keeps whatever the previous call left: the counter is the one part that must start at zero
-    if (count) CAST_CUDA_TRY(cudaMemsetAsync(d_flips, 0, sizeof(unsigned long long), s));
-    const TensorDesc d = make_desc(d_w, d_m, d_v, d_g, d_fwd, d_meta, scale ? d_scale : nullptr, scale_groups, rows, cols);
-    if ((rc = launch_single(d, M, k, count ? d_flips : nullptr, s)) != CAST_OK) return rc;
-    CAST_CUDA_TRY(cudaMemcpyAsync(w, d_w, 4 * P, cudaMemcpyDeviceToHost, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(m, d_m, 4 * P, cudaMemcpyDeviceToHost, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(v, d_v, 4 * P, cudaMemcpyDeviceToHost, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16, d_fwd, 2 * (size_t)fwd_total, cudaMemcpyDeviceToHost, s));
-    CAST_CUDA_TRY(cudaMemcpyAsync(meta, d_meta, P / 8, cudaMemcpyDeviceToHost, s));
     unsigned long long flips = 0;
-    if (count) CAST_CUDA_TRY(cudaMemcpyAsync(&flips, d_flips, sizeof flips, cudaMemcpyDeviceToHost, s));
-    CAST_CUDA_TRY(cudaStreamSynchronize(s));
+    // Everything is queued by this lambda; whatever it returns, the stream is drained before the call returns, so that
+    // no copy into or out of the caller's host buffers is still in flight when the caller gets control back.
+    auto queue_all = [&]() -> int {
+        CAST_CUDA_TRY(cudaMemcpyAsync(d_w, w, 4 * P, cudaMemcpyHostToDevice, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(d_m, m, 4 * P, cudaMemcpyHostToDevice, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(d_v, v, 4 * P, cudaMemcpyHostToDevice, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(d_g, g, 2 * P, cudaMemcpyHostToDevice, s));
+        if (need_prev) CAST_CUDA_TRY(cudaMemcpyAsync(d_meta, meta, P / 8, cudaMemcpyHostToDevice, s));
+        if (scale)
+            CAST_CUDA_TRY(cudaMemcpyAsync(d_scale, scale, 4 * (size_t)rows * (size_t)scale_groups, cudaMemcpyHostToDevice, s));
+        // the area keeps whatever the previous call left: the counter is the one part that must start at zero
+        if (count) CAST_CUDA_TRY(cudaMemsetAsync(d_flips, 0, sizeof(unsigned long long), s));
+        const TensorDesc d = make_desc(d_w, d_m, d_v, d_g, d_fwd, d_meta, scale ? d_scale : nullptr, scale_groups, rows, cols);
+        const int launch_rc = launch_single(d, M, k, count ? d_flips : nullptr, s);
+        if (launch_rc != CAST_OK) return launch_rc;
+        CAST_CUDA_TRY(cudaMemcpyAsync(w, d_w, 4 * P, cudaMemcpyDeviceToHost, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(m, d_m, 4 * P, cudaMemcpyDeviceToHost, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(v, d_v, 4 * P, cudaMemcpyDeviceToHost, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(w_fwd_bf16, d_fwd, 2 * (size_t)fwd_total, cudaMemcpyDeviceToHost, s));
+        CAST_CUDA_TRY(cudaMemcpyAsync(meta, d_meta, P / 8, cudaMemcpyDeviceToHost, s));
+        if (count) CAST_CUDA_TRY(cudaMemcpyAsync(&flips, d_flips, sizeof flips, cudaMemcpyDeviceToHost, s));
+        return CAST_OK;
+    };
+    rc = queue_all();
+    const cudaError_t drained = cudaStreamSynchronize(s);
+    if (rc != CAST_OK) return rc;             // the host buffers may hold a partly updated state: see the header
+    if (drained != cudaSuccess) return cuda_failed(drained);
     if (count) *flip_count += flips;
     return CAST_OK;
 }

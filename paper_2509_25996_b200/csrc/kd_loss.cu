@@ -1,22 +1,32 @@
 // Training loss of CAST (Sec. 4.3, Eq. 13) per token, L = eta D_KL(P_t || P_s) + (1 - eta) L_ce, and its gradient
 // with respect to the student logits, grad_scale (P_s - eta P_t - (1 - eta) onehot), in one kernel.
 //
-// Streaming and reduction-bound: a row of `vocab` logits per token, 2 + 2 B read and 2 B written per logit.
-// One CTA per token.  With
+// Streaming and reduction-bound: a row of `vocab` logits per token, 2 + 2 B read and 2 B written per logit.  With
 //     D_KL(P_t || P_s) = E_{P_t}[t - s] + lse(s) - lse(t),        L_ce = lse(s) - s_label,
 // a single sweep over the row yields everything the loss needs: the running maxima and sums of exp of both rows
 // (online softmax: a sum is rescaled when its maximum moves) and sum exp(t - max t) (t - s).  The gradient needs
-// the finished normalisers, i.e. a second sweep over the same values: the row is simply read again -- the rows in
-// flight (a few CTAs per SM x 2 x vocab x 2 B, tens of MB) sit well inside the 126 MB L2, so the second sweep does
-// not go to HBM.  (Keeping rows of up to 32768 logits in registers between the sweeps, 8 vectors per thread and
-// row, was measured slower: 118 registers allow one CTA per SM, whose phases then do not overlap.)
+// the finished normalisers, i.e. a second sweep over the same values: the row is read again, and that second read
+// has to come from the L2, not from HBM (6 instead of 10 B per logit).  Two things keep it there:
+//   * the rows in flight are bounded: a row is handled by a cluster of CTAs (1 CTA for short rows, 8 for rows
+//     beyond 64 K logits), each CTA sweeping its own segment of the row; the clusters' CTAs exchange their five
+//     partial sums through distributed shared memory (plain loads of a peer CTA's shared memory between two cluster
+//     barriers).  With 8 CTAs per row a 128 K-logit vocabulary has ~150 rows (75 MB) in flight instead of the
+//     ~2400 rows (1.2 GB) of one small CTA per row, whose second sweep went to HBM;
+//   * the second sweep runs back to front, so it starts on the lines the first sweep touched last.
 // The kernel is co-limited by the special-function unit: four exponentials per logit (two per sweep) at 16 per
-// clock and SM is the same ~1.1e12 logits/s as 6 B per logit at the HBM rate.
+// clock and SM is the same ~1.1e12 logits/s as 6 B per logit at the HBM rate; everything else per logit is kept
+// small: the weights of the gradient's two terms are folded into the exponents (one subtraction gives the
+// gradient), the label is looked for once per vector.
 // Arithmetic in fp32 in the base-2 domain (ex2.approx: 2 ulp; argument error ~1e-7 |x log2 e|); reductions by warp
-// shuffles and shared memory.  No device-side waits.
+// shuffles and shared memory.  No device-side waits other than the cluster's hardware barrier, at which every CTA of
+// a cluster arrives unconditionally.
 #include <cmath>
 
+#include <cooperative_groups.h>
+
 #include "cast_internal.h"
+
+namespace cg = cooperative_groups;
 
 namespace cast {
 namespace {
@@ -105,12 +115,13 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 struct Finished { float lse_s2, lse_t2; };      // log-sum-exp of both rows in the base-2 domain
 
 // loss of the token from the finished sums; written by one thread
-__device__ __forceinline__ Finished finish(const RowSums& r, const uint16_t* s_row, int label, float eta, float* loss_out)
+__device__ __forceinline__ Finished finish(const RowSums& r, const uint16_t* s_row, int label, float eta, float* loss_out,
+                                           bool writer = true)
 {
     Finished f;
     f.lse_s2 = r.ms2 + log2f(r.zs);
     f.lse_t2 = r.mt2 + log2f(r.zt);
-    if (threadIdx.x == 0) {
+    if (writer && threadIdx.x == 0) {
         const float lse_s = f.lse_s2 * kLn2;
         const float kl = r.a / r.zt + (f.lse_s2 - f.lse_t2) * kLn2;                       // E_t[t - s] + lse(s) - lse(t)
         float ce = 0.0f;
@@ -120,80 +131,90 @@ __device__ __forceinline__ Finished finish(const RowSums& r, const uint16_t* s_r
     return f;
 }
 
+// What the second sweep needs: exponent offsets with the weights of the gradient's two terms folded in,
+//   |grad_scale| w_s P_s = 2^(s log2 e + off_s),  off_s = log2(|grad_scale| w_s) - lse_s2     (w_s = 1, or eta without a target)
+//   |grad_scale| eta P_t = 2^(t log2 e + off_t),  off_t = log2(|grad_scale| eta) - lse_t2
+// (a zero weight gives off = -inf and a term that is exactly 0), the sign of grad_scale, and the one-hot term.
+struct GradConsts { float off_s, off_t, onehot; uint32_t sign_bits; };   // sign_bits: 0x80008000 flips a packed pair
+
+__device__ __forceinline__ GradConsts grad_consts(const Finished& f, int label, float eta, float grad_scale)
+{
+    const float mag = fabsf(grad_scale);
+    GradConsts g;
+    g.off_s = log2f(mag * (label >= 0 ? 1.0f : eta)) - f.lse_s2;
+    g.off_t = log2f(mag * eta) - f.lse_t2;
+    g.sign_bits = grad_scale < 0.0f ? 0x80008000u : 0u;      // the sign of grad_scale is applied to the packed result
+    g.onehot = label >= 0 ? mag * (1.0f - eta) : 0.0f;
+    return g;
+}
+
 // gradient of 8 logits starting at column `col`
-__device__ __forceinline__ uint4 grad8(const float (&s)[8], const float (&t)[8], const Finished& f, int col, int label,
-                                       float eta, float ps_weight, float onehot_weight, float grad_scale)
+__device__ __forceinline__ uint4 grad8(const float (&s)[8], const float (&t)[8], const GradConsts& k, int col, int label)
 {
     float g[8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const float ps = ex2(fmaf(s[i], kLog2e, -f.lse_s2)), pt = ex2(fmaf(t[i], kLog2e, -f.lse_t2));
-        float x = fmaf(ps_weight, ps, -eta * pt);
-        if (col + i == label) x -= onehot_weight;
-        g[i] = grad_scale * x;
+    for (int i = 0; i < 8; ++i)
+        g[i] = ex2(fmaf(s[i], kLog2e, k.off_s)) - ex2(fmaf(t[i], kLog2e, k.off_t));
+    const unsigned rel = (unsigned)(label - col);          // the label's place in this vector, if it is here
+    if (rel < 8u) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+            if (rel == (unsigned)i) g[i] -= k.onehot;
     }
-    return make_uint4(pack2(g[0], g[1]), pack2(g[2], g[3]), pack2(g[4], g[5]), pack2(g[6], g[7]));
+    return make_uint4(pack2(g[0], g[1]) ^ k.sign_bits, pack2(g[2], g[3]) ^ k.sign_bits, pack2(g[4], g[5]) ^ k.sign_bits,
+                      pack2(g[6], g[7]) ^ k.sign_bits);
 }
 
-// vocab % 8 == 0.  CH > 0 (not used by the entry point): the row (at most CH * THREADS vectors) is kept in registers
-// between the two sweeps.
-template <int THREADS, int CH>
+// vocab % 8 == 0.  A cluster of CLUSTER CTAs handles one row (token); CTA `rank` of the cluster sweeps the vectors
+// [rank * per, min(n_vec, (rank + 1) * per)) of it.
+template <int THREADS, int CLUSTER>
 __global__ void __launch_bounds__(THREADS)
 kd_loss_kernel(const uint16_t* __restrict__ student, const uint16_t* __restrict__ teacher, const int32_t* __restrict__ labels,
                float* __restrict__ loss, uint16_t* __restrict__ grad, int vocab, float eta, float grad_scale)
 {
-    const size_t row = (size_t)blockIdx.x * (size_t)vocab;
+    const unsigned token = blockIdx.x / CLUSTER;
+    unsigned rank = 0;
+    if constexpr (CLUSTER > 1) rank = cg::this_cluster().block_rank();
+    const size_t row = (size_t)token * (size_t)vocab;
     const uint4* s_vec = reinterpret_cast<const uint4*>(student + row);
     const uint4* t_vec = reinterpret_cast<const uint4*>(teacher + row);
     const int n_vec = vocab / 8;
-    int label = labels[blockIdx.x];
+    const int per = (n_vec + CLUSTER - 1) / CLUSTER;
+    const int v0 = (int)rank * per, v1 = min(n_vec, v0 + per);
+    int label = labels[token];
     if (label >= vocab) label = -1;          // out of range: no target (never read past the row)
+
     RowSums r = {-INFINITY, 0.0f, -INFINITY, 0.0f, 0.0f};
-    constexpr int HELD = CH > 0 ? CH : 1;
-    uint4 sv[HELD], tv[HELD];
-    if constexpr (CH > 0) {
-#pragma unroll
-        for (int k = 0; k < CH; ++k) {
-            const int c = threadIdx.x + k * THREADS;
-            if (c < n_vec) { sv[k] = s_vec[c]; tv[k] = t_vec[c]; }
-        }
-#pragma unroll
-        for (int k = 0; k < CH; ++k) {
-            if (threadIdx.x + k * THREADS < n_vec) {
-                float s[8], t[8];
-                unpack8(sv[k], s); unpack8(tv[k], t);
-                absorb8(r, s, t);
-            }
-        }
-    } else {
-        for (int c = threadIdx.x; c < n_vec; c += THREADS) {
-            float s[8], t[8];
-            unpack8(s_vec[c], s); unpack8(t_vec[c], t);
-            absorb8(r, s, t);
-        }
+#pragma unroll 2
+    for (int c = v0 + (int)threadIdx.x; c < v1; c += THREADS) {
+        float s[8], t[8];
+        unpack8(s_vec[c], s); unpack8(t_vec[c], t);
+        absorb8(r, s, t);
     }
     r = block_merge<THREADS>(r);
-    const Finished f = finish(r, student + row, label, eta, loss + blockIdx.x);
-    if (grad == nullptr) return;
-    // with a target: P_s - eta P_t - (1 - eta) onehot; without: the cross-entropy share of P_s drops out too
-    const float ps_weight = label >= 0 ? 1.0f : eta, onehot_weight = label >= 0 ? 1.0f - eta : 0.0f;
-    uint4* g_vec = reinterpret_cast<uint4*>(grad + row);
-    if constexpr (CH > 0) {
+    if constexpr (CLUSTER > 1) {
+        // every CTA of the cluster publishes the sums of its segment and merges all of them (in rank order, so that
+        // all CTAs of the row get the same bits)
+        __shared__ RowSums mine;
+        cg::cluster_group cluster = cg::this_cluster();
+        if (threadIdx.x == 0) mine = r;
+        cluster.sync();
+        RowSums total = *cluster.map_shared_rank(&mine, 0);
 #pragma unroll
-        for (int k = 0; k < CH; ++k) {
-            const int c = threadIdx.x + k * THREADS;
-            if (c < n_vec) {
-                float s[8], t[8];
-                unpack8(sv[k], s); unpack8(tv[k], t);
-                g_vec[c] = grad8(s, t, f, c * 8, label, eta, ps_weight, onehot_weight, grad_scale);
-            }
-        }
-    } else {
-        for (int c = threadIdx.x; c < n_vec; c += THREADS) {
-            float s[8], t[8];
-            unpack8(s_vec[c], s); unpack8(t_vec[c], t);
-            g_vec[c] = grad8(s, t, f, c * 8, label, eta, ps_weight, onehot_weight, grad_scale);
-        }
+        for (int k = 1; k < CLUSTER; ++k) merge(total, *cluster.map_shared_rank(&mine, k));
+        cluster.sync();                      // no CTA leaves (or overwrites `mine`) while a peer may still read it
+        r = total;
+    }
+    const Finished f = finish(r, student + row, label, eta, loss + token, rank == 0);
+    if (grad == nullptr) return;
+    const GradConsts k = grad_consts(f, label, eta, grad_scale);
+    uint4* g_vec = reinterpret_cast<uint4*>(grad + row);
+    // back to front: the second sweep starts on the part of the segment the first sweep read last
+#pragma unroll 2
+    for (int c = v1 - 1 - (int)threadIdx.x; c >= v0; c -= THREADS) {
+        float s[8], t[8];
+        unpack8(s_vec[c], s); unpack8(t_vec[c], t);
+        g_vec[c] = grad8(s, t, k, c * 8, label);
     }
 }
 
@@ -255,14 +276,31 @@ extern "C" int cast_kd_loss(const cast_bf16* student_logits, const cast_bf16* te
     const unsigned grid = (unsigned)tokens;
     const bool vec = vocab % 8 == 0 && !((uintptr_t)student_logits & 15u) && !((uintptr_t)teacher_logits & 15u) &&
                      !((uintptr_t)grad_logits & 15u);
-    // measured on B200: 512 threads per row up to ~64 K logits, 128 beyond (more rows in flight per SM)
-    if (vec && vocab <= 65536)
-        kd_loss_kernel<512, 0><<<grid, 512, 0, s>>>(student_logits, teacher_logits, labels, loss, grad_logits, (int)vocab, eta, grad_scale);
-    else if (vec)
-        kd_loss_kernel<128, 0><<<grid, 128, 0, s>>>(student_logits, teacher_logits, labels, loss, grad_logits, (int)vocab, eta, grad_scale);
-    else
+    if (vec && vocab <= 65536) {
+        // one CTA of 512 threads per row: ~450 rows of <= 256 KB in flight, inside the L2
+        kd_loss_kernel<512, 1><<<grid, 512, 0, s>>>(student_logits, teacher_logits, labels, loss, grad_logits, (int)vocab, eta, grad_scale);
+        CAST_CUDA_TRY(cudaGetLastError());
+    } else if (vec) {
+        // a cluster of 8 CTAs of 256 threads per row: the rows in flight stay inside the L2 for long rows too
+        constexpr int kCluster = 8;
+        if ((uint64_t)tokens * kCluster > 0x7FFFFFFFull) return CAST_ERR_SHAPE;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid * kCluster);
+        cfg.blockDim = dim3(256);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = kCluster;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        CAST_CUDA_TRY(cudaLaunchKernelEx(&cfg, kd_loss_kernel<256, kCluster>, (const uint16_t*)student_logits, (const uint16_t*)teacher_logits,
+                                         labels, loss, (uint16_t*)grad_logits, (int)vocab, eta, grad_scale));
+    } else {
         kd_loss_scalar_kernel<256><<<grid, 256, 0, s>>>(student_logits, teacher_logits, labels, loss, grad_logits, (int)vocab, eta, grad_scale);
-    CAST_CUDA_TRY(cudaGetLastError());
+        CAST_CUDA_TRY(cudaGetLastError());
+    }
     count_launch();
     return CAST_OK;
 }

@@ -6,7 +6,9 @@ allocation is not acceptable.  For them the library carries its own staging area
 library image).  This test calls that entry point through the C ABI and checks that it gives what the
 allocating entry point (cast_host_step) gives on the same inputs -- twice in a row, with a different
 shape, flags and metadata form the second time, because every call reuses the same area and must not see
-what the previous call left there.  The file name sorts last so that a run that stops at the first
+what the previous call left there -- and that the second call leaves the amount of free device memory
+untouched (the first call on a device is the one that may bring the library's device image in, which is why
+such callers make it at start-up).  The file name sorts last so that a run that stops at the first
 failure has already run every other test.
 """
 import numpy as np
@@ -71,8 +73,14 @@ def test_static_staging_matches_allocating_entry_point_on_two_calls_in_a_row():
         b = host_state(rows, cols, c["seed"], prev)
         step_with_context(a, rows, cols, N, M, h, flags)
         launches = cast.cast_kernel_launch_count()
+        free_before, _ = torch.cuda.mem_get_info()
         cast.check(step_static(b, rows, cols, N, M, h, flags, stream=(side if i else None)))
+        free_after, _ = torch.cuda.mem_get_info()
         assert cast.cast_kernel_launch_count() == launches + 1
+        if i:
+            # The first call on a device may load the part of the library that holds the staging area (CUDA loads
+            # device code lazily); every later call must leave the amount of free device memory exactly as it was.
+            assert free_after == free_before, f"the call changed free device memory by {free_before - free_after} bytes"
         got, want = outputs(b), outputs(a)
         U.assert_parity(got, want, f"call {i}: static staging vs allocated staging")
         assert got["flips"] == want["flips"] > 0
