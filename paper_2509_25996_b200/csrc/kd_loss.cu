@@ -63,21 +63,39 @@ __device__ __forceinline__ void unpack8(uint4 p, float (&f)[8])
     }
 }
 
-__device__ __forceinline__ void absorb8(RowSums& r, const float (&s)[8], const float (&t)[8])
+// Largest of the 8 bf16 values of a vector, taken on the packed pairs (three 2-wide maxima, then the two halves).
+__device__ __forceinline__ float max8_bf16(uint4 p)
 {
-    float cs = s[0], ct = t[0];
+    uint32_t m;
+    asm("{ .reg .b32 a, b;\n\t"
+        "max.bf16x2 a, %1, %2;\n\t"
+        "max.bf16x2 b, %3, %4;\n\t"
+        "max.bf16x2 %0, a, b; }" : "=r"(m) : "r"(p.x), "r"(p.y), "r"(p.z), "r"(p.w));
+    return fmaxf(__uint_as_float(m << 16), __uint_as_float(m & 0xFFFF0000u));
+}
+
+// One vector of both rows into the running sums.  Called by all lanes of a warp (there is a vote inside); a lane
+// with `have` false has no vector in this trip and leaves its sums alone.
+__device__ __forceinline__ void absorb8(RowSums& r, uint4 sp, uint4 tp, bool have)
+{
+    const float cs = max8_bf16(sp) * kLog2e, ct = max8_bf16(tp) * kLog2e;
+    // A running maximum moves in the first few vectors of a row and almost never after: the whole warp skips the
+    // rescaling with one vote instead of issuing its predicated-off instructions for every vector.
+    if (__any_sync(0xFFFFFFFFu, have && (cs > r.ms2 || ct > r.mt2))) {
+        if (have && cs > r.ms2) { r.zs *= ex2(r.ms2 - cs); r.ms2 = cs; }
+        if (have && ct > r.mt2) { const float f = ex2(r.mt2 - ct); r.zt *= f; r.a *= f; r.mt2 = ct; }
+    }
+    if (have) {
+        float s[8], t[8];
+        unpack8(sp, s);
+        unpack8(tp, t);
 #pragma unroll
-    for (int i = 1; i < 8; ++i) { cs = fmaxf(cs, s[i]); ct = fmaxf(ct, t[i]); }
-    cs *= kLog2e;
-    ct *= kLog2e;
-    if (cs > r.ms2) { r.zs *= ex2(r.ms2 - cs); r.ms2 = cs; }
-    if (ct > r.mt2) { const float f = ex2(r.mt2 - ct); r.zt *= f; r.a *= f; r.mt2 = ct; }
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        r.zs += ex2(fmaf(s[i], kLog2e, -r.ms2));
-        const float e = ex2(fmaf(t[i], kLog2e, -r.mt2));
-        r.zt += e;
-        r.a = fmaf(e, t[i] - s[i], r.a);
+        for (int i = 0; i < 8; ++i) {
+            r.zs += ex2(fmaf(s[i], kLog2e, -r.ms2));
+            const float e = ex2(fmaf(t[i], kLog2e, -r.mt2));
+            r.zt += e;
+            r.a = fmaf(e, t[i] - s[i], r.a);
+        }
     }
 }
 
@@ -148,19 +166,15 @@ __device__ __forceinline__ GradConsts grad_consts(const Finished& f, int label, 
     return g;
 }
 
-// gradient of 8 logits starting at column `col`
-__device__ __forceinline__ uint4 grad8(const float (&s)[8], const float (&t)[8], const GradConsts& k, int col, int label)
+// gradient of 8 logits, without the one-hot term (the label's owner adds it after its sweep)
+__device__ __forceinline__ uint4 grad8(uint4 sp, uint4 tp, const GradConsts& k)
 {
-    float g[8];
+    float s[8], t[8], g[8];
+    unpack8(sp, s);
+    unpack8(tp, t);
 #pragma unroll
     for (int i = 0; i < 8; ++i)
         g[i] = ex2(fmaf(s[i], kLog2e, k.off_s)) - ex2(fmaf(t[i], kLog2e, k.off_t));
-    const unsigned rel = (unsigned)(label - col);          // the label's place in this vector, if it is here
-    if (rel < 8u) {
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-            if (rel == (unsigned)i) g[i] -= k.onehot;
-    }
     return make_uint4(pack2(g[0], g[1]) ^ k.sign_bits, pack2(g[2], g[3]) ^ k.sign_bits, pack2(g[4], g[5]) ^ k.sign_bits,
                       pack2(g[6], g[7]) ^ k.sign_bits);
 }
@@ -185,11 +199,15 @@ kd_loss_kernel(const uint16_t* __restrict__ student, const uint16_t* __restrict_
     if (label >= vocab) label = -1;          // out of range: no target (never read past the row)
 
     RowSums r = {-INFINITY, 0.0f, -INFINITY, 0.0f, 0.0f};
+    // all lanes of a warp make the same number of trips (the vote inside absorb8 needs the whole warp); in the last
+    // trip some lanes may have no vector
+    const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+    const int warp_first = v0 + (int)(threadIdx.x & ~31u);
 #pragma unroll 2
-    for (int c = v0 + (int)threadIdx.x; c < v1; c += THREADS) {
-        float s[8], t[8];
-        unpack8(s_vec[c], s); unpack8(t_vec[c], t);
-        absorb8(r, s, t);
+    for (int base = warp_first; base < v1; base += THREADS) {
+        const int c = base + (int)(threadIdx.x & 31u);
+        const bool have = c < v1;
+        absorb8(r, have ? s_vec[c] : zero, have ? t_vec[c] : zero, have);
     }
     r = block_merge<THREADS>(r);
     if constexpr (CLUSTER > 1) {
@@ -211,10 +229,14 @@ kd_loss_kernel(const uint16_t* __restrict__ student, const uint16_t* __restrict_
     uint4* g_vec = reinterpret_cast<uint4*>(grad + row);
     // back to front: the second sweep starts on the part of the segment the first sweep read last
 #pragma unroll 2
-    for (int c = v1 - 1 - (int)threadIdx.x; c >= v0; c -= THREADS) {
-        float s[8], t[8];
-        unpack8(s_vec[c], s); unpack8(t_vec[c], t);
-        g_vec[c] = grad8(s, t, k, c * 8, label);
+    for (int c = v1 - 1 - (int)threadIdx.x; c >= v0; c -= THREADS) g_vec[c] = grad8(s_vec[c], t_vec[c], k);
+    // The one-hot term of the label's column: recomputed and stored by the thread that stored the label's vector
+    // (program order puts this store after that one), instead of a test in every trip of the sweep.
+    const int cv = label >> 3;                 // label < 0 gives a negative vector index: no owner
+    if (cv >= v0 && cv < v1 && (unsigned)((v1 - 1 - cv) % THREADS) == threadIdx.x) {
+        const float s = __uint_as_float((uint32_t)student[row + label] << 16), t = __uint_as_float((uint32_t)teacher[row + label] << 16);
+        const float g = ex2(fmaf(s, kLog2e, k.off_s)) - ex2(fmaf(t, kLog2e, k.off_t)) - k.onehot;
+        grad[row + label] = (uint16_t)((pack2(g, 0.0f) ^ k.sign_bits) & 0xFFFFu);
     }
 }
 
