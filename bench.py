@@ -52,6 +52,9 @@ def parse_args():
     p.add_argument("--count-flips", action="store_true")
     p.add_argument("--emit", choices=["pruned", "dense", "compressed"], default="pruned",
                    help="forward weight: pruned product in the dense layout (default), dense product, or kept entries only")
+    p.add_argument("--staging", choices=["plain", "bulk"], default="plain",
+                   help="how the step moves its tiles: per-thread 128-bit loads and stores (default), or bulk asynchronous copies "
+                        "through shared memory (2:4 headline configuration only; same results)")
     p.add_argument("--e2e-layers", type=int, default=1, help="LLaMA layers held in host memory for the e2e leg (0 = skip)")
     p.add_argument("--e2e-steps", type=int, default=4)
     p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
@@ -550,6 +553,8 @@ def cuda_arm(args):
     bytes_per_param = BYTES_PER_PARAM_FLIPS if args.count_flips else BYTES_PER_PARAM
     if args.emit == "dense":
         flags |= B.CAST_F_EMIT_DENSE
+    if args.staging == "bulk":
+        flags |= B.CAST_F_BULK_STAGING
     compressed = args.emit == "compressed"
     if compressed:
         if wl.resident_layers:
@@ -750,7 +755,7 @@ def cuda_arm(args):
     # ---- the other listed workloads (1 GPU, default headline only): reported in `configs`
     configs = None
     headline_default = (wl.name == "llama2_7b" and (N, M) == (2, 4) and args.emit == "pruned" and args.schedule == "every-step"
-                        and not args.count_flips and not args.learned_scale)
+                        and not args.count_flips and not args.learned_scale and args.staging == "plain")
     if args.configs == "all" and world == 1 and headline_default:
         configs = extra_configs(args, dev, stream, state, sampler, peak)
         del state, mats
@@ -808,14 +813,15 @@ def cuda_arm(args):
                                                                                   else "L2 flushed by a 512 MB write before every step, steps timed one by one"),
                    "resident_layers": wl.resident_layers, "streams": 2 if wl.resident_layers else 1,
                    "lr": hyper.lr, "betas": [hyper.beta1, hyper.beta2], "eps": hyper.eps, "l1_coeff": hyper.l1_coeff,
-                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "schedule": args.schedule, "learned_scale": bool(args.learned_scale), "seed": args.seed},
+                   "total_steps": wl.total_steps, "count_flips": bool(args.count_flips), "emit": args.emit, "staging": args.staging, "schedule": args.schedule, "learned_scale": bool(args.learned_scale), "seed": args.seed},
         "hbm_gbs_per_gpu": per_gpu_gbs, "frac_of_nominal_8tbs": per_gpu_gbs / NOMINAL_HBM_GBS,
         "warm_l2": (None if warm_ms_per_step is None else
                     {"ms_per_step": warm_ms_per_step, "value": wl.n_params / (warm_ms_per_step * 1e-3),
                      "note": "same steps back to back without the flush: the state stays in L2, not an HBM figure"}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}, {1 if (N, M) == (2, 4) else 0}>",
+                     "peak_kind": f"of {peak_kind}", "kernel": ("adams_nm_multi_bulk_kernel" if args.staging == "bulk" else
+                                f"adams_nm_multi_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}, {1 if (N, M) == (2, 4) else 0}>"),
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": step_launches,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,

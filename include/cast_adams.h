@@ -93,6 +93,14 @@ enum cast_flags {
                                        initial mask for the initial flip rate i_t; 0 is added where meta_ref is
                                        NULL).  Only cast_plan_step_stats takes this flag, on a plan created
                                        with it (other entry points answer CAST_ERR_PLAN)                  */
+    , CAST_F_BULK_STAGING = 1u << 8 /* an implementation switch, not part of the method: the tiles of the step are
+                                       staged through shared memory by bulk asynchronous copies (and stored back
+                                       the same way) instead of per-thread 128-bit loads and stores.  Results are
+                                       identical bit for bit.  Exists for 2:4 with CAST_F_RESELECT and index-form
+                                       metadata alone (the headline configuration); any other combination with
+                                       this bit answers CAST_ERR_NM.  Kept so that the two ways of moving the
+                                       data can be measured against each other; the plain form is the faster one
+                                       on B200 (see cast_bulk_timeout_count for its one failure mode)         */
 };
 
 /*
@@ -414,6 +422,11 @@ CAST_API int cast_host_step_static(float* w, float* m, float* v, const cast_bf16
 CAST_API int cast_probe_launch(int64_t n_ctas, cast_stream_t stream);
 CAST_API int cast_probe_stream(float* w, float* m, float* v, const cast_bf16* g, cast_bf16* w_fwd, uint32_t* meta,
                       int64_t n_params, cast_stream_t stream);
+
+/* Steps with CAST_F_BULK_STAGING wait for their bulk copies with a bounded number of polls; a tile whose data
+ * has not arrived by then is not updated and is counted.  *count_out receives that count over the life of the
+ * process on the current device (0 in every healthy run).  Synchronises the device. */
+CAST_API int cast_bulk_timeout_count(unsigned long long* count_out);
 
 /* Static description of a status code (never NULL). */
 CAST_API const char* cast_strerror(int status);

@@ -35,13 +35,14 @@ CAST_F_EMIT_DENSE = 1 << 4
 CAST_F_EMIT_COMPRESSED = 1 << 5
 CAST_F_GRAD_OF_SCALED = 1 << 6
 CAST_F_MASK_STATS = 1 << 7
+CAST_F_BULK_STAGING = 1 << 8
 
 EXPORTS = (
     "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_scale_adam_step",
     "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_step_stats", "cast_plan_destroy",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
-    "cast_probe_launch", "cast_probe_stream",
+    "cast_probe_launch", "cast_probe_stream", "cast_bulk_timeout_count",
     "cast_strerror", "cast_last_cuda_error", "cast_kernel_launch_count",
 )
 
@@ -137,6 +138,8 @@ def load_library() -> ctypes.CDLL:
     lib.cast_plan_mask_stats.restype = ctypes.c_int
     lib.cast_plan_mask_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_uint32, ctypes.c_void_p,
                                          ctypes.c_void_p]
+    lib.cast_bulk_timeout_count.restype = ctypes.c_int
+    lib.cast_bulk_timeout_count.argtypes = [ctypes.POINTER(ctypes.c_ulonglong)]
     lib.cast_probe_launch.restype = ctypes.c_int
     lib.cast_probe_launch.argtypes = [ctypes.c_int64, ctypes.c_void_p]
     lib.cast_probe_stream.restype = ctypes.c_int
@@ -335,6 +338,13 @@ def cast_plan_mask_stats(plan, meta_refs, flags, stats, stream=None) -> int:
     if meta_refs is not None:
         arr = (ctypes.c_void_p * len(meta_refs))(*[_ptr(r) for r in meta_refs])
     return load_library().cast_plan_mask_stats(plan, arr, int(flags), _ptr(stats), _stream(stream))
+
+
+def cast_bulk_timeout_count():
+    """Returns (status, count)."""
+    out = ctypes.c_ulonglong(0)
+    rc = load_library().cast_bulk_timeout_count(ctypes.byref(out))
+    return rc, int(out.value)
 
 
 def cast_probe_launch(n_ctas, stream=None) -> int:

@@ -1,0 +1,170 @@
+// The headline step (2:4, kept set selected now, index-form metadata) with its tiles staged through shared memory by
+// bulk asynchronous copies instead of per-thread 128-bit loads and stores (CAST_F_BULK_STAGING).  Same arithmetic
+// (compute_unit of the plain kernel), same results bit for bit; it exists so that the two ways of moving the data can
+// be measured against each other on the device at hand.
+//
+// Per CTA (128 threads, one tile of 1024 parameters): one elected thread arms an mbarrier with the tile's byte count
+// and issues four bulk copies global -> shared (w, m, v: 4 KB each, g: 2 KB; this GPU's own memory, no multicast);
+// all threads wait on the barrier's phase, compute from shared memory, write w, m, v and the forward weight back
+// into the same shared memory, make those writes visible to the asynchronous proxy, and the elected thread issues
+// four bulk copies shared -> global and waits until they have read the shared memory.  The metadata byte goes out by
+// an ordinary store.  16 KB of shared memory per CTA, 7 CTAs per SM as in the plain kernel.
+//
+// The wait on the barrier is bounded (a phase that has not completed after 2^16 polls with back-off, about 2 ms, is counted in a
+// device-side error counter, the CTA waits once more with the same limit and gives up without storing); the host
+// reads the counter with cast_bulk_timeout_count().  Every copy starts on a 16-byte boundary (tiles start at
+// multiples of 1024 elements of 16-byte aligned buffers) and has a size that is a multiple of 16 bytes.
+#include "cast_internal.h"
+
+namespace cast {
+namespace {
+
+constexpr uint32_t kBulkFlagWord = kReselect;
+constexpr uint32_t kPollLimit = 1u << 16;      // ~2 ms with the back-off below; a tile's copies take microseconds
+
+__device__ unsigned long long g_bulk_timeouts;      // phases given up on, over the life of the process
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void barrier_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void barrier_expect(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool barrier_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{ .reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p; }" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done != 0;
+}
+// Polls the phase with a limit; false if it gave up.
+__device__ __forceinline__ bool barrier_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < kPollLimit; ++i) {
+        if (barrier_try_wait(bar, parity)) return true;
+        if (i > 64) __nanosleep(32);
+    }
+    return false;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void* dst, uint32_t src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src_smem), "r"(bytes) : "memory");
+}
+
+struct __align__(128) BulkTile {
+    float w[kTileUnits * kUnitElems];
+    float m[kTileUnits * kUnitElems];
+    float v[kTileUnits * kUnitElems];
+    uint16_t g[kTileUnits * kUnitElems];       // gradient in, forward weight out
+    unsigned long long barrier;
+};
+
+__device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts& c, uint32_t first_unit)
+{
+    __shared__ BulkTile tile;
+    const uint32_t units = min((uint32_t)kTileUnits, t.n_units - first_unit);       // a matrix's last tile may be short
+    const size_t e0 = (size_t)first_unit * kUnitElems;
+    const uint32_t bar = smem_addr(&tile.barrier);
+    if (threadIdx.x == 0) {
+        barrier_init(bar, 1);
+        const uint32_t b4 = units * kUnitElems * 4u, b2 = units * kUnitElems * 2u;
+        barrier_expect(bar, 3u * b4 + b2);
+        bulk_load(smem_addr(tile.w), t.w + e0, b4, bar);
+        bulk_load(smem_addr(tile.m), t.m + e0, b4, bar);
+        bulk_load(smem_addr(tile.v), t.v + e0, b4, bar);
+        bulk_load(smem_addr(tile.g), t.g + e0, b2, bar);
+    }
+    __syncthreads();                            // the barrier is initialised before anyone polls it
+    bool arrived = barrier_wait_bounded(bar, 0);
+    if (!arrived) {
+        if (threadIdx.x == 0) atomicAdd(&g_bulk_timeouts, 1ull);
+        arrived = barrier_wait_bounded(bar, 0); // the copies may still land: give them the same time again
+    }
+    if (!__syncthreads_and(arrived)) return;    // nothing is stored for a tile whose data did not arrive
+
+    const uint32_t u_idx = threadIdx.x;
+    const bool active = u_idx < units;
+    UnitRegs u;
+    float a = 1.0f;
+    if (active) {
+        const float4 w0 = *reinterpret_cast<const float4*>(tile.w + u_idx * 8), w1 = *reinterpret_cast<const float4*>(tile.w + u_idx * 8 + 4);
+        const float4 m0 = *reinterpret_cast<const float4*>(tile.m + u_idx * 8), m1 = *reinterpret_cast<const float4*>(tile.m + u_idx * 8 + 4);
+        const float4 v0 = *reinterpret_cast<const float4*>(tile.v + u_idx * 8), v1 = *reinterpret_cast<const float4*>(tile.v + u_idx * 8 + 4);
+        u.g = *reinterpret_cast<const uint4*>(tile.g + u_idx * 8);
+        if (t.scale != nullptr) a = __ldg(t.scale + (uint32_t)(((uint64_t)(first_unit + u_idx) * t.seg_magic) >> t.seg_shift));
+        u.w[0] = w0.x; u.w[1] = w0.y; u.w[2] = w0.z; u.w[3] = w0.w; u.w[4] = w1.x; u.w[5] = w1.y; u.w[6] = w1.z; u.w[7] = w1.w;
+        u.m[0] = m0.x; u.m[1] = m0.y; u.m[2] = m0.z; u.m[3] = m0.w; u.m[4] = m1.x; u.m[5] = m1.y; u.m[6] = m1.z; u.m[7] = m1.w;
+        u.v[0] = v0.x; u.v[1] = v0.y; u.v[2] = v0.z; u.v[3] = v0.w; u.v[4] = v1.x; u.v[5] = v1.y; u.v[6] = v1.z; u.v[7] = v1.w;
+        u.prev_byte = 0;
+        u.ref_byte = 0;
+        float gw_sum;
+        UnitSums sums;
+        compute_unit<4, kBulkFlagWord, true>(u, c, a, false, gw_sum, sums);
+        *reinterpret_cast<float4*>(tile.w + u_idx * 8) = make_float4(u.w[0], u.w[1], u.w[2], u.w[3]);
+        *reinterpret_cast<float4*>(tile.w + u_idx * 8 + 4) = make_float4(u.w[4], u.w[5], u.w[6], u.w[7]);
+        *reinterpret_cast<float4*>(tile.m + u_idx * 8) = make_float4(u.m[0], u.m[1], u.m[2], u.m[3]);
+        *reinterpret_cast<float4*>(tile.m + u_idx * 8 + 4) = make_float4(u.m[4], u.m[5], u.m[6], u.m[7]);
+        *reinterpret_cast<float4*>(tile.v + u_idx * 8) = make_float4(u.v[0], u.v[1], u.v[2], u.v[3]);
+        *reinterpret_cast<float4*>(tile.v + u_idx * 8 + 4) = make_float4(u.v[4], u.v[5], u.v[6], u.v[7]);
+        *reinterpret_cast<uint4*>(tile.g + u_idx * 8) = u.g;
+        reinterpret_cast<uint8_t*>(t.meta)[first_unit + u_idx] = (uint8_t)u.meta_byte;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's shared-memory writes, for the bulk stores
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t b4 = units * kUnitElems * 4u, b2 = units * kUnitElems * 2u;
+        bulk_store(t.w + e0, smem_addr(tile.w), b4);
+        bulk_store(t.m + e0, smem_addr(tile.m), b4);
+        bulk_store(t.v + e0, smem_addr(tile.v), b4);
+        bulk_store(t.w_fwd + e0, smem_addr(tile.g), b2);
+        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the shared memory has been read: the CTA may end
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c)
+{
+    bulk_tile(t, c, blockIdx.x * kTileUnits);
+}
+
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+adams_nm_multi_bulk_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c)
+{
+    const uint32_t tile = blockIdx.x;
+    uint32_t k = p.hint[tile >> p.hint_shift];
+    while (tile >= p.tile_start[k + 1]) ++k;
+    bulk_tile(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits);
+}
+
+}  // namespace
+
+bool bulk_variant_exists(int M, int n_keep, uint32_t flag_word) { return M == 4 && n_keep == 2 && flag_word == kBulkFlagWord; }
+
+int launch_bulk(const StepLaunch& a)
+{
+    if (a.single) adams_nm_bulk_kernel<<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c);
+    else adams_nm_multi_bulk_kernel<<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(*a.multi, *a.c);
+    CAST_CUDA_TRY(cudaGetLastError());
+    return CAST_OK;
+}
+
+}  // namespace cast
+
+extern "C" int cast_bulk_timeout_count(unsigned long long* count_out)
+{
+    if (!count_out) return CAST_ERR_NULL;
+    CAST_CUDA_TRY(cudaMemcpyFromSymbol(count_out, cast::g_bulk_timeouts, sizeof(unsigned long long)));
+    return CAST_OK;
+}

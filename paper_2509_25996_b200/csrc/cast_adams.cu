@@ -29,7 +29,7 @@ int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count)
     if (!(flags & CAST_F_META_BITMASK) && !(N == 2 && M == 4)) return CAST_ERR_NM;
     const uint32_t known = CAST_F_RESELECT | CAST_F_COUNT_FLIPS | CAST_F_META_BITMASK |
                            CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE | CAST_F_EMIT_COMPRESSED |
-                           CAST_F_GRAD_OF_SCALED | CAST_F_MASK_STATS;
+                           CAST_F_GRAD_OF_SCALED | CAST_F_MASK_STATS | CAST_F_BULK_STAGING;
     if (flags & ~known) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && (flags & CAST_F_EMIT_DENSE)) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && M > kUnitElems) return CAST_ERR_NM;
@@ -177,6 +177,10 @@ static const StepLauncher kStepLaunchers[6][4] = {
 #undef CAST_SLICE
 #undef CAST_SLICES_OF
 
+// bulk_step.cu: the headline step staged through shared memory by bulk copies
+bool bulk_variant_exists(int M, int n_keep, uint32_t flag_word);
+int launch_bulk(const StepLaunch& a);
+
 uint32_t kernel_flag_word(uint32_t flags)
 {
     uint32_t f = flags & kCompileTimeFlags;
@@ -192,6 +196,12 @@ int launch_step(const StepLaunch& a, int M)
     if (!step_kernel_exists(M, two_four, f)) return CAST_ERR_NM;
     if (a.single ? tiles_of(*a.single) == 0 : a.multi->tile_start[a.multi->n_tensors] == 0) return CAST_OK;
     if (a.single && tiles_of(*a.single) > kMaxTiles) return CAST_ERR_SHAPE;
+    if (a.c->flags & CAST_F_BULK_STAGING) {
+        if (!bulk_variant_exists(M, a.c->n_keep, f)) return CAST_ERR_NM;      // staged form: the headline configuration only
+        const int brc = launch_bulk(a);
+        if (brc == CAST_OK) g_launches.fetch_add(1, std::memory_order_relaxed);
+        return brc;
+    }
     int row = -1;
     switch (M) {
         case 2:  row = 0; break;

@@ -34,16 +34,21 @@ constexpr int kPruneTileUnits = kThreads * kPruneUnitsPerThread;      // 512 uni
 
 // A CTA of the step moves 28 KB; this pass moves 6 bytes per parameter, so a CTA takes four times the
 // parameters (with one unit per thread the grid launched CTAs faster than they could be scheduled).
-template <int M>
+// The flag word (reselect, metadata form, compressed output) and "N:M is 2:4" are template arguments, as in the
+// step: the integer work per parameter (compares, keep bits, index nibbles) is what this kernel is bound by
+// besides HBM, so nothing is decided at run time and only what a configuration needs is computed.
+template <int M, uint32_t F, bool TF>
 __global__ void __launch_bounds__(kThreads)
-prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t flags)
+prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep)
 {
+    constexpr bool reselect = (F & kReselect) != 0, bitmask = (F & kMetaBitmask) != 0, compressed = (F & kEmitCompressed) != 0;
+    static_assert(TF || bitmask, "index-form metadata is 2:4 only");
+    static_assert(!compressed || M <= 8, "the compressed form needs the group in one thread");
     const uint32_t tile = blockIdx.x;
     uint32_t k = p.hint[tile >> p.hint_shift];
     while (tile >= p.tile_start[k + 1]) ++k;
     const PruneDesc& t = p.desc[k];
     const uint32_t first = (tile - p.tile_start[k]) * kPruneTileUnits + threadIdx.x;
-    const bool bitmask = (flags & kMetaBitmask) != 0;
     float x[kPruneUnitsPerThread][8];
     float a[kPruneUnitsPerThread];
     uint32_t stored[kPruneUnitsPerThread];
@@ -57,7 +62,7 @@ prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t fl
         if (unit < t.n_units) {
             const float4 lo = ld_f4(t.w + (size_t)unit * kUnitElems), hi = ld_f4(t.w + (size_t)unit * kUnitElems + 4);
             x[j][0] = lo.x; x[j][1] = lo.y; x[j][2] = lo.z; x[j][3] = lo.w; x[j][4] = hi.x; x[j][5] = hi.y; x[j][6] = hi.z; x[j][7] = hi.w;
-            if (!(flags & kReselect)) stored[j] = t.meta[unit];
+            if constexpr (!reselect) stored[j] = t.meta[unit];
             if (t.scale != nullptr) a[j] = __ldg(t.scale + (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift));
         }
     }
@@ -65,18 +70,32 @@ prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t fl
     for (int j = 0; j < kPruneUnitsPerThread; ++j) {
         const uint32_t unit = first + j * kThreads;
         const bool active = unit < t.n_units;
-        uint32_t ab[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) ab[i] = abs_bits(x[j][i]);
         bool kept[8];
-        uint32_t keep = 0;
-        const bool fast_2of4 = (flags & kReselect) && M == 4 && n_keep == 2;      // uniform
-        if (fast_2of4) {                                                          // the predicate network of the step
+        uint32_t keep = 0, meta_byte;
+        if constexpr (reselect && TF) {                                           // the predicate network of the step
+            uint32_t ab[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ab[i] = abs_bits(x[j][i]);
             select_2of4(ab, kept);
             select_2of4(ab + 4, kept + 4);
+            if constexpr (bitmask) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) keep |= (kept[i] ? 1u : 0u) << i;
+                meta_byte = keep;
+            } else {
+                meta_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);   // kept positions, lo | hi << 2 per group
+            }
         } else {
-            if (flags & kReselect) keep = select_top_n<M>(ab, n_keep);           // uniform branch: all lanes shuffle
-            else keep = keep_from_meta_byte(stored[j], bitmask);
+            if constexpr (reselect) {
+                uint32_t ab[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) ab[i] = abs_bits(x[j][i]);
+                keep = select_top_n<M>(ab, n_keep);                               // all lanes shuffle for M > 8
+                meta_byte = keep;
+            } else {
+                keep = keep_from_meta_byte(stored[j], bitmask);
+                meta_byte = stored[j];
+            }
 #pragma unroll
             for (int i = 0; i < 8; ++i) kept[i] = (keep >> i) & 1u;
         }
@@ -85,32 +104,65 @@ prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep, uint32_t fl
 #pragma unroll
         for (int i = 0; i < 8; ++i) f[i] = kept[i] ? a[j] * x[j][i] : 0.0f;
         const uint4 packed = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
-        const uint32_t idx_byte = idx2_from_kept(kept) | (idx2_from_kept(kept + 4) << 4);   // kept positions, lo | hi << 2 per group
-        if (fast_2of4 && bitmask) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) keep |= (kept[i] ? 1u : 0u) << i;
-        }
-        bool compressed = false;
-        if constexpr (M <= 8) compressed = (flags & kEmitCompressed) != 0;
-        if (compressed && M == 4 && n_keep == 2)
+        if constexpr (!compressed) {
+            *reinterpret_cast<uint4*>(t.out + (size_t)unit * kUnitElems) = packed;
+        } else if constexpr (TF && !bitmask) {
             *reinterpret_cast<uint2*>(t.out + (size_t)unit * 4) =
-                make_uint2(kept_pair_by_index(packed.x, packed.y, idx_byte & 3u, (idx_byte >> 2) & 3u),
-                           kept_pair_by_index(packed.z, packed.w, (idx_byte >> 4) & 3u, idx_byte >> 6));
-        else if (compressed) store_kept_values<M>(t.out, unit, keep, packed, n_keep);
-        else *reinterpret_cast<uint4*>(t.out + (size_t)unit * kUnitElems) = packed;
-        t.meta[unit] = (uint8_t)(bitmask ? keep : idx_byte);
+                make_uint2(kept_pair_by_index(packed.x, packed.y, meta_byte & 3u, (meta_byte >> 2) & 3u),
+                           kept_pair_by_index(packed.z, packed.w, (meta_byte >> 4) & 3u, meta_byte >> 6));
+        } else if constexpr (TF) {
+            *reinterpret_cast<uint2*>(t.out + (size_t)unit * 4) =
+                make_uint2(kept_pair_2of4(packed.x, packed.y, meta_byte & 0xFu), kept_pair_2of4(packed.z, packed.w, meta_byte >> 4));
+        } else {
+            store_kept_values<M>(t.out, unit, keep, packed, n_keep);
+        }
+        t.meta[unit] = (uint8_t)meta_byte;
     }
 }
 
 inline uint32_t prune_tiles(uint32_t n_units) { return (n_units + kPruneTileUnits - 1) / kPruneTileUnits; }
 
-template <int M>
-int launch_t(const PruneParams& p, int N, uint32_t flags, cudaStream_t s)
+template <int M, uint32_t F, bool TF>
+int launch_f(const PruneParams& p, int N, cudaStream_t s)
 {
-    prune_fold_kernel<M><<<p.tile_start[p.n_tensors], kThreads, 0, s>>>(p, N, flags);
+    prune_fold_kernel<M, F, TF><<<p.tile_start[p.n_tensors], kThreads, 0, s>>>(p, N);
     CAST_CUDA_TRY(cudaGetLastError());
     count_launch();
     return CAST_OK;
+}
+
+// Picks the instantiation of (flags, 2:4 or not) for one group size.
+template <int M>
+int launch_t(const PruneParams& p, int N, uint32_t flags, cudaStream_t s)
+{
+    constexpr uint32_t RS = kReselect, BM = kMetaBitmask, CP = kEmitCompressed;
+    const bool two_four = M == 4 && N == 2;
+    if constexpr (M == 4) {
+        if (two_four) {
+            switch (flags) {
+                case 0u:           return launch_f<4, 0u, true>(p, N, s);
+                case RS:           return launch_f<4, RS, true>(p, N, s);
+                case BM:           return launch_f<4, BM, true>(p, N, s);
+                case RS | BM:      return launch_f<4, RS | BM, true>(p, N, s);
+                case CP:           return launch_f<4, CP, true>(p, N, s);
+                case RS | CP:      return launch_f<4, RS | CP, true>(p, N, s);
+                case BM | CP:      return launch_f<4, BM | CP, true>(p, N, s);
+                case RS | BM | CP: return launch_f<4, RS | BM | CP, true>(p, N, s);
+            }
+            return CAST_ERR_HYPER;
+        }
+    }
+    switch (flags) {
+        case BM:           return launch_f<M, BM, false>(p, N, s);
+        case RS | BM:      return launch_f<M, RS | BM, false>(p, N, s);
+    }
+    if constexpr (M <= 8) {
+        switch (flags) {
+            case BM | CP:      return launch_f<M, BM | CP, false>(p, N, s);
+            case RS | BM | CP: return launch_f<M, RS | BM | CP, false>(p, N, s);
+        }
+    }
+    return CAST_ERR_NM;
 }
 
 int launch(PruneParams* p, int N, int M, uint32_t flags, cudaStream_t s)

@@ -326,3 +326,32 @@ def test_device_pointer_kind_is_checked():
     rc = cast.cast_adams_step(host_w, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view,
                               None, 1, 4, 64, 2, 4, 1e-4, 0.9, 0.95, 1e-8, 1e-3, 1, 10, RS, None, None)
     assert rc == B.CAST_ERR_MEMORY and cast.cast_kernel_launch_count() == before
+
+
+@pytest.mark.parametrize("rows,cols", [(1, 32), (3, 64), (7, 2080), (64, 4096)])
+def test_bulk_staged_variant_gives_the_same_bits(rows, cols):
+    """CAST_F_BULK_STAGING moves the tiles with bulk asynchronous copies through shared memory; the arithmetic is the
+    plain kernel's, so every output is identical bit for bit, short last tiles included (7 x 2080 = 14.2 tiles), and
+    no wait on a copy ever ran out."""
+    inp = inputs(rows, cols, seed=31)
+    h = Hyper()
+    plain = U.run_cuda_single(inp, 2, 4, h, RS)
+    staged = U.run_cuda_single(inp, 2, 4, h, RS | B.CAST_F_BULK_STAGING)
+    for k in ("w", "m", "v", "w_fwd", "meta"):
+        assert np.array_equal(plain[k].view(np.uint8), staged[k].view(np.uint8)), k
+    U.assert_parity(staged, U.run_oracle(inp, 2, 4, h, RS), f"bulk staging {rows}x{cols}")
+    rc, timeouts = cast.cast_bulk_timeout_count()
+    assert rc == 0 and timeouts == 0
+
+
+def test_bulk_staging_exists_for_the_headline_configuration_only():
+    inp = inputs(4, 64, seed=32)
+    st = U.to_device(inp, DEV)
+    before = cast.cast_kernel_launch_count()
+    lr, b1, b2, eps, lam = Hyper().as_f32()
+    for N, M, flags in ((2, 4, RS | BM), (2, 4, 0), (4, 8, RS | BM), (2, 4, RS | B.CAST_F_COUNT_FLIPS)):
+        flips = torch.zeros(1, dtype=torch.int64, device=DEV)
+        rc = cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale, 2, 4, 64, N, M,
+                                  lr, b1, b2, eps, lam, 1000, 30000, flags | B.CAST_F_BULK_STAGING, flips, None)
+        assert rc == B.CAST_ERR_NM
+    assert cast.cast_kernel_launch_count() == before

@@ -392,3 +392,24 @@ def test_host_step_pageable_memory():
     got = dict(w=inp.w.numpy(), m=inp.m.numpy(), v=inp.v.numpy(), w_fwd=workloads.bf16_bits(fwd),
                meta=meta.numpy().view(np.uint32))
     U.assert_parity(got, ref, "pageable")
+
+
+def test_plan_with_bulk_staging_gives_the_same_bits():
+    """All matrices of a plan in one launch of the staged variant: identical to the plain launch."""
+    from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
+    shapes = [(24, 256), (7, 2080), (3, 1056), (40, 512)]
+    a = DeviceModelState(shapes, 2, 4, seed=6, device="cuda:0", scale_mode="jitter")
+    b = DeviceModelState(shapes, 2, 4, seed=6, device="cuda:0", scale_mode="jitter")
+    h = RunHyper(total_steps=30000)
+    for _ in range(2):
+        a.step(h, B.CAST_F_RESELECT)
+        b.step(h, B.CAST_F_RESELECT | B.CAST_F_BULK_STAGING)
+        h.step += 1
+    torch.cuda.synchronize()
+    for x, y in zip(a.mats, b.mats):
+        for k in ("w", "m", "v", "w_fwd", "meta"):
+            assert torch.equal(getattr(x, k), getattr(y, k)), k
+    rc, timeouts = cast.cast_bulk_timeout_count()
+    assert rc == 0 and timeouts == 0
+    a.close()
+    b.close()
