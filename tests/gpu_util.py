@@ -75,7 +75,8 @@ def host_arrays(inp: workloads.TensorInputs):
 
 
 def oracle_flags(flags: int) -> int:
-    """The two flag sets use the same numbering; translated name by name so a renumbering would show."""
+    """The two flag sets use the same numbering; translated name by name so a renumbering would show.  Flags that
+    only choose an implementation (bulk staging) or ask for extra outputs (statistics) have no oracle counterpart."""
     out = 0
     for lib_bit, orc_bit in ((B.CAST_F_RESELECT, orc.F_RESELECT), (B.CAST_F_COUNT_FLIPS, orc.F_COUNT_FLIPS),
                              (B.CAST_F_META_BITMASK, orc.F_META_BITMASK), (B.CAST_F_V_KEPT_FROM_G, orc.F_V_KEPT_FROM_G),

@@ -262,3 +262,11 @@ def test_llama2_7b_whole_set_4_8_with_flips_every_element():
     """The same set under 4:8 with flip counting (bitmask metadata) against seeded previous-mask words: every element,
     and the flip total of the one launch equals the oracle's sum over all matrices."""
     _whole_set("llama2_7b", 4, 8, B.CAST_F_RESELECT | B.CAST_F_META_BITMASK | B.CAST_F_COUNT_FLIPS, True, need_gb=125)
+
+
+def test_llama2_7b_whole_set_bulk_staging_every_element():
+    """The headline launch in its bulk-staged form (tiles moved by bulk asynchronous copies through shared memory):
+    every element of the 6,476,005,376-parameter set against the oracle, and no wait on a copy ran out."""
+    _whole_set("llama2_7b", 2, 4, B.CAST_F_RESELECT | B.CAST_F_BULK_STAGING, False, need_gb=125)
+    rc, timeouts = cast.cast_bulk_timeout_count()
+    assert rc == 0 and timeouts == 0
