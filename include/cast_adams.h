@@ -96,11 +96,13 @@ enum cast_flags {
     , CAST_F_BULK_STAGING = 1u << 8 /* an implementation switch, not part of the method: the tiles of the step are
                                        staged through shared memory by bulk asynchronous copies (and stored back
                                        the same way) instead of per-thread 128-bit loads and stores.  Results are
-                                       identical bit for bit.  Exists for 2:4 with CAST_F_RESELECT and index-form
-                                       metadata alone (the headline configuration); any other combination with
-                                       this bit answers CAST_ERR_NM.  Kept so that the two ways of moving the
-                                       data can be measured against each other; the plain form is the faster one
-                                       on B200 (see cast_bulk_timeout_count for its one failure mode)         */
+                                       identical bit for bit.  Built for: 2:4 with any of CAST_F_RESELECT,
+                                       CAST_F_COUNT_FLIPS, CAST_F_META_BITMASK, CAST_F_EMIT_DENSE (not dense and
+                                       bitmask together); 4:8 and 1:4 (groups of 4 or 8) with CAST_F_RESELECT |
+                                       CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS.  Any other
+                                       combination with this bit answers CAST_ERR_NM.  As fast as the plain form
+                                       in short runs and ~2 % faster in sustained ones on B200; its one failure
+                                       mode is described at cast_bulk_timeout_count                          */
 };
 
 /*

@@ -179,7 +179,7 @@ static const StepLauncher kStepLaunchers[6][4] = {
 
 // bulk_step.cu: the headline step staged through shared memory by bulk copies
 bool bulk_variant_exists(int M, int n_keep, uint32_t flag_word);
-int launch_bulk(const StepLaunch& a);
+int launch_bulk(const StepLaunch& a, int M, uint32_t flag_word);
 
 uint32_t kernel_flag_word(uint32_t flags)
 {
@@ -197,8 +197,8 @@ int launch_step(const StepLaunch& a, int M)
     if (a.single ? tiles_of(*a.single) == 0 : a.multi->tile_start[a.multi->n_tensors] == 0) return CAST_OK;
     if (a.single && tiles_of(*a.single) > kMaxTiles) return CAST_ERR_SHAPE;
     if (a.c->flags & CAST_F_BULK_STAGING) {
-        if (!bulk_variant_exists(M, a.c->n_keep, f)) return CAST_ERR_NM;      // staged form: the headline configuration only
-        const int brc = launch_bulk(a);
+        if (!bulk_variant_exists(M, a.c->n_keep, f)) return CAST_ERR_NM;      // not one of the configurations the staged form is built for
+        const int brc = launch_bulk(a, M, f);
         if (brc == CAST_OK) g_launches.fetch_add(1, std::memory_order_relaxed);
         return brc;
     }

@@ -328,30 +328,41 @@ def test_device_pointer_kind_is_checked():
     assert rc == B.CAST_ERR_MEMORY and cast.cast_kernel_launch_count() == before
 
 
-@pytest.mark.parametrize("rows,cols", [(1, 32), (3, 64), (7, 2080), (64, 4096)])
-def test_bulk_staged_variant_gives_the_same_bits(rows, cols):
+BULK_CASES = [(2, 4, RS), (2, 4, RS | B.CAST_F_COUNT_FLIPS), (2, 4, RS | BM), (2, 4, RS | BM | B.CAST_F_COUNT_FLIPS),
+              (2, 4, RS | B.CAST_F_EMIT_DENSE), (2, 4, RS | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE), (2, 4, 0), (2, 4, B.CAST_F_EMIT_DENSE),
+              (2, 4, B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE),
+              (1, 4, RS | BM), (3, 4, RS | BM | B.CAST_F_COUNT_FLIPS), (4, 8, RS | BM), (4, 8, RS | BM | B.CAST_F_COUNT_FLIPS), (1, 8, RS | BM)]
+
+
+@pytest.mark.parametrize("N,M,flags", BULK_CASES)
+@pytest.mark.parametrize("rows,cols", [(1, 32), (7, 2080), (64, 4096)])
+def test_bulk_staged_variant_gives_the_same_bits(N, M, flags, rows, cols):
     """CAST_F_BULK_STAGING moves the tiles with bulk asynchronous copies through shared memory; the arithmetic is the
     plain kernel's, so every output is identical bit for bit, short last tiles included (7 x 2080 = 14.2 tiles), and
     no wait on a copy ever ran out."""
     inp = inputs(rows, cols, seed=31)
     h = Hyper()
-    plain = U.run_cuda_single(inp, 2, 4, h, RS)
-    staged = U.run_cuda_single(inp, 2, 4, h, RS | B.CAST_F_BULK_STAGING)
+    enc = flags & BM
+    prev = U.run_oracle(inputs(rows, cols, seed=33), N, M, Hyper(lr=0.0), RS | enc)["meta"]      # stored / previous mask
+    plain = U.run_cuda_single(inp, N, M, h, flags, meta_in=prev)
+    staged = U.run_cuda_single(inp, N, M, h, flags | B.CAST_F_BULK_STAGING, meta_in=prev)
     for k in ("w", "m", "v", "w_fwd", "meta"):
         assert np.array_equal(plain[k].view(np.uint8), staged[k].view(np.uint8)), k
-    U.assert_parity(staged, U.run_oracle(inp, 2, 4, h, RS), f"bulk staging {rows}x{cols}")
+    if flags & B.CAST_F_COUNT_FLIPS:
+        assert plain["flips"] == staged["flips"]
+    U.assert_parity(staged, U.run_oracle(inp, N, M, h, flags, meta_in=prev), f"bulk staging {N}:{M} flags {flags:#x} {rows}x{cols}")
     rc, timeouts = cast.cast_bulk_timeout_count()
     assert rc == 0 and timeouts == 0
 
 
-def test_bulk_staging_exists_for_the_headline_configuration_only():
+def test_bulk_staging_answers_nm_error_where_it_is_not_built():
     inp = inputs(4, 64, seed=32)
     st = U.to_device(inp, DEV)
     before = cast.cast_kernel_launch_count()
     lr, b1, b2, eps, lam = Hyper().as_f32()
-    for N, M, flags in ((2, 4, RS | BM), (2, 4, 0), (4, 8, RS | BM), (2, 4, RS | B.CAST_F_COUNT_FLIPS)):
-        flips = torch.zeros(1, dtype=torch.int64, device=DEV)
+    for N, M, flags in ((2, 4, RS | B.CAST_F_EMIT_COMPRESSED), (2, 4, RS | B.CAST_F_GRAD_OF_SCALED), (8, 16, RS | BM),
+                        (2, 4, RS | B.CAST_F_V_KEPT_FROM_G), (2, 4, BM | B.CAST_F_EMIT_DENSE)):
         rc = cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale, 2, 4, 64, N, M,
-                                  lr, b1, b2, eps, lam, 1000, 30000, flags | B.CAST_F_BULK_STAGING, flips, None)
-        assert rc == B.CAST_ERR_NM
+                                  lr, b1, b2, eps, lam, 1000, 30000, flags | B.CAST_F_BULK_STAGING, None, None)
+        assert rc == B.CAST_ERR_NM, (N, M, hex(flags))
     assert cast.cast_kernel_launch_count() == before
