@@ -53,10 +53,10 @@ def parse_args():
     p.add_argument("--emit", choices=["pruned", "dense", "compressed"], default="pruned",
                    help="forward weight: pruned product in the dense layout (default), dense product, or kept entries only")
     p.add_argument("--staging", choices=["auto", "plain", "bulk"], default="auto",
-                   help="how the step moves its tiles: plain = per-thread 128-bit loads and stores (the library's default), bulk = "
-                        "bulk asynchronous copies through shared memory (CAST_F_BULK_STAGING: exists for the 2:4 headline "
-                        "configuration only; same results bit for bit; measured ~2 %% faster in sustained runs under the power cap). "
-                        "auto (default) = bulk where it exists, plain elsewhere")
+                   help="how the step moves its tiles: plain = per-thread 128-bit loads and stores (CAST_F_PLAIN_ACCESS), bulk = "
+                        "bulk asynchronous copies through shared memory (CAST_F_BULK_STAGING; same results bit for bit; 2-7 %% "
+                        "faster in sustained runs under the power cap).  auto (default) = what the library's plans choose: "
+                        "bulk where it is built, plain elsewhere")
     p.add_argument("--e2e-layers", type=int, default=1, help="LLaMA layers held in host memory for the e2e leg (0 = skip)")
     p.add_argument("--e2e-steps", type=int, default=4)
     p.add_argument("--cpu-baseline", type=int, default=1, help="0 = skip the oracle timing leg")
@@ -302,13 +302,13 @@ def extra_configs(args, dev, stream, state_7b, sampler, peak):
         torch.cuda.synchronize(dev)
         return a.elapsed_time(b) / steps
 
-    # ---- config 3 once more with the library's default access path (per-thread loads and stores): the headline line
-    # above is the bulk-staged variant of the same step
+    # ---- config 3 once more with the plain access path (per-thread loads and stores, CAST_F_PLAIN_ACCESS): the headline
+    # line above takes the staged path, as plan steps do by default
     wl7 = workloads.workload("llama2_7b")
     picks = sorted({0, len(wl7.shapes) // 2, len(wl7.shapes) - 1})
     h = Hyper(l1_coeff=args.l1_coeff, step=2000, total_steps=wl7.total_steps)
     before = {t: _rows(state_7b.mats[t], 0, sample_rows, ("w", "m", "v", "g", "scale")) for t in picks}
-    state_7b.step(h, RS, stream)
+    state_7b.step(h, RS | B.CAST_F_PLAIN_ACCESS, stream)
     torch.cuda.synchronize(dev)
     parity_ok = True
     for t in picks:
@@ -318,7 +318,7 @@ def extra_configs(args, dev, stream, state_7b, sampler, peak):
     h.step += 1
 
     def plain7():
-        state_7b.step(h, RS, stream)
+        state_7b.step(h, RS | B.CAST_F_PLAIN_ACCESS, stream)
         h.step += 1
 
     for _ in range(3):
@@ -582,11 +582,15 @@ def cuda_arm(args):
     bytes_per_param = BYTES_PER_PARAM_FLIPS if args.count_flips else BYTES_PER_PARAM
     if args.emit == "dense":
         flags |= B.CAST_F_EMIT_DENSE
-    bulk_exists = ((N, M) == (2, 4) and args.emit == "pruned" and not args.count_flips and args.schedule == "every-step")
-    if args.staging == "auto":
-        args.staging = "bulk" if bulk_exists else "plain"
-    if args.staging == "bulk":
+    # the library's plans take the staged access path where it is built (2:4 and groups of 4 or 8, no compressed emission,
+    # no scale gradient); "plain" and "bulk" force one path
+    bulk_exists = M <= 8 and args.emit != "compressed" and not args.learned_scale
+    if args.staging == "plain":
+        flags |= B.CAST_F_PLAIN_ACCESS
+    elif args.staging == "bulk":
         flags |= B.CAST_F_BULK_STAGING
+    else:
+        args.staging = "bulk" if bulk_exists else "plain"
     compressed = args.emit == "compressed"
     if compressed:
         if wl.resident_layers:
@@ -610,8 +614,9 @@ def cuda_arm(args):
         if (N, M) != (2, 4) or args.emit != "pruned" or wl.resident_layers or args.count_flips:
             raise SystemExit("--schedule t1 is wired for 2:4 on a resident workload")
         scaled = B.CAST_F_GRAD_OF_SCALED if args.learned_scale else 0
-        refresh = B.CAST_F_RESELECT | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE | scaled
-        between = B.CAST_F_EMIT_DENSE | scaled
+        path = flags & (B.CAST_F_PLAIN_ACCESS | B.CAST_F_BULK_STAGING)
+        refresh = B.CAST_F_RESELECT | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE | scaled | path
+        between = B.CAST_F_EMIT_DENSE | scaled | path
         state.step(hyper, B.CAST_F_RESELECT, stream)           # establishes the stored mask (untimed)
         # reuse steps move 28.125 B/param (the metadata is read, not rewritten), refresh steps 28.25
         bytes_per_param = 28.125 + 0.125 / 10
@@ -733,7 +738,7 @@ def cuda_arm(args):
         n_e2e = sum(r * c for r, c in shapes)
         rc, ctx = cast.cast_host_ctx_create(min(16 * 1024 * 1024, max(r * c for r, c in shapes)), 3)
         cast.check(rc)
-        e_flags = flags & ~B.CAST_F_COUNT_FLIPS
+        e_flags = flags & ~(B.CAST_F_COUNT_FLIPS | B.CAST_F_BULK_STAGING | B.CAST_F_PLAIN_ACCESS)      # single-matrix launches: plain path
 
         def host_pass(step_no):
             for h in host:

@@ -62,7 +62,10 @@ enum cast_status {
     CAST_ERR_CUDA   = -6,   /* a CUDA runtime call failed; see cast_last_cuda_error()       */
     CAST_ERR_PLAN   = -7,   /* invalid plan / context handle, or it is too small            */
     CAST_ERR_ALIAS  = -8,   /* two buffers of one matrix overlap                            */
-    CAST_ERR_MEMORY = -9    /* a pointer is not of the required kind (device / host)        */
+    CAST_ERR_MEMORY = -9,   /* a pointer is not of the required kind (device / host)        */
+    CAST_ERR_STAGING = -10  /* an earlier step of this plan gave up waiting for one of its bulk
+                               copies (see CAST_F_BULK_STAGING): a tile of the state was left as it
+                               was; the plan refuses further steps                            */
 };
 
 enum cast_flags {
@@ -93,16 +96,23 @@ enum cast_flags {
                                        initial mask for the initial flip rate i_t; 0 is added where meta_ref is
                                        NULL).  Only cast_plan_step_stats takes this flag, on a plan created
                                        with it (other entry points answer CAST_ERR_PLAN)                  */
-    , CAST_F_BULK_STAGING = 1u << 8 /* an implementation switch, not part of the method: the tiles of the step are
-                                       staged through shared memory by bulk asynchronous copies (and stored back
-                                       the same way) instead of per-thread 128-bit loads and stores.  Results are
-                                       identical bit for bit.  Built for: 2:4 with any of CAST_F_RESELECT,
+    , CAST_F_BULK_STAGING = 1u << 8 /* Two switches that choose how a step moves its data, not what it computes
+                                       (results are identical bit for bit).  The plain access path is one thread =
+                                       8 consecutive columns by 128-bit loads and stores.  The staged path moves
+                                       each 1024-parameter tile with bulk asynchronous copies through shared
+                                       memory; it is built for: 2:4 with any of CAST_F_RESELECT,
                                        CAST_F_COUNT_FLIPS, CAST_F_META_BITMASK, CAST_F_EMIT_DENSE (not dense and
-                                       bitmask together); 4:8 and 1:4 (groups of 4 or 8) with CAST_F_RESELECT |
-                                       CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS.  Any other
-                                       combination with this bit answers CAST_ERR_NM.  As fast as the plain form
-                                       in short runs and ~2 % faster in sustained ones on B200; its one failure
-                                       mode is described at cast_bulk_timeout_count                          */
+                                       bitmask together); groups of 4 or 8 under general N:M with CAST_F_RESELECT |
+                                       CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS.  On B200 it is as
+                                       fast as the plain path in short runs and 2-7 % faster in sustained ones.
+                                       Without either switch: a plan step (cast_plan_step) takes the staged path
+                                       where it is built, everything else the plain one.
+                                       CAST_F_BULK_STAGING asks for the staged path (CAST_ERR_NM where it is not
+                                       built), CAST_F_PLAIN_ACCESS for the plain one.  The staged path's one
+                                       failure mode: its wait for a copy is bounded; a tile whose data has not
+                                       arrived by then is left as it was, counted (cast_bulk_timeout_count), and a
+                                       plan refuses its next step with CAST_ERR_STAGING                        */
+    , CAST_F_PLAIN_ACCESS = 1u << 9
 };
 
 /*
@@ -228,7 +238,8 @@ CAST_API int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* con
  * cast_plan_create  validates `n_tensors` descriptors (host array, copied) and returns an opaque handle
  *                   in *plan_out.  The plan is host memory only: it holds the launch tables, which travel
  *                   to the device as kernel parameters at every step, and allocates nothing on the
- *                   device (but see CAST_F_MASK_STATS under cast_plan_create_ex).  All matrices share N:M.  The buffers named by the descriptors stay owned by
+ *                   device (but see CAST_F_MASK_STATS under cast_plan_create_ex); it also holds one word of
+ *                   page-locked host memory in which staged steps report a copy they gave up on.  All matrices share N:M.  The buffers named by the descriptors stay owned by
  *                   the caller and must outlive the plan's use.
  * cast_plan_step    launches one grid over all matrices on `stream` (ceil(n_tensors / 320) grids for
  *                   larger lists); arguments as cast_adams_step.  The plan may be stepped any number of

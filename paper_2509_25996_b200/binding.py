@@ -25,6 +25,7 @@ CAST_ERR_CUDA = -6
 CAST_ERR_PLAN = -7
 CAST_ERR_ALIAS = -8
 CAST_ERR_MEMORY = -9
+CAST_ERR_STAGING = -10
 
 # flags
 CAST_F_RESELECT = 1 << 0
@@ -36,6 +37,7 @@ CAST_F_EMIT_COMPRESSED = 1 << 5
 CAST_F_GRAD_OF_SCALED = 1 << 6
 CAST_F_MASK_STATS = 1 << 7
 CAST_F_BULK_STAGING = 1 << 8
+CAST_F_PLAIN_ACCESS = 1 << 9
 
 EXPORTS = (
     "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_scale_adam_step",

@@ -13,8 +13,9 @@
 // an ordinary store.  16 KB of shared memory per CTA, 7 CTAs per SM as in the plain kernel.
 //
 // The wait on the barrier is bounded (a phase that has not completed after 2^16 polls with back-off, about 2 ms, is counted in a
-// device-side error counter, the CTA waits once more with the same limit and gives up without storing); the host
-// reads the counter with cast_bulk_timeout_count().  Every copy starts on a 16-byte boundary (tiles start at
+// device-side error counter and, for plans, in a word of host memory that the plan's next step checks; the CTA waits
+// once more with the same limit and gives up without storing); the host reads the counter with
+// cast_bulk_timeout_count().  Every copy starts on a 16-byte boundary (tiles start at
 // multiples of 1024 elements of 16-byte aligned buffers) and has a size that is a multiple of 16 bytes.
 #include "cast_internal.h"
 
@@ -73,7 +74,7 @@ struct __align__(128) BulkTile {
 
 template <int M, uint32_t F, bool TF>
 __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts& c, uint32_t first_unit,
-                                          unsigned long long* flip_count)
+                                          unsigned long long* flip_count, unsigned long long* fail_word)
 {
     using Cfg = StepCfg<M, F, TF>;
     static_assert(M <= 8 && !Cfg::compressed && !Cfg::of_scaled && !Cfg::stats, "staged form: plain emission, groups inside a thread");
@@ -90,31 +91,38 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
         bulk_load(smem_addr(tile.v), t.v + e0, b4, bar);
         bulk_load(smem_addr(tile.g), t.g + e0, b2, bar);
     }
+    // what does not come through the tile is asked for now, so that it travels while the tile does
+    const uint32_t u_idx = threadIdx.x;
+    const bool active = u_idx < units;
+    uint32_t prev_byte = 0;
+    float a = 1.0f;
+    if (active) {
+        if constexpr (Cfg::need_prev) prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[first_unit + u_idx];
+        if (t.scale != nullptr) a = __ldg(t.scale + (uint32_t)(((uint64_t)(first_unit + u_idx) * t.seg_magic) >> t.seg_shift));
+    }
     __syncthreads();                            // the barrier is initialised before anyone polls it
     bool arrived = barrier_wait_bounded(bar, 0);
     if (!arrived) {
-        if (threadIdx.x == 0) atomicAdd(&g_bulk_timeouts, 1ull);
+        if (threadIdx.x == 0) {
+            atomicAdd(&g_bulk_timeouts, 1ull);
+            if (fail_word != nullptr) atomicAdd_system(fail_word, 1ull);      // host memory: the next call on the host sees it
+        }
         arrived = barrier_wait_bounded(bar, 0); // the copies may still land: give them the same time again
     }
     if (!__syncthreads_and(arrived)) return;    // nothing is stored for a tile whose data did not arrive (uniform over the CTA)
 
-    const uint32_t u_idx = threadIdx.x;
-    const bool active = u_idx < units;
     UnitRegs u;
     UnitSums sums;
-    float a = 1.0f;
     if (active) {
         const float4 w0 = *reinterpret_cast<const float4*>(tile.w + u_idx * 8), w1 = *reinterpret_cast<const float4*>(tile.w + u_idx * 8 + 4);
         const float4 m0 = *reinterpret_cast<const float4*>(tile.m + u_idx * 8), m1 = *reinterpret_cast<const float4*>(tile.m + u_idx * 8 + 4);
         const float4 v0 = *reinterpret_cast<const float4*>(tile.v + u_idx * 8), v1 = *reinterpret_cast<const float4*>(tile.v + u_idx * 8 + 4);
         u.g = *reinterpret_cast<const uint4*>(tile.g + u_idx * 8);
-        if (t.scale != nullptr) a = __ldg(t.scale + (uint32_t)(((uint64_t)(first_unit + u_idx) * t.seg_magic) >> t.seg_shift));
         u.w[0] = w0.x; u.w[1] = w0.y; u.w[2] = w0.z; u.w[3] = w0.w; u.w[4] = w1.x; u.w[5] = w1.y; u.w[6] = w1.z; u.w[7] = w1.w;
         u.m[0] = m0.x; u.m[1] = m0.y; u.m[2] = m0.z; u.m[3] = m0.w; u.m[4] = m1.x; u.m[5] = m1.y; u.m[6] = m1.z; u.m[7] = m1.w;
         u.v[0] = v0.x; u.v[1] = v0.y; u.v[2] = v0.z; u.v[3] = v0.w; u.v[4] = v1.x; u.v[5] = v1.y; u.v[6] = v1.z; u.v[7] = v1.w;
-        u.prev_byte = 0;
+        u.prev_byte = prev_byte;
         u.ref_byte = 0;
-        if constexpr (Cfg::need_prev) u.prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[first_unit + u_idx];
         float gw_sum;
         compute_unit<M, F, TF>(u, c, a, false, gw_sum, sums);
         *reinterpret_cast<float4*>(tile.w + u_idx * 8) = make_float4(u.w[0], u.w[1], u.w[2], u.w[3]);
@@ -142,27 +150,28 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
 
 template <int M, uint32_t F, bool TF>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
-adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c, unsigned long long* __restrict__ flip_count)
+adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c, unsigned long long* __restrict__ flip_count,
+                     unsigned long long* fail_word)
 {
-    bulk_tile<M, F, TF>(t, c, blockIdx.x * kTileUnits, flip_count);
+    bulk_tile<M, F, TF>(t, c, blockIdx.x * kTileUnits, flip_count, fail_word);
 }
 
 template <int M, uint32_t F, bool TF>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 adams_nm_multi_bulk_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
-                           unsigned long long* __restrict__ flip_count)
+                           unsigned long long* __restrict__ flip_count, unsigned long long* fail_word)
 {
     const uint32_t tile = blockIdx.x;
     uint32_t k = p.hint[tile >> p.hint_shift];
     while (tile >= p.tile_start[k + 1]) ++k;
-    bulk_tile<M, F, TF>(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits, flip_count);
+    bulk_tile<M, F, TF>(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits, flip_count, fail_word);
 }
 
 template <int M, uint32_t F, bool TF>
 int launch_bulk_t(const StepLaunch& a)
 {
-    if (a.single) adams_nm_bulk_kernel<M, F, TF><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count);
-    else adams_nm_multi_bulk_kernel<M, F, TF><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(*a.multi, *a.c, a.flip_count);
+    if (a.single) adams_nm_bulk_kernel<M, F, TF><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.fail_word);
+    else adams_nm_multi_bulk_kernel<M, F, TF><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(*a.multi, *a.c, a.flip_count, a.fail_word);
     CAST_CUDA_TRY(cudaGetLastError());
     return CAST_OK;
 }

@@ -29,8 +29,9 @@ int check_nm_flags(int N, int M, uint32_t flags, const void* flip_count)
     if (!(flags & CAST_F_META_BITMASK) && !(N == 2 && M == 4)) return CAST_ERR_NM;
     const uint32_t known = CAST_F_RESELECT | CAST_F_COUNT_FLIPS | CAST_F_META_BITMASK |
                            CAST_F_V_KEPT_FROM_G | CAST_F_EMIT_DENSE | CAST_F_EMIT_COMPRESSED |
-                           CAST_F_GRAD_OF_SCALED | CAST_F_MASK_STATS | CAST_F_BULK_STAGING;
+                           CAST_F_GRAD_OF_SCALED | CAST_F_MASK_STATS | CAST_F_BULK_STAGING | CAST_F_PLAIN_ACCESS;
     if (flags & ~known) return CAST_ERR_HYPER;
+    if ((flags & CAST_F_BULK_STAGING) && (flags & CAST_F_PLAIN_ACCESS)) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && (flags & CAST_F_EMIT_DENSE)) return CAST_ERR_HYPER;
     if ((flags & CAST_F_EMIT_COMPRESSED) && M > kUnitElems) return CAST_ERR_NM;
     if ((flags & CAST_F_COUNT_FLIPS) && flip_count == nullptr) return CAST_ERR_NULL;
@@ -196,8 +197,9 @@ int launch_step(const StepLaunch& a, int M)
     if (!step_kernel_exists(M, two_four, f)) return CAST_ERR_NM;
     if (a.single ? tiles_of(*a.single) == 0 : a.multi->tile_start[a.multi->n_tensors] == 0) return CAST_OK;
     if (a.single && tiles_of(*a.single) > kMaxTiles) return CAST_ERR_SHAPE;
-    if (a.c->flags & CAST_F_BULK_STAGING) {
-        if (!bulk_variant_exists(M, a.c->n_keep, f)) return CAST_ERR_NM;      // not one of the configurations the staged form is built for
+    const bool staged_built = bulk_variant_exists(M, a.c->n_keep, f);
+    if ((a.c->flags & CAST_F_BULK_STAGING) && !staged_built) return CAST_ERR_NM;      // not a configuration the staged form is built for
+    if ((a.c->flags & CAST_F_BULK_STAGING) || (a.prefer_staged && staged_built && !(a.c->flags & CAST_F_PLAIN_ACCESS))) {
         const int brc = launch_bulk(a, M, f);
         if (brc == CAST_OK) g_launches.fetch_add(1, std::memory_order_relaxed);
         return brc;
@@ -218,14 +220,15 @@ int launch_step(const StepLaunch& a, int M)
 
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream)
 {
-    const StepLaunch a = {&d, nullptr, &c, flip_count, nullptr, stream};
+    const StepLaunch a = {&d, nullptr, &c, flip_count, nullptr, stream, nullptr, false};
     return launch_step(a, M);
 }
 
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
-                 MaskStats* stat_slots)
+                 MaskStats* stat_slots, unsigned long long* fail_word)
 {
-    const StepLaunch a = {nullptr, &p, &c, flip_count, stat_slots, stream};
+    // a plan that owns a failure word lets the library choose the access path
+    const StepLaunch a = {nullptr, &p, &c, flip_count, stat_slots, stream, fail_word, fail_word != nullptr};
     return launch_step(a, M);
 }
 
@@ -259,6 +262,7 @@ struct Plan {
     uint32_t plan_flags;                 // CAST_F_EMIT_COMPRESSED fixes the size of the w_fwd buffers; CAST_F_MASK_STATS
                                          // says the plan owns the statistics slots
     MaskStats* stat_slots;               // device, kStatSlots accumulators (zero between steps), or nullptr
+    unsigned long long* fail_word;       // page-locked host memory the staged kernels count abandoned copies in, or nullptr
     std::vector<MultiParams> launches;   // one table per launch of up to kMaxLaunchTensors matrices
 };
 
@@ -463,7 +467,19 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
     if (!p) return CAST_ERR_PLAN;
     p->magic = 0;
     p->stat_slots = nullptr;
+    p->fail_word = nullptr;
     cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) {
+        // One word of page-locked host memory that the device can write: without it the plan simply keeps to the
+        // plain access path (the staged one is only taken where a failure can be reported to the next call).
+        void* hw = nullptr;
+        if (cudaHostAlloc(&hw, sizeof(unsigned long long), cudaHostAllocPortable | cudaHostAllocMapped) == cudaSuccess) {
+            p->fail_word = static_cast<unsigned long long*>(hw);
+            *p->fail_word = 0ull;
+        } else {
+            (void)cudaGetLastError();
+        }
+    }
     if (e == cudaSuccess && (plan_flags & CAST_F_MASK_STATS)) {
         e = cudaMalloc(&p->stat_slots, sizeof(MaskStats) * kStatSlots);
         if (e == cudaSuccess) e = cudaMemset(p->stat_slots, 0, sizeof(MaskStats) * kStatSlots);
@@ -471,6 +487,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
     }
     if (e != cudaSuccess) {
         if (p->stat_slots) cudaFree(p->stat_slots);
+        if (p->fail_word) cudaFreeHost(p->fail_word);
         delete p;
         return cuda_failed(e);
     }
@@ -498,6 +515,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
         }
     } catch (const std::bad_alloc&) {
         if (p->stat_slots) cudaFree(p->stat_slots);
+        if (p->fail_word) cudaFreeHost(p->fail_word);
         delete p;
         return CAST_ERR_PLAN;
     }
@@ -523,6 +541,8 @@ extern "C" int cast_plan_step_stats(void* plan, const cast_hyper_t* h, unsigned 
     if ((rc = check_nm_flags(p->N, p->M, h->flags, flip_count)) != CAST_OK) return rc;
     if ((rc = check_stats_ptr(h->flags, stats)) != CAST_OK) return rc;
     if ((h->flags & CAST_F_EMIT_COMPRESSED) != (p->plan_flags & CAST_F_EMIT_COMPRESSED)) return CAST_ERR_PLAN;
+    // a staged step of this plan gave up on a copy earlier: some tile was not updated, and the caller must know
+    if (p->fail_word && *static_cast<volatile unsigned long long*>(p->fail_word) != 0ull) return CAST_ERR_STAGING;
     const bool with_stats = (h->flags & CAST_F_MASK_STATS) != 0;
     if (with_stats && !p->stat_slots) return CAST_ERR_PLAN;      // the plan was not created for statistics
     StepConsts c;
@@ -536,7 +556,7 @@ extern "C" int cast_plan_step_stats(void* plan, const cast_hyper_t* h, unsigned 
         if ((rc = check_device_memory(fp, 1)) != CAST_OK) return rc;
     }
     for (const MultiParams& mp : p->launches)
-        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream, with_stats ? p->stat_slots : nullptr)) != CAST_OK) {
+        if ((rc = launch_multi(mp, p->M, c, flip_count, (cudaStream_t)stream, with_stats ? p->stat_slots : nullptr, p->fail_word)) != CAST_OK) {
             // what the launches so far left in the slots must not reach a later step
             if (with_stats) (void)cudaMemsetAsync(p->stat_slots, 0, sizeof(MaskStats) * kStatSlots, (cudaStream_t)stream);
             return rc;
@@ -559,6 +579,10 @@ extern "C" int cast_plan_destroy(void* plan)
         const cudaError_t e = cudaFree(p->stat_slots);
         if (e != cudaSuccess) rc = cuda_failed(e);
     }
+    if (p->fail_word) {
+        const cudaError_t e = cudaFreeHost(p->fail_word);
+        if (e != cudaSuccess) rc = cuda_failed(e);
+    }
     delete p;
     return rc;
 }
@@ -576,6 +600,7 @@ extern "C" const char* cast_strerror(int status)
         case CAST_ERR_PLAN:   return "invalid plan or context handle";
         case CAST_ERR_ALIAS:  return "buffers of one matrix overlap";
         case CAST_ERR_MEMORY: return "a pointer is not of the required memory kind";
+        case CAST_ERR_STAGING: return "an earlier staged step of this plan gave up waiting for a bulk copy: a tile was not updated";
     }
     return "unknown status";
 }

@@ -68,10 +68,12 @@ struct StepLaunch {
     unsigned long long* flip_count;
     MaskStats* stats;                 // the plan's kStatSlots accumulators, or nullptr
     cudaStream_t stream;
+    unsigned long long* fail_word;    // host memory the staged kernels report a copy they gave up on to, or nullptr
+    bool prefer_staged;               // no access path was asked for: take the staged one where it is built
 };
 int launch_single(const TensorDesc& d, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream);
 int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long long* flip_count, cudaStream_t stream,
-                 MaskStats* stat_slots = nullptr);
+                 MaskStats* stat_slots = nullptr, unsigned long long* fail_word = nullptr);
 
 // Fill the tile-to-matrix hint table (kHintEntries entries) of a launch whose tile_start[0..n_tensors] is set:
 // hint[b] = the matrix that holds tile b << *hint_shift.

@@ -38,7 +38,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_strerror_covers_all_statuses():
-    for s in range(0, -10, -1):
+    for s in range(0, -11, -1):
         assert cast.cast_strerror(s) != "unknown status"
     assert cast.cast_strerror(-99) == "unknown status"
 
@@ -81,7 +81,8 @@ def call(**over):
     (dict(eps=0.0), B.CAST_ERR_HYPER),
     (dict(lr=float("nan")), B.CAST_ERR_HYPER),
     (dict(l1_coeff=float("inf")), B.CAST_ERR_HYPER),
-    (dict(flags=1 << 9), B.CAST_ERR_HYPER),
+    (dict(flags=1 << 10), B.CAST_ERR_HYPER),                                            # unknown flag bit
+    (dict(flags=B.CAST_F_RESELECT | B.CAST_F_BULK_STAGING | B.CAST_F_PLAIN_ACCESS), B.CAST_ERR_HYPER),
     (dict(m=W + 64), B.CAST_ERR_ALIAS),
     (dict(meta=F + 16), B.CAST_ERR_ALIAS),
 ])

@@ -394,22 +394,33 @@ def test_host_step_pageable_memory():
     U.assert_parity(got, ref, "pageable")
 
 
-def test_plan_with_bulk_staging_gives_the_same_bits():
-    """All matrices of a plan in one launch of the staged variant: identical to the plain launch."""
+def test_plan_access_paths_give_the_same_bits():
+    """A plan step takes the staged access path where it is built unless told otherwise: the default, the forced staged
+    and the forced plain launches of the same steps agree bit for bit, flips included, and no staged wait ran out."""
     from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
     shapes = [(24, 256), (7, 2080), (3, 1056), (40, 512)]
-    a = DeviceModelState(shapes, 2, 4, seed=6, device="cuda:0", scale_mode="jitter")
-    b = DeviceModelState(shapes, 2, 4, seed=6, device="cuda:0", scale_mode="jitter")
+    paths = (0, B.CAST_F_BULK_STAGING, B.CAST_F_PLAIN_ACCESS)
+    states = [DeviceModelState(shapes, 2, 4, seed=6, device="cuda:0", scale_mode="jitter") for _ in paths]
     h = RunHyper(total_steps=30000)
-    for _ in range(2):
-        a.step(h, B.CAST_F_RESELECT)
-        b.step(h, B.CAST_F_RESELECT | B.CAST_F_BULK_STAGING)
+    launches = cast.cast_kernel_launch_count()
+    for flags in (B.CAST_F_RESELECT, B.CAST_F_EMIT_DENSE, B.CAST_F_RESELECT | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE):
+        for st, path in zip(states, paths):
+            st.step(h, flags | path)
         h.step += 1
     torch.cuda.synchronize()
-    for x, y in zip(a.mats, b.mats):
-        for k in ("w", "m", "v", "w_fwd", "meta"):
-            assert torch.equal(getattr(x, k), getattr(y, k)), k
+    assert cast.cast_kernel_launch_count() == launches + 9
+    for other in states[1:]:
+        for x, y in zip(states[0].mats, other.mats):
+            for k in ("w", "m", "v", "w_fwd", "meta"):
+                assert torch.equal(getattr(x, k), getattr(y, k)), k
+        assert int(other.flips.item()) == int(states[0].flips.item()) > 0
     rc, timeouts = cast.cast_bulk_timeout_count()
     assert rc == 0 and timeouts == 0
-    a.close()
-    b.close()
+    # a configuration the staged path is not built for runs plain by default and is refused when staged is forced
+    hy = B.make_hyper(1e-4, 0.9, 0.95, 1e-8, 1e-3, h.step, 30000, B.CAST_F_RESELECT | B.CAST_F_V_KEPT_FROM_G)
+    cast.check(cast.cast_plan_step(states[0].plan, hy, None, None))
+    hy.flags |= B.CAST_F_BULK_STAGING
+    assert cast.cast_plan_step(states[0].plan, hy, None, None) == B.CAST_ERR_NM
+    torch.cuda.synchronize()
+    for st in states:
+        st.close()
