@@ -590,7 +590,7 @@ def cuda_arm(args):
     elif args.staging == "bulk":
         flags |= B.CAST_F_BULK_STAGING
     else:
-        args.staging = "bulk" if bulk_exists else "plain"
+        args.staging = "bulk" if bulk_exists and wl.n_params >= (16384 << 10) else "plain"
     compressed = args.emit == "compressed"
     if compressed:
         if wl.resident_layers:

@@ -105,8 +105,9 @@ enum cast_flags {
                                        bitmask together); groups of 4 or 8 under general N:M with CAST_F_RESELECT |
                                        CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS.  On B200 it is as
                                        fast as the plain path in short runs and 2-7 % faster in sustained ones.
-                                       Without either switch: a plan step (cast_plan_step) takes the staged path
-                                       where it is built, everything else the plain one.
+                                       Without either switch: a plan step (cast_plan_step) over at least
+                                       16.8 M parameters takes the staged path where it is built, everything
+                                       else the plain one.
                                        CAST_F_BULK_STAGING asks for the staged path (CAST_ERR_NM where it is not
                                        built), CAST_F_PLAIN_ACCESS for the plain one.  The staged path's one
                                        failure mode: its wait for a copy is bounded; a tile whose data has not

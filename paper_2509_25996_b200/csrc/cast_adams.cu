@@ -199,7 +199,12 @@ int launch_step(const StepLaunch& a, int M)
     if (a.single && tiles_of(*a.single) > kMaxTiles) return CAST_ERR_SHAPE;
     const bool staged_built = bulk_variant_exists(M, a.c->n_keep, f);
     if ((a.c->flags & CAST_F_BULK_STAGING) && !staged_built) return CAST_ERR_NM;      // not a configuration the staged form is built for
-    if ((a.c->flags & CAST_F_BULK_STAGING) || (a.prefer_staged && staged_built && !(a.c->flags & CAST_F_PLAIN_ACCESS))) {
+    // Left to itself a plan stages launches of at least 16 Ki tiles (16.8 M parameters): below that a launch is over
+    // before the device's power limit matters, and the staged form's extra latency per CTA shows instead (one
+    // 3072 x 768 matrix, cold: 20.3 against 18.6 us).
+    const uint64_t n_tiles = a.single ? tiles_of(*a.single) : a.multi->tile_start[a.multi->n_tensors];
+    const bool by_default = a.prefer_staged && staged_built && n_tiles >= 16384u && !(a.c->flags & CAST_F_PLAIN_ACCESS);
+    if ((a.c->flags & CAST_F_BULK_STAGING) || by_default) {
         const int brc = launch_bulk(a, M, f);
         if (brc == CAST_OK) g_launches.fetch_add(1, std::memory_order_relaxed);
         return brc;

@@ -398,8 +398,8 @@ def test_plan_access_paths_give_the_same_bits():
     """A plan step takes the staged access path where it is built unless told otherwise: the default, the forced staged
     and the forced plain launches of the same steps agree bit for bit, flips included, and no staged wait ran out."""
     from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
-    shapes = [(24, 256), (7, 2080), (3, 1056), (40, 512)]
-    paths = (0, B.CAST_F_BULK_STAGING, B.CAST_F_PLAIN_ACCESS)
+    shapes = [(24, 256), (7, 2080), (3, 1056), (4096, 4096), (40, 512)]         # 16.8 M parameters: above the size from which
+    paths = (0, B.CAST_F_BULK_STAGING, B.CAST_F_PLAIN_ACCESS)                   # a plan stages by default
     states = [DeviceModelState(shapes, 2, 4, seed=6, device="cuda:0", scale_mode="jitter") for _ in paths]
     h = RunHyper(total_steps=30000)
     launches = cast.cast_kernel_launch_count()
