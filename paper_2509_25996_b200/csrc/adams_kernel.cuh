@@ -463,6 +463,25 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
     u.g.w = pack_bf16x2(fwd[6], fwd[7]);
 }
 
+// dL/dA of Eq. 12: sums gw_sum over the lanes of the warp that share a row segment (segments are runs of consecutive
+// lanes), then one atomic per run.  Lanes without data carry a segment of their own and add nothing.  All lanes of
+// the warp call this (the pointer is uniform over the CTA).
+__device__ __forceinline__ void add_scale_grad(float* scale_grad, uint32_t seg, bool active, float gw_sum)
+{
+    if (scale_grad == nullptr) return;
+    const unsigned lane = threadIdx.x & 31u;
+    const uint32_t my_seg = active ? seg : 0xFFFFFFFFu;
+    float p = active ? gw_sum : 0.0f;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const float q = __shfl_up_sync(0xFFFFFFFFu, p, d);
+        const uint32_t s = __shfl_up_sync(0xFFFFFFFFu, my_seg, d);
+        if (lane >= (unsigned)d && s == my_seg) p += q;
+    }
+    const uint32_t next_seg = __shfl_down_sync(0xFFFFFFFFu, my_seg, 1);
+    if (active && (lane == 31u || next_seg != my_seg)) atomicAdd(scale_grad + seg, p);
+}
+
 // The whole per-unit body: loads, arithmetic, stores.
 // `active` is false for threads past the end of the matrix; they take part in the shuffles only.
 template <int M, uint32_t F, bool TF>
@@ -500,23 +519,7 @@ __device__ __forceinline__ void process_unit(const TensorDesc& t, const StepCons
     float gw_sum;
     UnitSums mine;
     compute_unit<M, F, TF>(u, c, a, has_ref, gw_sum, mine);
-    if constexpr (Cfg::of_scaled) {
-        if (t.scale_grad != nullptr) {                              // uniform over the CTA: all lanes shuffle
-            // Sum gw_sum over the lanes of the warp that share a row segment (segments are runs of consecutive
-            // lanes), then one atomic per run.  Lanes without data carry a segment of their own and add nothing.
-            const unsigned lane = threadIdx.x & 31u;
-            const uint32_t my_seg = active ? seg : 0xFFFFFFFFu;
-            float p = active ? gw_sum : 0.0f;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const float q = __shfl_up_sync(0xFFFFFFFFu, p, d);
-                const uint32_t s = __shfl_up_sync(0xFFFFFFFFu, my_seg, d);
-                if (lane >= (unsigned)d && s == my_seg) p += q;
-            }
-            const uint32_t next_seg = __shfl_down_sync(0xFFFFFFFFu, my_seg, 1);
-            if (active && (lane == 31u || next_seg != my_seg)) atomicAdd(t.scale_grad + seg, p);
-        }
-    }
+    if constexpr (Cfg::of_scaled) add_scale_grad(t.scale_grad, seg, active, gw_sum);
 
     if (active) {
         st_f4(t.w + e, make_float4(u.w[0], u.w[1], u.w[2], u.w[3]));

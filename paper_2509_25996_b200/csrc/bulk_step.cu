@@ -74,10 +74,11 @@ struct __align__(128) BulkTile {
 
 template <int M, uint32_t F, bool TF>
 __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts& c, uint32_t first_unit,
-                                          unsigned long long* flip_count, unsigned long long* fail_word)
+                                          unsigned long long* flip_count, MaskStats* stats, unsigned long long* fail_word)
 {
     using Cfg = StepCfg<M, F, TF>;
-    static_assert(M <= 8 && !Cfg::compressed && !Cfg::of_scaled && !Cfg::stats, "staged form: plain emission, groups inside a thread");
+    static_assert(M <= 8, "staged form: groups inside a thread");
+    static_assert(!Cfg::compressed || (TF && !Cfg::bitmask), "staged compressed emission: 2:4 with index-form metadata");
     __shared__ BulkTile tile;
     const uint32_t units = min((uint32_t)kTileUnits, t.n_units - first_unit);       // a matrix's last tile may be short
     const size_t e0 = (size_t)first_unit * kUnitElems;
@@ -94,11 +95,16 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
     // what does not come through the tile is asked for now, so that it travels while the tile does
     const uint32_t u_idx = threadIdx.x;
     const bool active = u_idx < units;
-    uint32_t prev_byte = 0;
+    uint32_t prev_byte = 0, ref_byte = 0, seg = 0;
     float a = 1.0f;
+    const bool has_ref = Cfg::stats && t.meta_ref != nullptr;      // uniform over the CTA
     if (active) {
         if constexpr (Cfg::need_prev) prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[first_unit + u_idx];
-        if (t.scale != nullptr) a = __ldg(t.scale + (uint32_t)(((uint64_t)(first_unit + u_idx) * t.seg_magic) >> t.seg_shift));
+        if (has_ref) ref_byte = t.meta_ref[first_unit + u_idx];
+        if (t.scale != nullptr) {
+            seg = (uint32_t)(((uint64_t)(first_unit + u_idx) * t.seg_magic) >> t.seg_shift);
+            a = __ldg(t.scale + seg);
+        }
     }
     __syncthreads();                            // the barrier is initialised before anyone polls it
     bool arrived = barrier_wait_bounded(bar, 0);
@@ -113,6 +119,8 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
 
     UnitRegs u;
     UnitSums sums;
+    float gw_sum = 0.0f;
+    uint2 kept_out = make_uint2(0u, 0u);
     if (active) {
         const float4 w0 = *reinterpret_cast<const float4*>(tile.w + u_idx * 8), w1 = *reinterpret_cast<const float4*>(tile.w + u_idx * 8 + 4);
         const float4 m0 = *reinterpret_cast<const float4*>(tile.m + u_idx * 8), m1 = *reinterpret_cast<const float4*>(tile.m + u_idx * 8 + 4);
@@ -122,18 +130,31 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
         u.m[0] = m0.x; u.m[1] = m0.y; u.m[2] = m0.z; u.m[3] = m0.w; u.m[4] = m1.x; u.m[5] = m1.y; u.m[6] = m1.z; u.m[7] = m1.w;
         u.v[0] = v0.x; u.v[1] = v0.y; u.v[2] = v0.z; u.v[3] = v0.w; u.v[4] = v1.x; u.v[5] = v1.y; u.v[6] = v1.z; u.v[7] = v1.w;
         u.prev_byte = prev_byte;
-        u.ref_byte = 0;
-        float gw_sum;
-        compute_unit<M, F, TF>(u, c, a, false, gw_sum, sums);
+        u.ref_byte = ref_byte;
+        compute_unit<M, F, TF>(u, c, a, has_ref, gw_sum, sums);
         *reinterpret_cast<float4*>(tile.w + u_idx * 8) = make_float4(u.w[0], u.w[1], u.w[2], u.w[3]);
         *reinterpret_cast<float4*>(tile.w + u_idx * 8 + 4) = make_float4(u.w[4], u.w[5], u.w[6], u.w[7]);
         *reinterpret_cast<float4*>(tile.m + u_idx * 8) = make_float4(u.m[0], u.m[1], u.m[2], u.m[3]);
         *reinterpret_cast<float4*>(tile.m + u_idx * 8 + 4) = make_float4(u.m[4], u.m[5], u.m[6], u.m[7]);
         *reinterpret_cast<float4*>(tile.v + u_idx * 8) = make_float4(u.v[0], u.v[1], u.v[2], u.v[3]);
         *reinterpret_cast<float4*>(tile.v + u_idx * 8 + 4) = make_float4(u.v[4], u.v[5], u.v[6], u.v[7]);
-        *reinterpret_cast<uint4*>(tile.g + u_idx * 8) = u.g;
+        if constexpr (Cfg::compressed) {
+            // the kept pair of each group, picked by the index nibbles: 4 values per unit
+            const uint32_t mb = u.meta_byte;
+            kept_out = make_uint2(kept_pair_by_index(u.g.x, u.g.y, mb & 3u, (mb >> 2) & 3u),
+                                  kept_pair_by_index(u.g.z, u.g.w, (mb >> 4) & 3u, mb >> 6));
+        } else {
+            *reinterpret_cast<uint4*>(tile.g + u_idx * 8) = u.g;
+        }
         if constexpr (Cfg::reselect) reinterpret_cast<uint8_t*>(t.meta)[first_unit + u_idx] = (uint8_t)u.meta_byte;
     }
+    if constexpr (Cfg::compressed) {
+        // packed densely, a unit's 8 bytes land in the gradient slot of another unit: every thread has read its
+        // gradient before anyone writes
+        __syncthreads();
+        if (active) *reinterpret_cast<uint2*>(tile.g + u_idx * 4) = kept_out;
+    }
+    if constexpr (Cfg::of_scaled) add_scale_grad(t.scale_grad, seg, active, gw_sum);      // all lanes: warp shuffles inside
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's shared-memory writes, for the bulk stores
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -141,11 +162,12 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
         bulk_store(t.w + e0, smem_addr(tile.w), b4);
         bulk_store(t.m + e0, smem_addr(tile.m), b4);
         bulk_store(t.v + e0, smem_addr(tile.v), b4);
-        bulk_store(t.w_fwd + e0, smem_addr(tile.g), b2);
+        if constexpr (Cfg::compressed) bulk_store(t.w_fwd + e0 / 2, smem_addr(tile.g), b2 / 2);      // units are a multiple of 4: 16-byte sizes
+        else bulk_store(t.w_fwd + e0, smem_addr(tile.g), b2);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the shared memory has been read: the CTA may end
     }
-    add_sums<Cfg::count_flips, false>(sums, flip_count, nullptr);
+    add_sums<Cfg::count_flips, Cfg::stats>(sums, flip_count, stats);
 }
 
 template <int M, uint32_t F, bool TF>
@@ -153,25 +175,30 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c, unsigned long long* __restrict__ flip_count,
                      unsigned long long* fail_word)
 {
-    bulk_tile<M, F, TF>(t, c, blockIdx.x * kTileUnits, flip_count, fail_word);
+    bulk_tile<M, F, TF>(t, c, blockIdx.x * kTileUnits, flip_count, nullptr, fail_word);
 }
 
 template <int M, uint32_t F, bool TF>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 adams_nm_multi_bulk_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
-                           unsigned long long* __restrict__ flip_count, unsigned long long* fail_word)
+                           unsigned long long* __restrict__ flip_count, MaskStats* __restrict__ stats, unsigned long long* fail_word)
 {
     const uint32_t tile = blockIdx.x;
     uint32_t k = p.hint[tile >> p.hint_shift];
     while (tile >= p.tile_start[k + 1]) ++k;
-    bulk_tile<M, F, TF>(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits, flip_count, fail_word);
+    bulk_tile<M, F, TF>(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits, flip_count, stats, fail_word);
 }
 
 template <int M, uint32_t F, bool TF>
 int launch_bulk_t(const StepLaunch& a)
 {
-    if (a.single) adams_nm_bulk_kernel<M, F, TF><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.fail_word);
-    else adams_nm_multi_bulk_kernel<M, F, TF><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(*a.multi, *a.c, a.flip_count, a.fail_word);
+    if (a.single) {
+        if constexpr ((F & kMaskStats) != 0) return CAST_ERR_NM;      // the statistics epilogue exists for plans only
+        else adams_nm_bulk_kernel<M, F, TF><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.fail_word);
+    } else {
+        adams_nm_multi_bulk_kernel<M, F, TF><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(
+            *a.multi, *a.c, a.flip_count, a.stats, a.fail_word);
+    }
     CAST_CUDA_TRY(cudaGetLastError());
     return CAST_OK;
 }
@@ -179,9 +206,13 @@ int launch_bulk_t(const StepLaunch& a)
 // The configurations the staged form is built for: the steps of training and of the listed workloads.
 //   2:4:      select (index or bitmask form), with flips, with dense emission; stored mask with pruned / dense emission
 //   4:8, 1:4: select, with flips (bitmask form)
-constexpr uint32_t RS = kReselect, FL = kCountFlips, BM = kMetaBitmask, DN = kEmitDense;
+//   2:4 also: compressed emission with index-form metadata; the steps of training with a learned scale (gradient
+//             through Eq. 12) and / or with the statistics epilogue
+constexpr uint32_t RS = kReselect, FL = kCountFlips, BM = kMetaBitmask, DN = kEmitDense, CP = kEmitCompressed, GS = kGradOfScaled,
+                   ST = kMaskStats;
 #define CAST_BULK_CASES_2OF4(X) X(4, RS, true) X(4, RS | FL, true) X(4, RS | BM, true) X(4, RS | BM | FL, true) X(4, RS | DN, true) \
-    X(4, RS | FL | DN, true) X(4, 0u, true) X(4, DN, true)
+    X(4, RS | FL | DN, true) X(4, 0u, true) X(4, DN, true) X(4, RS | CP, true) X(4, DN | GS, true) X(4, RS | FL | DN | GS, true) \
+    X(4, RS | FL | DN | ST, true) X(4, RS | FL | DN | GS | ST, true) X(4, DN | ST, true) X(4, DN | GS | ST, true)
 #define CAST_BULK_CASES_NM(X) X(4, RS | BM, false) X(4, RS | BM | FL, false) X(8, RS | BM, false) X(8, RS | BM | FL, false)
 
 }  // namespace
