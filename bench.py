@@ -34,8 +34,8 @@ FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
 # taken on); every byte is touched once, so the traffic of a launch is this figure times its parameter count.
 # Set to None when that kernel changes, until the counters are taken again; reported only for the workload and
 # configuration they were taken on (the 2:4 headline over LLaMA2-7B shapes).
-NCU_DRAM_BYTES_PER_PARAM = {"plain": 27.849, "bulk": None}
-NCU_KERNEL = {"plain": "adams_nm_multi_kernel<4, 1, 1>", "bulk": "adams_nm_multi_bulk_kernel"}
+NCU_DRAM_BYTES_PER_PARAM = {"plain": 27.849, "bulk": 27.843}
+NCU_KERNEL = {"plain": "adams_nm_multi_kernel<4, 1, 1>", "bulk": "adams_nm_multi_bulk_kernel<4, 1, 1>"}
 
 METRIC = "AdamS 2:4 step params/s"
 
@@ -584,7 +584,7 @@ def cuda_arm(args):
         flags |= B.CAST_F_EMIT_DENSE
     # the library's plans take the staged access path where it is built (2:4 and groups of 4 or 8, no compressed emission,
     # no scale gradient); "plain" and "bulk" force one path
-    bulk_exists = M <= 8 and args.emit != "compressed" and not args.learned_scale
+    bulk_exists = M <= 8 and ((N, M) == (2, 4) or (args.emit != "compressed" and not args.learned_scale))
     if args.staging == "plain":
         flags |= B.CAST_F_PLAIN_ACCESS
     elif args.staging == "bulk":
@@ -862,8 +862,7 @@ def cuda_arm(args):
                      "note": "same steps back to back without the flush: the state stays in L2, not an HBM figure"}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": ("adams_nm_multi_bulk_kernel" if args.staging == "bulk" else
-                                f"adams_nm_multi_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}, {1 if (N, M) == (2, 4) else 0}>"),
+                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi{'_bulk' if args.staging == 'bulk' else ''}_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}, {1 if (N, M) == (2, 4) else 0}>",
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": step_launches,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,
