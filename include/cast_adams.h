@@ -83,7 +83,13 @@ enum cast_flags {
                                        forward pass used (Eq. 12) instead of the gradient with respect to W: the
                                        step applies the chain rule dL/dW = A (.) g itself and, where a scale_grad
                                        buffer is given, adds dL/dA[r, s] = sum_{c in segment s} g[r, c] W_{t-1}[r, c]
-                                       to it                                                              */
+                                       to it.  The factor A is the `scale` buffer as it stands when the step runs
+                                       (the same buffer also scales the emitted weight).  If the scale is updated
+                                       (cast_scale_adam_step) between the emission of the forward weight that
+                                       produced g and this step, the factor is the updated A_t where the forward
+                                       pass used A_{t-1}: a one-step lag of relative size lr_A, inherent to doing
+                                       the scale gradient and the emission in one pass.  A caller that wants the
+                                       forward's own factor passes the buffer that scaled that emission       */
     CAST_F_EMIT_COMPRESSED = 1u << 5, /* emit only the kept entries of the pruned product (Alg. 2, final loop):
                                        w_fwd_bf16 is then [rows][cols*N/M], the N kept values of each group in
                                        column order; with the metadata it is the whole pruned matrix, and a

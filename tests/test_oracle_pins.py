@@ -426,6 +426,26 @@ def test_stored_mask_gates_the_decay_when_it_is_not_the_top_n(bitmask):
     assert np.array_equal(fresh["w"][outside], w0[outside]) and not np.any(fresh["w"][~outside] == w0[~outside])
 
 
+def test_chain_rule_factor_is_the_scale_passed_to_the_call():
+    """With the gradient taken through the scaling (Eq. 12) the oracle multiplies g by the scale it is given in THIS
+    call -- also when that scale differs from the one an earlier call emitted the forward weight with (the one-step
+    lag the header describes).  beta1 = 0, t = 1, m0 = v0 = 0, full density: the stored first moment is exactly
+    A (.) g, per row segment, for whatever A is passed; the emitted weight uses the same A."""
+    rng = np.random.default_rng(77)
+    w0 = rng.normal(0, 0.02, size=(3, 64)).astype(np.float32)
+    g, gb = bf16_exact(rng.normal(0, 1e-3, size=(3, 64)))
+    a_old = (1 + 0.1 * rng.random((3, 2))).astype(np.float32)
+    a_new = (a_old * np.float32(1.25)).astype(np.float32)                  # an exact, visible change of the scale
+    h = Hyper(lr=1e-4, beta1=0.0, beta2=0.95, eps=1e-8, l1_coeff=0.0, step=1, total_steps=10)
+    flags = orc.F_RESELECT | orc.F_META_BITMASK | orc.F_GRAD_OF_SCALED | orc.F_EMIT_DENSE
+    for a in (a_old, a_new):
+        out = run(w0, g=gb, scale=a, N=4, M=4, hyper=h, flags=flags)
+        seg = np.repeat(a, 32, axis=1).astype(np.float64)
+        np.testing.assert_allclose(out["m"], seg * g, rtol=1e-7)
+        np.testing.assert_allclose(bf16_bits_to_f32(out["w_fwd"]), seg * out["w"], rtol=2.0 ** -8)
+        np.testing.assert_allclose(out["scale_grad"], (g.astype(np.float64) * w0).reshape(3, 2, 32).sum(-1), rtol=1e-12)
+
+
 # --------------------------------------------------------------------------- numerics and long-run behaviour
 
 def test_fp32_order_stays_within_tolerance_of_fp64():
