@@ -337,6 +337,10 @@ extern "C" int cast_kd_loss(const cast_bf16* student_logits, const cast_bf16* te
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(grid * kCluster);
         cfg.blockDim = dim3(256);
+        // 40 KB of (unused) dynamic shared memory per CTA cap the residency at 5 CTAs per SM: ~90 rows in flight, whose
+        // inputs and gradient (770 KB per 128 K-logit row) then stay inside the L2 between the two sweeps.  At the 8 CTAs
+        // per SM the registers would allow, the rows in flight outgrow it (7.6 instead of 5.9 B per logit of DRAM traffic).
+        cfg.dynamicSmemBytes = 40 * 1024;
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
