@@ -347,7 +347,7 @@ def test_bulk_staged_variant_gives_the_same_bits(N, M, flags, rows, cols):
         inp.scale = None
     h = Hyper()
     enc = flags & BM
-    prev = U.run_oracle(inputs(rows, cols, seed=33), N, M, Hyper(lr=0.0), RS | enc)["meta"]      # stored / previous mask
+    prev = U.run_oracle(inputs(rows, cols, seed=33, scale_mode="none"), N, M, Hyper(lr=0.0), RS | enc)["meta"]      # stored / previous mask
     plain = U.run_cuda_single(inp, N, M, h, flags, meta_in=prev)
     staged = U.run_cuda_single(inp, N, M, h, flags | B.CAST_F_BULK_STAGING, meta_in=prev)
     for k in ("w", "m", "v", "w_fwd", "meta"):
