@@ -332,8 +332,7 @@ BULK_CASES = [(2, 4, RS), (2, 4, RS | B.CAST_F_COUNT_FLIPS), (2, 4, RS | BM), (2
               (2, 4, RS | B.CAST_F_EMIT_DENSE), (2, 4, RS | B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE), (2, 4, 0), (2, 4, B.CAST_F_EMIT_DENSE),
               (2, 4, B.CAST_F_COUNT_FLIPS | B.CAST_F_EMIT_DENSE),
               (2, 4, RS | B.CAST_F_EMIT_COMPRESSED),
-              (1, 4, RS | BM), (3, 4, RS | BM | B.CAST_F_COUNT_FLIPS), (4, 8, RS | BM), (4, 8, RS | BM | B.CAST_F_COUNT_FLIPS), (1, 8, RS | BM),
-              (5, 16, RS | BM), (8, 16, RS | BM | B.CAST_F_COUNT_FLIPS), (8, 32, RS | BM), (31, 32, RS | BM | B.CAST_F_COUNT_FLIPS)]
+              (1, 4, RS | BM), (3, 4, RS | BM | B.CAST_F_COUNT_FLIPS), (4, 8, RS | BM), (4, 8, RS | BM | B.CAST_F_COUNT_FLIPS), (1, 8, RS | BM)]
 
 
 @pytest.mark.parametrize("N,M,flags", BULK_CASES)
@@ -364,7 +363,7 @@ def test_bulk_staging_answers_nm_error_where_it_is_not_built():
     st = U.to_device(inp, DEV)
     before = cast.cast_kernel_launch_count()
     lr, b1, b2, eps, lam = Hyper().as_f32()
-    for N, M, flags in ((2, 4, RS | BM | B.CAST_F_EMIT_COMPRESSED), (2, 4, RS | B.CAST_F_GRAD_OF_SCALED), (8, 16, BM),
+    for N, M, flags in ((2, 4, RS | BM | B.CAST_F_EMIT_COMPRESSED), (2, 4, RS | B.CAST_F_GRAD_OF_SCALED), (8, 16, RS | BM),
                         (2, 4, RS | B.CAST_F_V_KEPT_FROM_G), (2, 4, BM | B.CAST_F_EMIT_DENSE)):
         rc = cast.cast_adams_step(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale, 2, 4, 64, N, M,
                                   lr, b1, b2, eps, lam, 1000, 30000, flags | B.CAST_F_BULK_STAGING, None, None)
