@@ -284,6 +284,10 @@ CAST_API int cast_plan_step(void* plan, const cast_hyper_t* hyper, unsigned long
 CAST_API int cast_plan_step_stats(void* plan, const cast_hyper_t* hyper, unsigned long long* flip_count,
                          cast_mask_stats_t* stats, cast_stream_t stream);
 CAST_API int cast_plan_destroy(void* plan);
+/* Fault injection on the host, for tests of a caller's error handling: marks the plan exactly as a staged kernel does
+ * when it gives up waiting for a bulk copy (see CAST_F_BULK_STAGING).  Every later step of the plan answers
+ * CAST_ERR_STAGING; the plan can still be destroyed.  Touches no device. */
+CAST_API int cast_plan_report_staging_failure(void* plan);
 
 /*
  * Host-resident optimizer state (the same iteration of Alg. 1, with w, m, v, g, w_fwd, meta and scale

@@ -41,7 +41,7 @@ CAST_F_PLAIN_ACCESS = 1 << 9
 
 EXPORTS = (
     "cast_adams_step", "cast_adams_step_ex", "cast_scale_adam_step", "cast_plan_scale_adam_step",
-    "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_step_stats", "cast_plan_destroy",
+    "cast_plan_create", "cast_plan_create_ex", "cast_plan_step", "cast_plan_step_stats", "cast_plan_destroy", "cast_plan_report_staging_failure",
     "cast_host_ctx_create", "cast_host_step", "cast_host_ctx_sync", "cast_host_ctx_destroy",
     "cast_host_step_static", "cast_kd_loss", "cast_prune_fold", "cast_plan_prune_fold", "cast_mask_stats", "cast_plan_mask_stats",
     "cast_probe_launch", "cast_probe_stream", "cast_bulk_timeout_count",
@@ -119,6 +119,8 @@ def load_library() -> ctypes.CDLL:
     lib.cast_plan_step.argtypes = [ctypes.c_void_p, ctypes.POINTER(cast_hyper_t), ctypes.c_void_p, ctypes.c_void_p]
     lib.cast_plan_step_stats.restype = ctypes.c_int
     lib.cast_plan_step_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(cast_hyper_t), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    lib.cast_plan_report_staging_failure.restype = ctypes.c_int
+    lib.cast_plan_report_staging_failure.argtypes = [ctypes.c_void_p]
     lib.cast_plan_destroy.restype = ctypes.c_int
     lib.cast_plan_destroy.argtypes = [ctypes.c_void_p]
     lib.cast_host_ctx_create.restype = ctypes.c_int
@@ -273,6 +275,10 @@ def cast_plan_step_stats(plan, hyper: Optional[cast_hyper_t], flip_count=None, s
     """`stats`: device buffer of sizeof(cast_mask_stats_t) = 32 bytes that a step with CAST_F_MASK_STATS adds to."""
     h = ctypes.byref(hyper) if hyper is not None else None
     return load_library().cast_plan_step_stats(plan, h, _ptr(flip_count), _ptr(stats), _stream(stream))
+
+
+def cast_plan_report_staging_failure(plan) -> int:
+    return load_library().cast_plan_report_staging_failure(plan)
 
 
 def cast_plan_destroy(plan) -> int:

@@ -574,6 +574,15 @@ extern "C" int cast_plan_step_stats(void* plan, const cast_hyper_t* h, unsigned 
     return CAST_OK;
 }
 
+extern "C" int cast_plan_report_staging_failure(void* plan)
+{
+    Plan* p = (Plan*)plan;
+    if (!p || p->magic != kPlanMagic) return CAST_ERR_PLAN;
+    if (!p->fail_word) return CAST_ERR_PLAN;
+    *static_cast<volatile unsigned long long*>(p->fail_word) += 1ull;      // what a staged kernel does when it gives up on a copy
+    return CAST_OK;
+}
+
 extern "C" int cast_plan_destroy(void* plan)
 {
     Plan* p = (Plan*)plan;

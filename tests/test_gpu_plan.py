@@ -460,3 +460,24 @@ def test_plan_access_paths_agree_with_a_learned_scale_and_statistics():
     assert cast.cast_bulk_timeout_count() == (0, 0)
     for st in states:
         st.close()
+
+
+def test_a_plan_that_gave_up_on_a_staged_copy_refuses_further_steps():
+    """The staged kernels wait for their copies a bounded time; a tile they give up on is reported in a word of host
+    memory the plan owns, and the plan then answers CAST_ERR_STAGING instead of stepping on over a state that was not
+    fully updated.  The report is injected on the host here (no GPU wait is made to run out)."""
+    from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
+    st = DeviceModelState([(16, 512)], 2, 4, seed=9, device="cuda:0", scale_mode="ones")
+    h = RunHyper(total_steps=30000)
+    st.step(h, B.CAST_F_RESELECT)
+    torch.cuda.synchronize()
+    launches = cast.cast_kernel_launch_count()
+    assert cast.cast_plan_report_staging_failure(st.plan) == B.CAST_OK
+    hy = B.make_hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step + 1, h.total_steps, B.CAST_F_RESELECT)
+    assert cast.cast_plan_step(st.plan, hy, None, None) == B.CAST_ERR_STAGING
+    hy.flags |= B.CAST_F_PLAIN_ACCESS
+    assert cast.cast_plan_step(st.plan, hy, None, None) == B.CAST_ERR_STAGING          # whatever the path
+    assert cast.cast_kernel_launch_count() == launches
+    assert "bulk copy" in cast.cast_strerror(B.CAST_ERR_STAGING)
+    assert cast.cast_plan_report_staging_failure(None) == B.CAST_ERR_PLAN
+    st.close()
