@@ -584,7 +584,7 @@ def cuda_arm(args):
         flags |= B.CAST_F_EMIT_DENSE
     # the library's plans take the staged access path where it is built (2:4 and groups of 4 or 8, no compressed emission,
     # no scale gradient); "plain" and "bulk" force one path
-    bulk_exists = (N, M) == (2, 4) or (M <= 8 and args.emit != "compressed" and not args.learned_scale)
+    bulk_exists = not args.learned_scale and ((N, M) == (2, 4) or (M <= 8 and args.emit != "compressed"))
     if args.staging == "plain":
         flags |= B.CAST_F_PLAIN_ACCESS
     elif args.staging == "bulk":

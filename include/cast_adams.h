@@ -108,10 +108,8 @@ enum cast_flags {
                                        each 1024-parameter tile with bulk asynchronous copies through shared
                                        memory; it is built for: 2:4 with any of CAST_F_RESELECT,
                                        CAST_F_COUNT_FLIPS, CAST_F_META_BITMASK, CAST_F_EMIT_DENSE (not dense and
-                                       bitmask together), with CAST_F_RESELECT | CAST_F_EMIT_COMPRESSED, and for the
-                                       steps of the training schedule (CAST_F_EMIT_DENSE alone or with
-                                       CAST_F_RESELECT | CAST_F_COUNT_FLIPS) also with CAST_F_GRAD_OF_SCALED and / or
-                                       CAST_F_MASK_STATS; groups of 4 or 8 under general N:M with CAST_F_RESELECT |
+                                       bitmask together) and with CAST_F_RESELECT | CAST_F_EMIT_COMPRESSED; groups
+                                       of 4 or 8 under general N:M with CAST_F_RESELECT |
                                        CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS.  On B200 it is as
                                        fast as the plain path in short runs and 2-7 % faster in sustained ones.
                                        Without either switch: a plan step (cast_plan_step) over at least
