@@ -457,8 +457,9 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
             sums.total_abs += mag;
             if (kept[i]) sums.kept_abs += mag;
         }
-        // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for
-        fwd[i] = (kept[i] || Cfg::dense) ? a * wn : 0.0f;
+        // forward weight: scaled (Eq. 12), pruned by the mask unless the dense form is asked for (the compressed
+        // form picks the kept values out afterwards, so it needs no zeros either)
+        fwd[i] = (kept[i] || Cfg::dense || Cfg::compressed) ? a * wn : 0.0f;
     }
     u.g.x = pack_bf16x2(fwd[0], fwd[1]);
     u.g.y = pack_bf16x2(fwd[2], fwd[3]);

@@ -102,7 +102,7 @@ prune_fold_kernel(const __grid_constant__ PruneParams p, int n_keep)
         if (!active) continue;
         float f[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) f[i] = kept[i] ? a[j] * x[j][i] : 0.0f;
+        for (int i = 0; i < 8; ++i) f[i] = (kept[i] || compressed) ? a[j] * x[j][i] : 0.0f;      // compressed: the kept ones are picked out below
         const uint4 packed = make_uint4(pack_bf16x2(f[0], f[1]), pack_bf16x2(f[2], f[3]), pack_bf16x2(f[4], f[5]), pack_bf16x2(f[6], f[7]));
         if constexpr (!compressed) {
             *reinterpret_cast<uint4*>(t.out + (size_t)unit * kUnitElems) = packed;
