@@ -95,14 +95,14 @@ enum cast_flags {
                                        column order; with the metadata it is the whole pruned matrix, and a
                                        step writes 2 N/M instead of 2 bytes per parameter.  M <= 8 only; not
                                        together with CAST_F_EMIT_DENSE                                   */
-    CAST_F_MASK_STATS    = 1u << 7  /* the step also adds the mask statistics the paper monitors (App. C) to a
+    CAST_F_MASK_STATS    = 1u << 7, /* the step also adds the mask statistics the paper monitors (App. C) to a
                                        cast_mask_stats_t, from the registers it holds anyway: ||W_t (.) M_t||_1 and
                                        ||W_t||_1 on the UPDATED weights with this step's kept set M_t, and
                                        ||M_t - M_ref||_0 against the reference mask `meta_ref` of the matrix (the
                                        initial mask for the initial flip rate i_t; 0 is added where meta_ref is
                                        NULL).  Only cast_plan_step_stats takes this flag, on a plan created
                                        with it (other entry points answer CAST_ERR_PLAN)                  */
-    , CAST_F_BULK_STAGING = 1u << 8 /* Two switches that choose how a step moves its data, not what it computes
+    CAST_F_BULK_STAGING  = 1u << 8, /* Two switches that choose how a step moves its data, not what it computes
                                        (results are identical bit for bit).  The plain access path is one thread =
                                        8 consecutive columns by 128-bit loads and stores.  The staged path moves
                                        each 1024-parameter tile with bulk asynchronous copies through shared
@@ -120,7 +120,7 @@ enum cast_flags {
                                        failure mode: its wait for a copy is bounded; a tile whose data has not
                                        arrived by then is left as it was, counted (cast_bulk_timeout_count), and a
                                        plan refuses its next step with CAST_ERR_STAGING                        */
-    , CAST_F_PLAIN_ACCESS = 1u << 9
+    CAST_F_PLAIN_ACCESS  = 1u << 9
 };
 
 /*
