@@ -270,3 +270,48 @@ def test_llama2_7b_whole_set_bulk_staging_every_element():
     _whole_set("llama2_7b", 2, 4, B.CAST_F_RESELECT | B.CAST_F_BULK_STAGING, False, need_gb=125)
     rc, timeouts = cast.cast_bulk_timeout_count()
     assert rc == 0 and timeouts == 0
+
+
+def test_one_matrix_at_the_size_limit_every_element():
+    """The largest matrix the entry points take (rows * cols < 2^31): 65535 x 32768 = 2,147,450,880 parameters, 2^21
+    tiles, unit indices up to 2^28.  Stepped once as a one-matrix plan (staged access path) and once through
+    cast_adams_step (plain path): the two agree bit for bit, and every element matches the oracle (compared in blocks
+    of 2048 rows)."""
+    import gc
+    from types import SimpleNamespace
+    gc.collect()
+    torch.cuda.empty_cache()
+    free, _ = torch.cuda.mem_get_info()
+    if free < 110e9:
+        pytest.skip("needs 110 GB of device memory")
+    rows, cols, N, M = 65535, 32768, 2, 4
+    assert rows * cols < 2 ** 31 <= (rows + 1) * cols
+    flags = B.CAST_F_RESELECT
+    a = DeviceModelState([(rows, cols)], N, M, seed=3, device=DEV, scale_mode="jitter")
+    b = DeviceModelState([(rows, cols)], N, M, seed=3, device=DEV, scale_mode="jitter")
+    h = RunHyper(total_steps=7500)
+    a.step(h, flags)
+    mb = b.mats[0]
+    cast.check(cast.cast_adams_step(mb.w, mb.m, mb.v, mb.g, mb.w_fwd, mb.meta, mb.scale, mb.scale.shape[1], rows, cols, N, M,
+                                    h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps, flags, None, None))
+    torch.cuda.synchronize()
+    ma = a.mats[0]
+    for k in ("w", "m", "v", "w_fwd", "meta"):
+        assert torch.equal(getattr(ma, k), getattr(mb, k)), f"{k}: plan (staged) and single-matrix (plain) launches differ"
+    b.close()
+    del b, mb
+    gc.collect()
+    torch.cuda.empty_cache()
+    again = workloads.gen_tensor_inputs(rows, cols, seed=3, tensor_index=0, device=DEV, scale_mode="jitter")
+    assert torch.equal(again.g, ma.g)
+    oh = orc.Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
+    block = 2048
+    stage = U.HostStage(block * cols)
+    threads = U.host_threads()
+    for r0 in range(0, rows, block):
+        r1 = min(rows, r0 + block)
+        part = SimpleNamespace(rows=r1 - r0, cols=cols, w=ma.w[r0:r1], m=ma.m[r0:r1], v=ma.v[r0:r1], w_fwd=ma.w_fwd[r0:r1], meta=ma.meta[r0:r1])
+        inp = workloads.TensorInputs(again.w[r0:r1], again.g[r0:r1], again.m[r0:r1], again.v[r0:r1], again.scale[r0:r1])
+        U.whole_matrix_parity(part, inp, None, N, M, oh, flags, stage, threads, f"size limit rows {r0}+")
+    assert cast.cast_bulk_timeout_count() == (0, 0)
+    a.close()
