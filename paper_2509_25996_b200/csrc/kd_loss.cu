@@ -339,7 +339,8 @@ extern "C" int cast_kd_loss(const cast_bf16* student_logits, const cast_bf16* te
         cfg.blockDim = dim3(256);
         // Residency is left to the registers (8 CTAs per SM, ~140 rows in flight): capping it at 5 CTAs per SM by a
         // dummy shared-memory request brings the DRAM traffic from 7.6 down to 5.9 B per logit but costs 11 % of time
-        // (0.95 against 0.85 ms for 4096 x 128256): the kernel is bound by the special-function unit, not by bytes.
+        // (0.95 against 0.85 ms for 4096 x 128256), and so does any such request, even one that leaves the residency
+        // alone (28 KB: 0.955 ms): the shared-memory carve-out shrinks the L1 the sweeps run through.
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
