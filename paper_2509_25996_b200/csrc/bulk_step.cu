@@ -1,22 +1,22 @@
 // The AdamS step with its tiles staged through shared memory by bulk asynchronous copies instead of per-thread
-// 128-bit loads and stores (CAST_F_BULK_STAGING).  Same arithmetic (compute_unit of the plain kernels), same results
-// bit for bit.  Built for the configurations a training run and the listed workloads step in (2:4: mask selected or
-// stored, index or bitmask form, pruned or dense emission, with or without flip counting; 4:8 and 1:4 in bitmask
-// form); measured on B200 it is as fast as the plain form in short runs and ~2 % faster in sustained ones (the
-// global accesses bypass the L1/texture path: less power, higher clock under the power cap).
+// 128-bit loads and stores (CAST_F_BULK_STAGING; what plan steps of model size take by default).  Same arithmetic
+// (compute_unit of the plain kernels), same results bit for bit.  Built for the configurations listed at the end of
+// this file; measured on B200 it is as fast as the plain form in short runs and 2-7 % faster in sustained ones (the
+// tile traffic bypasses the L1/texture path: less power, higher clock under the board's power cap).
 //
 // Per CTA (128 threads, one tile of 1024 parameters): one elected thread arms an mbarrier with the tile's byte count
-// and issues four bulk copies global -> shared (w, m, v: 4 KB each, g: 2 KB; this GPU's own memory, no multicast);
-// all threads wait on the barrier's phase, compute from shared memory, write w, m, v and the forward weight back
-// into the same shared memory, make those writes visible to the asynchronous proxy, and the elected thread issues
-// four bulk copies shared -> global and waits until they have read the shared memory.  The metadata byte goes out by
-// an ordinary store.  16 KB of shared memory per CTA, 7 CTAs per SM as in the plain kernel.
+// and issues four bulk copies global -> shared (w, m, v: 4 KB each, g: 2 KB; this GPU's own memory, no multicast).
+// Meanwhile every thread loads what does not come through the tile (its previous metadata byte, its scale), so that
+// these travel with the tile.  All threads then wait on the barrier's phase, compute from shared memory, write w, m, v
+// and the forward weight back into the same shared memory, make those writes visible to the asynchronous proxy, and the
+// elected thread issues four bulk copies shared -> global and waits until they have read the shared memory.  The
+// metadata byte goes out by an ordinary store.  14.4 KB of shared memory and 56 registers: 9 CTAs per SM.
 //
-// The wait on the barrier is bounded (a phase that has not completed after 2^16 polls with back-off, about 2 ms, is counted in a
-// device-side error counter and, for plans, in a word of host memory that the plan's next step checks; the CTA waits
-// once more with the same limit and gives up without storing); the host reads the counter with
-// cast_bulk_timeout_count().  Every copy starts on a 16-byte boundary (tiles start at
-// multiples of 1024 elements of 16-byte aligned buffers) and has a size that is a multiple of 16 bytes.
+// The wait on the barrier is bounded: a phase that has not completed after 2^16 polls with back-off (about 2 ms) is
+// counted in a device-side counter (cast_bulk_timeout_count) and, for plans, in a word of host memory that the plan's
+// next step checks; the CTA waits once more with the same limit and then gives up without storing.  Every copy starts
+// on a 16-byte boundary (tiles start at multiples of 1024 elements of 16-byte aligned buffers) and has a size that is
+// a multiple of 16 bytes (a matrix has a multiple of 4 units).
 #include "cast_internal.h"
 
 namespace cast {
