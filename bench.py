@@ -722,6 +722,31 @@ def cuda_arm(args):
     per_gpu_gbs = wl.n_params * bytes_per_param / (ms_per_step * 1e-3) / 1e9
     peak, peak_kind = measured_hbm_peak()
 
+    # ---- the device's streaming ceiling for this access pattern, measured in this run: cast_probe_stream performs the step's
+    # loads and stores (same launch shape, no arithmetic) over the largest matrices of the first layer; an even number of
+    # launches, because each one flips the signs of w, m, v (two restore them exactly)
+    stream_probe = None
+    if rank == 0 and not wl.resident_layers and not compressed:
+        big = sorted(mats[:min(len(mats), 7)], key=lambda q: -q.rows * q.cols)[:3]
+        n_probe = sum(q.rows * q.cols for q in big)
+
+        def probe_pass():
+            for q in big:
+                cast.check(cast.cast_probe_stream(q.w, q.m, q.v, q.g, q.w_fwd, q.meta, q.rows * q.cols, stream))
+
+        for _ in range(2):
+            probe_pass()
+        pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pa.record(stream)
+        for _ in range(20):
+            probe_pass()
+        pb.record(stream)
+        torch.cuda.synchronize(dev)
+        probe_ms = pa.elapsed_time(pb) / 20
+        stream_probe = {"gbs": n_probe * BYTES_PER_PARAM / (probe_ms * 1e-3) / 1e9, "params_per_pass": n_probe,
+                        "how": "cast_probe_stream (the step's loads and stores in its launch shape, no arithmetic) over the 3 largest "
+                               "matrices of the first layer, 20 passes, CUDA events"}
+
     # ---- e2e leg: the same step through cast_host_step with page-locked HOST buffers; every step copies
     # its inputs host->device and its results device->host inside the timed region
     e2e = None
@@ -866,6 +891,8 @@ def cuda_arm(args):
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": step_launches,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,
+                     "stream_probe": stream_probe,
+                     "frac_of_stream_probe": (None if stream_probe is None else per_gpu_gbs / stream_probe["gbs"]),
                      "traffic": (None if ncu_bpp is None else ncu_bpp * wl.n_params / step_launches),
                      "traffic_from": (None if ncu_bpp is None else
                                       f"ncu dram bytes per parameter of {NCU_KERNEL[args.staging]} on one LLaMA2-7B layer (profiles/), "
