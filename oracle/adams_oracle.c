@@ -149,7 +149,10 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
           double lr_d, double beta1_d, double beta2_d, double eps_d, double l1_coeff_d,
           int64_t step, int64_t total_steps,
           uint32_t flags, uint64_t *flip_count,
-          double *scale_grad)   /* [rows][n_seg], added to; may be NULL; used with ORACLE_F_GRAD_OF_SCALED */
+          double *scale_grad,   /* [rows][n_seg], added to; may be NULL; used with ORACLE_F_GRAD_OF_SCALED */
+          const float *scale_chain) /* [rows][n_seg]: the scale the forward pass that produced g was emitted with, where
+                                       it differs from `scale` (which scales THIS step's emission); NULL = `scale`.
+                                       Only the chain rule dL/dW = A (.) g of ORACLE_F_GRAD_OF_SCALED reads it. */
 {
     if (!w || !m || !v || !g || !w_fwd || !meta) return ORACLE_BAD_ARGS;
     if (rows < 0 || cols < 0 || M < 1 || M > 32 || N < 1 || N > M) return ORACLE_BAD_ARGS;
@@ -161,6 +164,7 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
     if ((flags & ORACLE_F_COUNT_FLIPS) && !flip_count) return ORACLE_BAD_ARGS;
     if ((flags & ORACLE_F_EMIT_COMPRESSED) && (flags & ORACLE_F_EMIT_DENSE)) return ORACLE_BAD_ARGS;
     if (scale_grad && !(flags & ORACLE_F_GRAD_OF_SCALED)) return ORACLE_BAD_ARGS;
+    if (scale_chain && (!scale || !(flags & ORACLE_F_GRAD_OF_SCALED))) return ORACLE_BAD_ARGS;
 
     /* scalars of the step, formed in double and rounded once to the working type */
     const real alpha = (real)((double)step / (double)total_steps);   /* alpha_t = t/T   (Alg. 1) */
@@ -211,7 +215,7 @@ int ENTRY(float *w, float *m, float *v, const uint16_t *g,
                     const int64_t col_g = i * M + j;
                     const int64_t seg = scale ? col_g / (cols / n_seg) : 0;
                     if (scale_grad) scale_grad[r * (scale ? n_seg : 1) + seg] += (double)grad * (double)w[idx];
-                    if (scale) grad = (real)scale[r * n_seg + seg] * grad;
+                    if (scale) grad = (real)(scale_chain ? scale_chain : scale)[r * n_seg + seg] * grad;
                 }
 
                 /* first moment (Alg. 1: mu_t = beta1 mu_{t-1} + (1 - beta1) g_t); stored undecayed */

@@ -41,6 +41,7 @@ def _load():
                 ctypes.c_int64, ctypes.c_int64,                                       # step total_steps
                 ctypes.c_uint32, ctypes.c_void_p,                                     # flags flip_count
                 ctypes.c_void_p,                                                      # scale_grad
+                ctypes.c_void_p,                                                      # scale_chain
             ]
         lib.oracle_prune_fold.restype = ctypes.c_int
         lib.oracle_prune_fold.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
@@ -76,7 +77,7 @@ class Hyper:
 
 
 def adams_step_inplace(w, m, v, g_bits, w_fwd_bits, meta, scale, rows, cols, N, M, hyper: Hyper,
-                       flags: int, precision: str = "f64", scale_grad=None) -> int:
+                       flags: int, precision: str = "f64", scale_grad=None, scale_chain=None) -> int:
     """Run the oracle in place on C-contiguous numpy arrays.
 
     w, m, v: float32 [rows*cols]; g_bits, w_fwd_bits: uint16 (raw bf16);
@@ -97,19 +98,23 @@ def adams_step_inplace(w, m, v, g_bits, w_fwd_bits, meta, scale, rows, cols, N, 
         scale_ptr = scale.ctypes.data
     if scale_grad is not None:
         assert scale_grad.dtype == np.float64 and scale_grad.flags["C_CONTIGUOUS"] and scale_grad.size == rows * n_seg
+    chain_ptr = None
+    if scale_chain is not None:
+        assert scale is not None and scale_chain.dtype == np.float32 and scale_chain.flags["C_CONTIGUOUS"] and scale_chain.shape == scale.shape
+        chain_ptr = scale_chain.ctypes.data
     flips = ctypes.c_uint64(0)
     lr, b1, b2, eps, lam = hyper.as_f32()
     rc = fn(w.ctypes.data, m.ctypes.data, v.ctypes.data, g_bits.ctypes.data,
             w_fwd_bits.ctypes.data, meta.ctypes.data, scale_ptr, n_seg,
             rows, cols, N, M, lr, b1, b2, eps, lam, hyper.step, hyper.total_steps,
-            flags, ctypes.addressof(flips), None if scale_grad is None else scale_grad.ctypes.data)
+            flags, ctypes.addressof(flips), None if scale_grad is None else scale_grad.ctypes.data, chain_ptr)
     if rc != 0:
         raise ValueError(f"oracle rejected its arguments (status {rc})")
     return int(flips.value)
 
 
 def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELECT,
-               meta_in=None, precision: str = "f64"):
+               meta_in=None, precision: str = "f64", scale_chain=None):
     """Out-of-place convenience wrapper for 2-D inputs.
 
     Returns dict(w, m, v, w_fwd (uint16 bf16 bits; [rows, cols*N/M] with F_EMIT_COMPRESSED), meta (uint32
@@ -129,7 +134,8 @@ def adams_step(w, m, v, g_bits, scale, N, M, hyper: Hyper, flags: int = F_RESELE
     scale_grad = None
     if flags & F_GRAD_OF_SCALED:
         scale_grad = np.zeros((rows, 1 if sc is None else sc.shape[1]), dtype=np.float64)
-    flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision, scale_grad)
+    chain = None if scale_chain is None else np.ascontiguousarray(scale_chain, dtype=np.float32)
+    flips = adams_step_inplace(w2, m2, v2, g2, fwd, meta, sc, rows, cols, N, M, hyper, flags, precision, scale_grad, chain)
     return dict(scale_grad=scale_grad, w=w2.reshape(rows, cols), m=m2.reshape(rows, cols), v=v2.reshape(rows, cols),
                 w_fwd=fwd.reshape(rows, fwd_cols), meta=meta.reshape(rows, cols // 32), flips=flips)
 

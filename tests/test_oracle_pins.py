@@ -444,6 +444,16 @@ def test_chain_rule_factor_is_the_scale_passed_to_the_call():
         np.testing.assert_allclose(out["m"], seg * g, rtol=1e-7)
         np.testing.assert_allclose(bf16_bits_to_f32(out["w_fwd"]), seg * out["w"], rtol=2.0 ** -8)
         np.testing.assert_allclose(out["scale_grad"], (g.astype(np.float64) * w0).reshape(3, 2, 32).sum(-1), rtol=1e-12)
+    # the exact form: the forward pass used A_old (chain-rule factor), this step emits with A_new.  torch autograd
+    # on L = sum(c (.) (A_old (.) W)) gives dL/dW = A_old (.) c: that is what the stored first moment must be.
+    W = torch.tensor(w0, dtype=torch.float64, requires_grad=True)
+    A_f = torch.tensor(np.repeat(a_old, 32, axis=1), dtype=torch.float64)
+    (torch.tensor(g, dtype=torch.float64) * (A_f * W)).sum().backward()
+    out = orc.adams_step(w0, np.zeros_like(w0), np.zeros_like(w0), gb, a_new, 4, 4, h, flags, scale_chain=a_old)
+    np.testing.assert_allclose(out["m"], W.grad.numpy(), rtol=1e-7)
+    np.testing.assert_allclose(bf16_bits_to_f32(out["w_fwd"]), np.repeat(a_new, 32, axis=1) * out["w"].astype(np.float64), rtol=2.0 ** -8)
+    both = orc.adams_step(w0, np.zeros_like(w0), np.zeros_like(w0), gb, a_old, 4, 4, h, flags)
+    assert np.array_equal(out["m"], both["m"]) and np.array_equal(out["w"], both["w"])      # only the emission differs
 
 
 # --------------------------------------------------------------------------- numerics and long-run behaviour
