@@ -83,13 +83,13 @@ enum cast_flags {
                                        forward pass used (Eq. 12) instead of the gradient with respect to W: the
                                        step applies the chain rule dL/dW = A (.) g itself and, where a scale_grad
                                        buffer is given, adds dL/dA[r, s] = sum_{c in segment s} g[r, c] W_{t-1}[r, c]
-                                       to it.  The factor A is the `scale` buffer as it stands when the step runs
-                                       (the same buffer also scales the emitted weight).  If the scale is updated
-                                       (cast_scale_adam_step) between the emission of the forward weight that
-                                       produced g and this step, the factor is the updated A_t where the forward
-                                       pass used A_{t-1}: a one-step lag of relative size lr_A, inherent to doing
-                                       the scale gradient and the emission in one pass.  A caller that wants the
-                                       forward's own factor passes the buffer that scaled that emission       */
+                                       to it.  Which A: the forward pass that produced g used the scale of the
+                                       PREVIOUS emission; once the scale is trained (cast_scale_adam_step between
+                                       the steps) that is no longer the `scale` buffer, which holds the updated
+                                       A_t for this step's emission.  Give the previous one as `scale_chain` of the
+                                       matrix (cast_plan_scale_adam_step maintains it); without it the factor is
+                                       `scale` as it stands, i.e. exact while the scale is fixed and one scale
+                                       update (relative size lr_A) off while it is trained                  */
     CAST_F_EMIT_COMPRESSED = 1u << 5, /* emit only the kept entries of the pruned product (Alg. 2, final loop):
                                        w_fwd_bf16 is then [rows][cols*N/M], the N kept values of each group in
                                        column order; with the metadata it is the whole pruned matrix, and a
@@ -197,6 +197,12 @@ typedef struct cast_tensor {
                                 CAST_F_GRAD_OF_SCALED (zero it before the step); may be NULL; needs `scale` */
     const uint32_t* meta_ref;/* device, uint32 [rows*cols/32], same form as `meta`: the reference mask of
                                 CAST_F_MASK_STATS (never written); may be NULL                              */
+    const float* scale_chain;/* device, fp32 [rows][scale_groups]: the scale the forward pass that produced `g` was
+                                emitted with, where that is not `scale` any more (the scale is being trained and
+                                has been updated since).  Read only by steps with CAST_F_GRAD_OF_SCALED, as the
+                                factor of the chain rule dL/dW = A (.) g; `scale` still scales the emission.
+                                NULL = use `scale`.  cast_plan_scale_adam_step keeps it up to date itself (it
+                                stores each scale's value before the update there); needs `scale`              */
 } cast_tensor_t;
 
 /* Hyper-parameters of one iteration (Alg. 1 inputs); ranges as in cast_adams_step. */
@@ -233,7 +239,9 @@ CAST_API int cast_scale_adam_step(float* a, float* m_a, float* v_a, float* grad,
  * The scales and their gradients are the `scale` and `scale_grad` buffers the plan's descriptors name (every matrix
  * must have both; the scale buffers are UPDATED by this call although the descriptor declares them const for the
  * step); `m_a` and `v_a` are HOST arrays of n_tensors device pointers to the two moments of each scale matrix
- * (fp32 [rows * scale_groups]).  Other arguments as cast_scale_adam_step.
+ * (fp32 [rows * scale_groups]).  Where a matrix has a `scale_chain` buffer, the scale's value BEFORE this update is
+ * stored there (the forward pass of the coming iteration was emitted with it, so it is the chain-rule factor of the
+ * next step).  Other arguments as cast_scale_adam_step.
  */
 CAST_API int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* const* v_a,
                               float lr, float beta1, float beta2, float eps, int64_t step,

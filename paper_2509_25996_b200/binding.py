@@ -63,6 +63,7 @@ class cast_tensor_t(ctypes.Structure):
         ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
         ("scale_grad", ctypes.c_void_p),
         ("meta_ref", ctypes.c_void_p),
+        ("scale_chain", ctypes.c_void_p),
     ]
 
 
@@ -227,9 +228,10 @@ def cast_plan_scale_adam_step(plan, m_as, v_as, lr, beta1, beta2, eps, step, cle
                                                     _stream(stream))
 
 
-def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols, scale_grad=None, meta_ref=None) -> cast_tensor_t:
+def make_tensor(w, m, v, g, w_fwd, meta, scale, scale_groups, rows, cols, scale_grad=None, meta_ref=None,
+                scale_chain=None) -> cast_tensor_t:
     return cast_tensor_t(_ptr(w), _ptr(m), _ptr(v), _ptr(g), _ptr(w_fwd), _ptr(meta), _ptr(scale),
-                         int(scale_groups), int(rows), int(cols), _ptr(scale_grad), _ptr(meta_ref))
+                         int(scale_groups), int(rows), int(cols), _ptr(scale_grad), _ptr(meta_ref), _ptr(scale_chain))
 
 
 def cast_adams_step_ex(tensor: Optional[cast_tensor_t], N: int, M: int, hyper: Optional[cast_hyper_t],

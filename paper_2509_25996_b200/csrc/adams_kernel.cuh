@@ -76,6 +76,7 @@ struct TensorDesc {
     const float* scale;        // A[rows][n] or nullptr
     float* scale_grad;         // dL/dA[rows][n], added to, or nullptr
     const uint8_t* meta_ref;   // reference mask of the statistics (same form as meta), or nullptr
+    const float* scale_chain;  // A the forward pass that produced g was scaled with, where it is not `scale`; or nullptr
     uint32_t n_units;          // rows * cols / 8
     uint32_t seg_magic;        // unit / seg_units == (uint64(unit) * seg_magic) >> seg_shift
     uint32_t seg_shift;
@@ -380,7 +381,8 @@ struct StepCfg {
 // roundings of 2^-24), i.e. below 2.5e-10 absolute for updates up to 5e-4, which is under both the
 // fp32 spacing of typical weights (1.9e-9 at 0.02) and the 1e-9 floor of the accepted error.
 template <int M, uint32_t F, bool TF>
-__device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, float a, bool has_ref, float& gw_sum, UnitSums& sums)
+__device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, float a, bool has_ref, float& gw_sum, UnitSums& sums,
+                                             float a_chain = 1.0f)
 {
     using Cfg = StepCfg<M, F, TF>;
     uint32_t ab[8];
@@ -428,7 +430,9 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
     // With kGradOfScaled the gradient is taken with respect to W_scale = Diag(A) W (Eq. 12): the chain rule
     // gives dL/dW = A g (formed exactly in fp64) and dL/dA = sum of g W over the row segment, whose part
     // for this unit is returned in gw_sum (fp32 chain of 8 fused multiply-adds on the weights before the update).
-    const double omb1_g = Cfg::of_scaled ? c.omb1 * (double)a : c.omb1;
+    // The chain-rule factor is a_chain: the scale of the forward pass that produced g (the unit's `a` unless the
+    // caller keeps the previous emission's scale apart from the one being trained).
+    const double omb1_g = Cfg::of_scaled ? c.omb1 * (double)a_chain : c.omb1;
     gw_sum = 0.0f;
     float fwd[8];
 #pragma unroll
@@ -437,7 +441,7 @@ __device__ __forceinline__ void compute_unit(UnitRegs& u, const StepConsts& c, f
         if constexpr (Cfg::of_scaled) gw_sum = fmaf(g32, u.w[i], gw_sum);
         // first moment, stored undecayed (Alg. 1)
         const double mu = fma(c.beta1, (double)u.m[i], omb1_g * (double)g32);
-        if constexpr (Cfg::of_scaled && Cfg::v_from_g) g32 *= a;      // the alternate reading of v below uses dL/dW itself
+        if constexpr (Cfg::of_scaled && Cfg::v_from_g) g32 *= a_chain;      // the alternate reading of v below uses dL/dW itself
         const float mu_f = (float)mu;
         u.m[i] = mu_f;
         // proportional L1 decay outside the kept set (Eq. 7): alpha lambda Sign(w), Sign(+-0) = 0
@@ -497,7 +501,7 @@ __device__ __forceinline__ void process_unit(const TensorDesc& t, const StepCons
     u.prev_byte = 0;
     u.ref_byte = 0;
     const size_t e = (size_t)unit * kUnitElems;
-    float a = 1.0f;
+    float a = 1.0f, a_chain = 1.0f;
     uint32_t seg = 0;
     const bool has_ref = Cfg::stats && t.meta_ref != nullptr;      // uniform over the CTA
 
@@ -511,6 +515,10 @@ __device__ __forceinline__ void process_unit(const TensorDesc& t, const StepCons
         if (t.scale != nullptr) {
             seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
             a = __ldg(t.scale + seg);
+            a_chain = a;
+            if constexpr (Cfg::of_scaled) {
+                if (t.scale_chain != nullptr) a_chain = __ldg(t.scale_chain + seg);
+            }
         }
         u.w[0] = w0.x; u.w[1] = w0.y; u.w[2] = w0.z; u.w[3] = w0.w; u.w[4] = w1.x; u.w[5] = w1.y; u.w[6] = w1.z; u.w[7] = w1.w;
         u.m[0] = m0.x; u.m[1] = m0.y; u.m[2] = m0.z; u.m[3] = m0.w; u.m[4] = m1.x; u.m[5] = m1.y; u.m[6] = m1.z; u.m[7] = m1.w;
@@ -522,7 +530,7 @@ __device__ __forceinline__ void process_unit(const TensorDesc& t, const StepCons
 
     float gw_sum;
     UnitSums mine;
-    compute_unit<M, F, TF>(u, c, a, has_ref, gw_sum, mine);
+    compute_unit<M, F, TF>(u, c, a, has_ref, gw_sum, mine, a_chain);
     if constexpr (Cfg::of_scaled) add_scale_grad(t.scale_grad, seg, active, gw_sum);
 
     if (active) {
@@ -568,6 +576,7 @@ struct MultiParams {
     TensorDesc desc[kMaxLaunchTensors];
 };
 static_assert(sizeof(MultiParams) + sizeof(StepConsts) + 32 <= 32764, "kernel parameters are limited to 32764 bytes");
+static_assert(sizeof(TensorDesc) == 96, "one matrix of a launch table");
 
 // What the CTA counted, added to the caller's counters: one atomic per counter per CTA.
 template <bool FLIPS, bool STATS>

@@ -146,13 +146,14 @@ static void fast_div(uint32_t d, uint32_t* magic, uint32_t* shift)
 
 TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
                      const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad,
-                     const uint32_t* meta_ref)
+                     const uint32_t* meta_ref, const float* scale_chain)
 {
     TensorDesc d;
     std::memset(&d, 0, sizeof d);
     d.w = w; d.m = m; d.v = v; d.g = g; d.w_fwd = w_fwd; d.meta = meta; d.scale = scale;
     d.scale_grad = scale ? scale_grad : nullptr;
     d.meta_ref = reinterpret_cast<const uint8_t*>(meta_ref);
+    d.scale_chain = scale ? scale_chain : nullptr;
     d.n_units = (uint32_t)((uint64_t)rows * (uint64_t)cols / kUnitElems);
     if (scale) {
         const uint32_t seg_units = (uint32_t)(cols / scale_groups / kUnitElems);
@@ -397,6 +398,22 @@ int check_stats_ptr(uint32_t flags, const cast_mask_stats_t* stats)
     const void* p[1] = {stats};
     return check_device_memory(p, 1);
 }
+// The optional second scale of one matrix (the forward pass's): needs `scale`, 16-byte aligned device memory of the
+// same size that the step does not write.
+int check_scale_chain(const cast_tensor_t& t)
+{
+    if (!t.scale_chain) return CAST_OK;
+    if (!t.scale) return CAST_ERR_NULL;
+    if ((uintptr_t)t.scale_chain & 15u) return CAST_ERR_ALIGN;
+    const uint64_t P = (uint64_t)t.rows * (uint64_t)t.cols;
+    const uintptr_t lo = (uintptr_t)t.scale_chain, hi = lo + 4ull * (uint64_t)t.rows * (uint64_t)t.scale_groups;
+    const void* written[6] = {t.w, t.m, t.v, t.w_fwd, t.meta, t.scale_grad};
+    const uint64_t bytes[6] = {4 * P, 4 * P, 4 * P, 2 * P, P / 8, t.scale_grad ? 4ull * (uint64_t)t.rows * (uint64_t)t.scale_groups : 0};
+    for (int i = 0; i < 6; ++i)
+        if (written[i] && lo < (uintptr_t)written[i] + bytes[i] && (uintptr_t)written[i] < hi) return CAST_ERR_ALIAS;
+    const void* p[1] = {t.scale_chain};
+    return check_device_memory(p, 1);
+}
 // The optional reference mask of one matrix: 16-byte aligned device memory that the step does not write.
 int check_meta_ref(const cast_tensor_t& t)
 {
@@ -430,8 +447,9 @@ extern "C" int cast_adams_step_ex(const cast_tensor_t* t, int N, int M, const ca
     if ((rc = check_device_memory(ptrs, 8)) != CAST_OK) return rc;
     if ((rc = check_tensor_scale_grad(*t, N, M, h->flags)) != CAST_OK) return rc;
     if ((rc = check_meta_ref(*t)) != CAST_OK) return rc;
+    if ((rc = check_scale_chain(*t)) != CAST_OK) return rc;
     const TensorDesc d = make_desc(t->w, t->m, t->v, t->g, t->w_fwd, t->meta, t->scale, t->scale_groups, t->rows, t->cols,
-                                   t->scale_grad, t->meta_ref);
+                                   t->scale_grad, t->meta_ref, t->scale_chain);
     return launch_single(d, M, c, flip_count, (cudaStream_t)stream);
 }
 
@@ -466,6 +484,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
         if ((rc = check_device_memory(ptrs, 7)) != CAST_OK) return rc;
         if ((rc = check_tensor_scale_grad(t, N, M, fwd_flags)) != CAST_OK) return rc;
         if ((rc = check_meta_ref(t)) != CAST_OK) return rc;
+        if ((rc = check_scale_chain(t)) != CAST_OK) return rc;
     }
 
     Plan* p = new (std::nothrow) Plan;
@@ -507,7 +526,7 @@ extern "C" int cast_plan_create_ex(const cast_tensor_t* tensors, int n_tensors, 
             while (i < n_tensors && mp.n_tensors < (uint32_t)kMaxLaunchTensors) {
                 const cast_tensor_t& t = tensors[i];
                 const TensorDesc d = make_desc(t.w, t.m, t.v, t.g, t.w_fwd, t.meta, t.scale, t.scale_groups, t.rows, t.cols, t.scale_grad,
-                                               t.meta_ref);
+                                               t.meta_ref, t.scale_chain);
                 if (tiles + tiles_of(d) > kMaxTiles) break;      // a single matrix always fits (rows*cols < 2^31)
                 mp.desc[mp.n_tensors] = d;
                 mp.tile_start[mp.n_tensors] = (uint32_t)tiles;

@@ -50,7 +50,7 @@ int check_device_memory(const void* const* ptrs, int n);
 // Kernel-side description of one (already validated) matrix.
 TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* w_fwd, uint32_t* meta,
                      const float* scale, int scale_groups, int64_t rows, int64_t cols, float* scale_grad = nullptr,
-                     const uint32_t* meta_ref = nullptr);
+                     const uint32_t* meta_ref = nullptr, const float* scale_chain = nullptr);
 
 // The optional scale-gradient buffer of one matrix: needs a scale, 16-byte alignment, device memory, no overlap
 // with the matrix's other buffers (checked by address only).

@@ -27,7 +27,7 @@ __global__ void scale_adam_kernel(float* __restrict__ a, float* __restrict__ m, 
 // All scale matrices of a plan in one grid (each is a few thousand entries: one launch per matrix would be
 // hundreds of launches of a microsecond each).  Tables in kernel parameter space, like the step's.
 constexpr int kScaleTile = 256;
-struct ScaleDesc { float* a; float* m; float* v; float* grad; uint32_t n; uint32_t pad_; };
+struct ScaleDesc { float* a; float* m; float* v; float* grad; float* keep_old; uint32_t n; uint32_t pad_; };   // keep_old: receives a before the update, or nullptr
 struct ScaleParams {
     uint32_t n_tensors;
     uint32_t hint_shift;
@@ -47,6 +47,7 @@ scale_adam_multi_kernel(const __grid_constant__ ScaleParams p, double lr_bc1, do
     const uint32_t i = (tile - p.tile_start[k]) * kScaleTile + threadIdx.x;
     if (i >= t.n) return;
     const double g = (double)t.grad[i];
+    if (t.keep_old != nullptr) t.keep_old[i] = t.a[i];      // the scale the last emission used: the next step's chain-rule factor
     const double mu = beta1 * (double)t.m[i] + (1.0 - beta1) * g;
     const double nu = beta2 * (double)t.v[i] + (1.0 - beta2) * g * g;
     t.m[i] = (float)mu;
@@ -96,7 +97,8 @@ extern "C" int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* c
             plan_tensor_desc(plan, i, &N, &M, &d);
             // entries of A: rows * n = units / (units per segment); recovered from the descriptor's segment divisor
             const uint32_t n_entries = (uint32_t)(((uint64_t)(d.n_units - 1) * d.seg_magic) >> d.seg_shift) + 1;
-            p.desc[p.n_tensors] = ScaleDesc{const_cast<float*>(d.scale), m_a[i], v_a[i], d.scale_grad, n_entries, 0};
+            p.desc[p.n_tensors] = ScaleDesc{const_cast<float*>(d.scale), m_a[i], v_a[i], d.scale_grad, const_cast<float*>(d.scale_chain),
+                                            n_entries, 0};
             p.tile_start[p.n_tensors] = (uint32_t)tiles;
             tiles += (n_entries + kScaleTile - 1) / kScaleTile;
             ++p.n_tensors;

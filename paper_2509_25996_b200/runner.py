@@ -30,6 +30,7 @@ class MatrixState:
     scale_m: Optional[torch.Tensor] = None         # Adam moments of the scale
     scale_v: Optional[torch.Tensor] = None
     meta_ref: Optional[torch.Tensor] = None        # int32 [rows, cols/32]; reference mask of the App. C statistics
+    scale_chain: Optional[torch.Tensor] = None     # fp32 [rows, n]; the scale the last emission used (with a learned scale)
 
 
 @dataclass
@@ -78,6 +79,7 @@ class DeviceModelState:
                 mat.scale_grad = torch.zeros_like(inp.scale)
                 mat.scale_m = torch.zeros_like(inp.scale)
                 mat.scale_v = torch.zeros_like(inp.scale)
+                mat.scale_chain = inp.scale.clone()
             if reference_masks:
                 self.mats[-1].meta_ref = torch.zeros_like(self.mats[-1].meta)
         self.n_params = sum(s.rows * s.cols for s in self.mats)
@@ -87,7 +89,7 @@ class DeviceModelState:
 
     def _make_plan(self) -> None:
         tensors = [B.make_tensor(s.w, s.m, s.v, s.g, s.w_fwd, s.meta, s.scale,
-                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad, s.meta_ref)
+                                 1 if s.scale is None else s.scale.shape[1], s.rows, s.cols, s.scale_grad, s.meta_ref, s.scale_chain)
                    for s in self.mats]
         rc, self.plan = B.cast_plan_create_ex(tensors, self.N, self.M, (B.CAST_F_EMIT_COMPRESSED if self.compressed else 0) |
                                               (B.CAST_F_MASK_STATS if self.reference_masks else 0))

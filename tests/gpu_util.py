@@ -87,9 +87,9 @@ def oracle_flags(flags: int) -> int:
     return out
 
 
-def run_oracle(inp: workloads.TensorInputs, N, M, hyper: orc.Hyper, flags, meta_in=None, precision="f64"):
+def run_oracle(inp: workloads.TensorInputs, N, M, hyper: orc.Hyper, flags, meta_in=None, precision="f64", scale_chain=None):
     w, m, v, g, sc = host_arrays(inp)
-    return orc.adams_step(w, m, v, g, sc, N, M, hyper, oracle_flags(flags), meta_in, precision)
+    return orc.adams_step(w, m, v, g, sc, N, M, hyper, oracle_flags(flags), meta_in, precision, scale_chain)
 
 
 def device_outputs(st: DeviceState, flips=None):

@@ -215,3 +215,56 @@ def test_scale_adam_rejections():
     assert cast.cast_scale_adam_step(x, x, z, g, 64, 1e-3, 0.9, 0.95, 1e-8, 1) == B.CAST_ERR_ALIAS
     assert cast.cast_scale_adam_step(x, y, z, torch.zeros(64), 64, 1e-3, 0.9, 0.95, 1e-8, 1) == B.CAST_ERR_MEMORY
     assert cast.cast_kernel_launch_count() == before
+
+
+@pytest.mark.parametrize("N,M,extra", [(2, 4, 0), (2, 4, B.CAST_F_EMIT_DENSE), (4, 8, BM), (8, 16, BM)])
+def test_chain_rule_with_the_scale_of_the_forward_pass(N, M, extra):
+    """A trained scale: the forward pass that produced g was emitted with A_old (`scale_chain`), this step emits with
+    the updated A_new (`scale`).  The chain rule must use A_old, the emission A_new, exactly as the oracle does."""
+    rows, cols, n_seg = 5, 2080 if M <= 8 else 2048, 2
+    inp = scaled_inputs(rows, cols, n_seg, seed=260)
+    gen = torch.Generator().manual_seed(261)
+    a_old = (inp.scale * (1.0 + 0.05 * torch.rand((rows, n_seg), generator=gen))).contiguous()
+    h = Hyper()
+    flags = RS | extra | GS
+    st = U.to_device(inp, DEV)
+    sg = torch.zeros((rows, n_seg), dtype=torch.float32, device=DEV)
+    chain = a_old.to(DEV)
+    t = B.make_tensor(st.w.view, st.m.view, st.v.view, st.g.view, st.w_fwd.view, st.meta.view, st.scale, n_seg, rows, cols, sg, None, chain)
+    cast.check(cast.cast_adams_step_ex(t, N, M, hyper_struct(h, flags), None, torch.cuda.current_stream()))
+    torch.cuda.synchronize()
+    assert st.all_intact()
+    ref = U.run_oracle(inp, N, M, h, flags, scale_chain=a_old.numpy())
+    U.assert_parity(U.device_outputs(st), ref, f"two scales {N}:{M}")
+    assert_scale_grad(sg.cpu().numpy(), inp, ref["scale_grad"], n_seg, "scale grad with two scales")
+    same = U.run_oracle(inp, N, M, h, flags)                        # and it does differ from the one-scale result
+    assert not np.array_equal(same["m"], ref["m"])
+
+
+def test_plan_scale_adam_keeps_the_previous_scale_for_the_next_chain_rule():
+    """Two iterations of weights and scales through a plan with `scale_chain` buffers: the scale Adam step stores each
+    scale's value before its update, and the next AdamS step's chain rule uses that stored value while its emission
+    uses the updated scale -- checked against the oracle fed the two scales the same way."""
+    from paper_2509_25996_b200.runner import DeviceModelState, Hyper as RunHyper
+    shapes = [(6, 1056), (9, 2048)]
+    st = DeviceModelState(shapes, 2, 4, seed=11, device=DEV, scale_mode="jitter", learned_scale=True)
+    h = RunHyper(total_steps=30000)
+    flags = RS | GS | B.CAST_F_EMIT_DENSE | B.CAST_F_PLAIN_ACCESS
+    st.step(h, flags)                                               # iteration 1: chain = scale (initially equal)
+    a_before = [m.scale.clone() for m in st.mats]
+    st.scale_step(1e-2, h)                                          # A_1 -> A_2; chain buffers now hold A_1
+    torch.cuda.synchronize()
+    for m, a0 in zip(st.mats, a_before):
+        assert torch.equal(m.scale_chain, a0) and not torch.equal(m.scale, a0)
+    h.step += 1
+    st.fresh_gradients(h.step)
+    snaps = [workloads.TensorInputs(m.w.cpu(), m.g.cpu(), m.m.cpu(), m.v.cpu(), m.scale.cpu()) for m in st.mats]
+    chains = [m.scale_chain.cpu().numpy() for m in st.mats]
+    st.step(h, flags)                                               # iteration 2: chain rule with A_1, emission with A_2
+    torch.cuda.synchronize()
+    oh = orc.Hyper(h.lr, h.beta1, h.beta2, h.eps, h.l1_coeff, h.step, h.total_steps)
+    for i, (m, inp, ch) in enumerate(zip(st.mats, snaps, chains)):
+        got = dict(w=m.w.cpu().numpy(), m=m.m.cpu().numpy(), v=m.v.cpu().numpy(), w_fwd=workloads.bf16_bits(m.w_fwd),
+                   meta=m.meta.cpu().numpy().view(np.uint32))
+        U.assert_parity(got, U.run_oracle(inp, 2, 4, oh, flags & ~B.CAST_F_PLAIN_ACCESS, scale_chain=ch), f"iteration 2 matrix {i}")
+    st.close()
