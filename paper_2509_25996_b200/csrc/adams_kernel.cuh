@@ -76,7 +76,7 @@ struct TensorDesc {
     const float* scale;        // A[rows][n] or nullptr
     float* scale_grad;         // dL/dA[rows][n], added to, or nullptr
     const uint8_t* meta_ref;   // reference mask of the statistics (same form as meta), or nullptr
-    const float* scale_chain;  // A the forward pass that produced g was scaled with, where it is not `scale`; or nullptr
+    const float* scale_chain;  // A the forward pass that produced g was scaled with (`scale` itself where the caller gave none)
     uint32_t n_units;          // rows * cols / 8
     uint32_t seg_magic;        // unit / seg_units == (uint64(unit) * seg_magic) >> seg_shift
     uint32_t seg_shift;
@@ -515,10 +515,7 @@ __device__ __forceinline__ void process_unit(const TensorDesc& t, const StepCons
         if (t.scale != nullptr) {
             seg = (uint32_t)(((uint64_t)unit * t.seg_magic) >> t.seg_shift);   // row * n + segment of the row
             a = __ldg(t.scale + seg);
-            a_chain = a;
-            if constexpr (Cfg::of_scaled) {
-                if (t.scale_chain != nullptr) a_chain = __ldg(t.scale_chain + seg);
-            }
+            if constexpr (Cfg::of_scaled) a_chain = __ldg(t.scale_chain + seg);      // the host points it at `scale` where there is no other
         }
         u.w[0] = w0.x; u.w[1] = w0.y; u.w[2] = w0.z; u.w[3] = w0.w; u.w[4] = w1.x; u.w[5] = w1.y; u.w[6] = w1.z; u.w[7] = w1.w;
         u.m[0] = m0.x; u.m[1] = m0.y; u.m[2] = m0.z; u.m[3] = m0.w; u.m[4] = m1.x; u.m[5] = m1.y; u.m[6] = m1.z; u.m[7] = m1.w;

@@ -153,7 +153,7 @@ TensorDesc make_desc(float* w, float* m, float* v, const uint16_t* g, uint16_t* 
     d.w = w; d.m = m; d.v = v; d.g = g; d.w_fwd = w_fwd; d.meta = meta; d.scale = scale;
     d.scale_grad = scale ? scale_grad : nullptr;
     d.meta_ref = reinterpret_cast<const uint8_t*>(meta_ref);
-    d.scale_chain = scale ? scale_chain : nullptr;
+    d.scale_chain = scale ? (scale_chain ? scale_chain : scale) : nullptr;
     d.n_units = (uint32_t)((uint64_t)rows * (uint64_t)cols / kUnitElems);
     if (scale) {
         const uint32_t seg_units = (uint32_t)(cols / scale_groups / kUnitElems);

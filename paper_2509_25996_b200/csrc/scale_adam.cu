@@ -97,8 +97,9 @@ extern "C" int cast_plan_scale_adam_step(void* plan, float* const* m_a, float* c
             plan_tensor_desc(plan, i, &N, &M, &d);
             // entries of A: rows * n = units / (units per segment); recovered from the descriptor's segment divisor
             const uint32_t n_entries = (uint32_t)(((uint64_t)(d.n_units - 1) * d.seg_magic) >> d.seg_shift) + 1;
-            p.desc[p.n_tensors] = ScaleDesc{const_cast<float*>(d.scale), m_a[i], v_a[i], d.scale_grad, const_cast<float*>(d.scale_chain),
-                                            n_entries, 0};
+            // a descriptor without a second scale names `scale` itself there: nothing to keep
+            p.desc[p.n_tensors] = ScaleDesc{const_cast<float*>(d.scale), m_a[i], v_a[i], d.scale_grad,
+                                            d.scale_chain != d.scale ? const_cast<float*>(d.scale_chain) : nullptr, n_entries, 0};
             p.tile_start[p.n_tensors] = (uint32_t)tiles;
             tiles += (n_entries + kScaleTile - 1) / kScaleTile;
             ++p.n_tensors;
