@@ -32,7 +32,7 @@ namespace cast {
 constexpr int kThreads = 128;          // threads per CTA
 constexpr int kUnitElems = 8;          // parameters per thread
 constexpr int kTileUnits = kThreads;   // units per tile (1024 parameters)
-constexpr int kMinCtasPerSm = 7;       // register budget the kernels are compiled for
+constexpr int kMinCtasPerSm = 7;       // register budget most kernels are compiled for (plain_ctas_per_sm below)
 
 // flag bits (values of the public header)
 constexpr uint32_t kReselect = 1u << 0;
@@ -621,8 +621,24 @@ __device__ __forceinline__ void add_sums(UnitSums x, unsigned long long* flip_co
 }
 
 // One matrix: CTA b handles tile b.
+// Resident CTAs per SM a variant of the plain kernels is compiled for (85, 73, 64 registers per thread at 6, 7, 8).  In
+// sustained runs under the board's power cap the variants that do more work per parameter react to the budget by 1-4 %,
+// in either direction; the exceptions to 7 are the measured winners on the LLaMA2-7B set (ms per step at 6 / 7 / 8):
+// 2:4 refresh 27.45 / 28.7 / 27.97, 2:4 refresh with the statistics 28.9 / 28.7 / 27.7, 4:8 select 28.2 / 27.8 / 27.2, 4:8
+// refresh with the scale gradient 31.3 / 28.6 / 27.97, 8:16 select 28.4 / 27.3 / 26.8, 8:16 select + flips 28.4 / 29.3 /
+// 29.2, 8:32 select 29.1 / 28.4 / 28.0, 8:32 select + flips 28.97 / 30.3 / 29.45.
 template <int M, uint32_t F, bool TF>
-__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+constexpr int plain_ctas_per_sm()
+{
+    constexpr uint32_t refresh = kReselect | kCountFlips | kEmitDense;
+    if (TF) return F == refresh ? 6 : F == (refresh | kMaskStats) ? 8 : kMinCtasPerSm;
+    if (M == 8) return 8;
+    if (M >= 16) return (F & kGradOfScaled) ? kMinCtasPerSm : (F & kCountFlips) ? 6 : 8;
+    return kMinCtasPerSm;
+}
+
+template <int M, uint32_t F, bool TF>
+__global__ void __launch_bounds__(kThreads, plain_ctas_per_sm<M, F, TF>())
 adams_nm_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c,
                 unsigned long long* __restrict__ flip_count, MaskStats* __restrict__ stats)
 {
@@ -634,7 +650,7 @@ adams_nm_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ St
 
 // Up to kMaxLaunchTensors matrices in one grid: CTA b handles tile b of the concatenated index space.
 template <int M, uint32_t F, bool TF>
-__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+__global__ void __launch_bounds__(kThreads, plain_ctas_per_sm<M, F, TF>())
 adams_nm_multi_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
                       unsigned long long* __restrict__ flip_count, MaskStats* __restrict__ stats)
 {

@@ -10,7 +10,8 @@
 // these travel with the tile.  All threads then wait on the barrier's phase, compute from shared memory, write w, m, v
 // and the forward weight back into the same shared memory, make those writes visible to the asynchronous proxy, and the
 // elected thread issues four bulk copies shared -> global and waits until they have read the shared memory.  The
-// metadata byte goes out by an ordinary store.  14.4 KB of shared memory and 56 registers: 9 CTAs per SM.
+// metadata byte goes out by an ordinary store.  14.4 KB of shared memory; the register budget (8, 9 or 10 CTAs per SM) is
+// chosen per variant from measurements (staged_ctas_per_sm below).
 //
 // The wait on the barrier is bounded: a phase that has not completed after 2^16 polls with back-off (about 2 ms) is
 // counted in a device-side counter (cast_bulk_timeout_count) and, for plans, in a word of host memory that the plan's
@@ -172,8 +173,21 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
     add_sums<Cfg::count_flips, false>(sums, flip_count, nullptr);
 }
 
+// Resident CTAs per SM a variant is compiled for (64, 56 or 48 registers per thread).  Sustained runs are limited by the
+// board's power cap as much as by HBM, and which budget wins depends on the code ptxas makes of each variant: measured on
+// the LLaMA2-7B set (ms per step at 8 / 9 / 10 CTAs): select 26.64 / 26.84 / 27.10, select + dense 26.59 / 26.71 / 26.68,
+// select + flips 28.3 / 27.7 / 31.2, refresh (select + flips + dense) 28.1 / 26.9 / 30.8, bitmask + flips 27.45 / 27.8 /
+// 27.27, stored mask 26.25 / 26.15 / 26.37, 4:8 select 27.8 / 26.3 / 29.1, 4:8 select + flips 28.7 / 27.25 / 29.7.
 template <int M, uint32_t F, bool TF>
-__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+constexpr int staged_ctas_per_sm()
+{
+    if (TF && (F == kReselect || F == (kReselect | kEmitDense))) return 8;
+    if (TF && F == (kReselect | kMetaBitmask | kCountFlips)) return 10;
+    return 9;
+}
+
+template <int M, uint32_t F, bool TF>
+__global__ void __launch_bounds__(kThreads, staged_ctas_per_sm<M, F, TF>())
 adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c, unsigned long long* __restrict__ flip_count,
                      unsigned long long* fail_word)
 {
@@ -181,7 +195,7 @@ adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant
 }
 
 template <int M, uint32_t F, bool TF>
-__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
+__global__ void __launch_bounds__(kThreads, staged_ctas_per_sm<M, F, TF>())
 adams_nm_multi_bulk_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
                            unsigned long long* __restrict__ flip_count, unsigned long long* fail_word)
 {
