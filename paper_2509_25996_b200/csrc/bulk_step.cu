@@ -1,7 +1,7 @@
 // The AdamS step with its tiles staged through shared memory by bulk asynchronous copies instead of per-thread
 // 128-bit loads and stores (CAST_F_BULK_STAGING; what plan steps of model size take by default).  Same arithmetic
 // (compute_unit of the plain kernels), same results bit for bit.  Built for the configurations listed at the end of
-// this file; measured on B200 it is as fast as the plain form in short runs and 2-7 % faster in sustained ones (the
+// this file; measured on B200 it is as fast as the plain form in short runs and 0-3 % faster in sustained ones (the
 // tile traffic bypasses the L1/texture path: less power, higher clock under the board's power cap).
 //
 // Per CTA (128 threads, one tile of 1024 parameters): one elected thread arms an mbarrier with the tile's byte count
