@@ -234,6 +234,12 @@ int launch_multi(const MultiParams& p, int M, const StepConsts& c, unsigned long
                  MaskStats* stat_slots, unsigned long long* fail_word)
 {
     // a plan that owns a failure word lets the library choose the access path
+    if (p.n_tensors == 1 && stat_slots == nullptr) {
+        // one matrix: the single-matrix kernels take a 96-byte descriptor instead of the 32 KB table (a launch of a
+        // few thousand CTAs is 2-3 us shorter: 3072 x 768, cold, 17.6 against 20.1 us)
+        const StepLaunch one = {&p.desc[0], nullptr, &c, flip_count, nullptr, stream, fail_word, fail_word != nullptr};
+        return launch_step(one, M);
+    }
     const StepLaunch a = {nullptr, &p, &c, flip_count, stat_slots, stream, fail_word, fail_word != nullptr};
     return launch_step(a, M);
 }
