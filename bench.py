@@ -887,7 +887,7 @@ def cuda_arm(args):
                      "note": "same steps back to back without the flush: the state stays in L2, not an HBM figure"}),
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "achieved": per_gpu_gbs, "peak": peak, "unit": "GB/s", "frac": per_gpu_gbs / peak,
-                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi{'_bulk' if args.staging == 'bulk' else ''}_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step))}, {1 if (N, M) == (2, 4) else 0}>",
+                     "peak_kind": f"of {peak_kind}", "kernel": f"adams_nm_multi{'_bulk' if args.staging == 'bulk' else ''}_kernel<{M}, {B.kernel_flag_word(flags_at(hyper.step) | (B.CAST_F_EMIT_COMPRESSED if args.emit == 'compressed' else 0))}, {1 if (N, M) == (2, 4) else 0}>",
                      "bytes_per_param": bytes_per_param,
                      "launches_per_step": step_launches,
                      "algorithmic_bytes_per_launch": bytes_per_param * wl.n_params / step_launches,
