@@ -10,7 +10,7 @@
 // these travel with the tile.  All threads then wait on the barrier's phase, compute from shared memory, write w, m, v
 // and the forward weight back into the same shared memory, make those writes visible to the asynchronous proxy, and the
 // elected thread issues four bulk copies shared -> global and waits until they have read the shared memory.  The
-// metadata byte goes out by an ordinary store.  14.4 KB of shared memory; the register budget (8, 9 or 10 CTAs per SM) is
+// metadata byte goes out by an ordinary store.  14.4 KB of shared memory; the register budget (8 or 9 CTAs per SM) is
 // chosen per variant from measurements (staged_ctas_per_sm below).
 //
 // The wait on the barrier is bounded: a phase that has not completed after 2^16 polls with back-off (about 2 ms) is
@@ -158,6 +158,13 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
         __syncthreads();
         if (active) *reinterpret_cast<uint2*>(tile.g + u_idx * 4) = kept_out;
     }
+    // The flip count rides on the barrier the stores need anyway: a reduction after the stores made every warp wait
+    // for the elected thread's wait on them (4:8 with flips over the 7B set: 27.45 against 26.35 ms).
+    __shared__ uint32_t warp_flips[kThreads / 32];
+    if constexpr (Cfg::count_flips) {
+        const uint32_t f = __reduce_add_sync(0xFFFFFFFFu, sums.flips);
+        if ((threadIdx.x & 31) == 0) warp_flips[threadIdx.x >> 5] = f;
+    }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's shared-memory writes, for the bulk stores
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -168,22 +175,27 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
         if constexpr (Cfg::compressed) bulk_store(t.w_fwd + e0 / 2, smem_addr(tile.g), b2 / 2);      // units are a multiple of 4: 16-byte sizes
         else bulk_store(t.w_fwd + e0, smem_addr(tile.g), b2);
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+        if constexpr (Cfg::count_flips) {
+            unsigned long long total = 0;
+#pragma unroll
+            for (int i = 0; i < kThreads / 32; ++i) total += warp_flips[i];
+            if (total) atomicAdd(flip_count, total);
+        }
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the shared memory has been read: the CTA may end
     }
-    add_sums<Cfg::count_flips, false>(sums, flip_count, nullptr);
 }
 
-// Resident CTAs per SM a variant is compiled for (64, 56 or 48 registers per thread).  Sustained runs are limited by the
-// board's power cap as much as by HBM, and which budget wins depends on the code ptxas makes of each variant: measured on
-// the LLaMA2-7B set (ms per step at 8 / 9 / 10 CTAs): select 26.64 / 26.84 / 27.10, select + dense 26.59 / 26.71 / 26.68,
-// select + flips 28.3 / 27.7 / 31.2, refresh (select + flips + dense) 28.1 / 26.9 / 30.8, bitmask + flips 27.45 / 27.8 /
-// 27.27, stored mask 26.25 / 26.15 / 26.37, 4:8 select 27.8 / 26.3 / 29.1, 4:8 select + flips 28.7 / 27.25 / 29.7.
+// Resident CTAs per SM a variant is compiled for (64 or 56 registers per thread; 48 was measured too).  Sustained runs
+// are limited by the board's power cap as much as by HBM, and which budget wins depends on the code ptxas makes of each
+// variant: measured on the LLaMA2-7B set (ms per step at 8 / 9 / 10 CTAs): select 26.70 / 26.94 / 27.1, select + flips
+// 27.2 / 27.5 / 29.8, bitmask 26.76 / 26.82 / 27.06, bitmask + flips 27.2 / 27.4 / 28.7, select + dense 26.65 / 26.77 /
+// 26.70, refresh (select + flips + dense) 27.05 / 26.8 / 28.8, stored mask 26.23 / 26.15 / 26.36, 4:8 select 27.0 /
+// 26.3 / 29.1, 4:8 select + flips 27.4 / 26.95 / 29.4, 1:4 select + flips 26.6 / 26.4 / 27.2.
 template <int M, uint32_t F, bool TF>
 constexpr int staged_ctas_per_sm()
 {
-    if (TF && (F == kReselect || F == (kReselect | kEmitDense))) return 8;
-    if (TF && F == (kReselect | kMetaBitmask | kCountFlips)) return 10;
-    return 9;
+    constexpr uint32_t refresh = kReselect | kCountFlips | kEmitDense;
+    return (TF && (F & kReselect) && F != refresh) ? 8 : 9;
 }
 
 template <int M, uint32_t F, bool TF>
