@@ -110,8 +110,9 @@ enum cast_flags {
                                        CAST_F_COUNT_FLIPS, CAST_F_META_BITMASK, CAST_F_EMIT_DENSE (not dense and
                                        bitmask together) and with CAST_F_RESELECT | CAST_F_EMIT_COMPRESSED; groups
                                        of 4 or 8 under general N:M with CAST_F_RESELECT |
-                                       CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS.  On B200 it is as
-                                       fast as the plain path in short runs and 2-7 % faster in sustained ones.
+                                       CAST_F_META_BITMASK, with or without CAST_F_COUNT_FLIPS; 2:4 with
+                                       CAST_F_EMIT_DENSE | CAST_F_MASK_STATS (plans).  On B200 it is as fast as
+                                       the plain path in short runs and 0-3 % faster in sustained ones.
                                        Without either switch: a plan step (cast_plan_step) over at least
                                        16.8 M parameters takes the staged path where it is built, everything
                                        else the plain one.

@@ -75,10 +75,10 @@ struct __align__(128) BulkTile {
 
 template <int M, uint32_t F, bool TF>
 __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts& c, uint32_t first_unit,
-                                          unsigned long long* flip_count, unsigned long long* fail_word)
+                                          unsigned long long* flip_count, MaskStats* stats, unsigned long long* fail_word)
 {
     using Cfg = StepCfg<M, F, TF>;
-    static_assert(M <= 8 && !Cfg::of_scaled && !Cfg::stats, "staged form: groups inside a thread, no scale gradient, no statistics");
+    static_assert(M <= 8 && !Cfg::of_scaled, "staged form: groups inside a thread, no scale gradient");
     static_assert(!Cfg::compressed || (TF && !Cfg::bitmask), "staged compressed emission: 2:4 with index-form metadata");
     __shared__ BulkTile tile;
     const uint32_t units = min((uint32_t)kTileUnits, t.n_units - first_unit);       // a matrix's last tile may be short
@@ -96,10 +96,12 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
     // what does not come through the tile is asked for now, so that it travels while the tile does
     const uint32_t u_idx = threadIdx.x;
     const bool active = u_idx < units;
-    uint32_t prev_byte = 0;
+    uint32_t prev_byte = 0, ref_byte = 0;
     float a = 1.0f;
+    const bool has_ref = Cfg::stats && t.meta_ref != nullptr;      // uniform over the CTA
     if (active) {
         if constexpr (Cfg::need_prev) prev_byte = reinterpret_cast<const uint8_t*>(t.meta)[first_unit + u_idx];
+        if (has_ref) ref_byte = t.meta_ref[first_unit + u_idx];
         if (t.scale != nullptr) a = __ldg(t.scale + (uint32_t)(((uint64_t)(first_unit + u_idx) * t.seg_magic) >> t.seg_shift));
     }
     __syncthreads();                            // the barrier is initialised before anyone polls it
@@ -131,9 +133,9 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
         for (int i = 0; i < 8; ++i) { u.w[i] = 0.f; u.m[i] = 0.f; u.v[i] = 0.f; }
     }
     u.prev_byte = prev_byte;
-    u.ref_byte = 0;
+    u.ref_byte = ref_byte;
     UnitSums mine;
-    compute_unit<M, F, TF>(u, c, a, false, gw_sum, mine);
+    compute_unit<M, F, TF>(u, c, a, has_ref, gw_sum, mine);
     if (active) {
         sums = mine;
         *reinterpret_cast<float4*>(tile.w + u_idx * 8) = make_float4(u.w[0], u.w[1], u.w[2], u.w[3]);
@@ -160,10 +162,21 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
     }
     // The flip count rides on the barrier the stores need anyway: a reduction after the stores made every warp wait
     // for the elected thread's wait on them (4:8 with flips over the 7B set: 27.45 against 26.35 ms).
-    __shared__ uint32_t warp_flips[kThreads / 32];
+    __shared__ uint32_t warp_flips[kThreads / 32], warp_diff[kThreads / 32];
+    __shared__ double warp_kept[kThreads / 32], warp_total[kThreads / 32];
     if constexpr (Cfg::count_flips) {
         const uint32_t f = __reduce_add_sync(0xFFFFFFFFu, sums.flips);
         if ((threadIdx.x & 31) == 0) warp_flips[threadIdx.x >> 5] = f;
+    }
+    if constexpr (Cfg::stats) {      // the App. C sums of the step's epilogue take the same ride
+        const uint32_t d = __reduce_add_sync(0xFFFFFFFFu, sums.mask_diff);
+        double k = sums.kept_abs, tt = sums.total_abs;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            k += __shfl_down_sync(0xFFFFFFFFu, k, o);
+            tt += __shfl_down_sync(0xFFFFFFFFu, tt, o);
+        }
+        if ((threadIdx.x & 31) == 0) { warp_diff[threadIdx.x >> 5] = d; warp_kept[threadIdx.x >> 5] = k; warp_total[threadIdx.x >> 5] = tt; }
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // this thread's shared-memory writes, for the bulk stores
     __syncthreads();
@@ -180,6 +193,16 @@ __device__ __forceinline__ void bulk_tile(const TensorDesc& t, const StepConsts&
 #pragma unroll
             for (int i = 0; i < kThreads / 32; ++i) total += warp_flips[i];
             if (total) atomicAdd(flip_count, total);
+        }
+        if constexpr (Cfg::stats) {
+            unsigned long long d = 0;
+            double k = 0.0, tt = 0.0;
+#pragma unroll
+            for (int i = 0; i < kThreads / 32; ++i) { d += warp_diff[i]; k += warp_kept[i]; tt += warp_total[i]; }
+            MaskStats* slot = stats + (blockIdx.x & (kStatSlots - 1u));
+            if (d) atomicAdd(&slot->mask_diff, d);
+            atomicAdd(&slot->kept_abs_sum, k);
+            atomicAdd(&slot->total_abs_sum, tt);
         }
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");      // the shared memory has been read: the CTA may end
     }
@@ -203,25 +226,30 @@ __global__ void __launch_bounds__(kThreads, staged_ctas_per_sm<M, F, TF>())
 adams_nm_bulk_kernel(const __grid_constant__ TensorDesc t, const __grid_constant__ StepConsts c, unsigned long long* __restrict__ flip_count,
                      unsigned long long* fail_word)
 {
-    bulk_tile<M, F, TF>(t, c, blockIdx.x * kTileUnits, flip_count, fail_word);
+    bulk_tile<M, F, TF>(t, c, blockIdx.x * kTileUnits, flip_count, nullptr, fail_word);
 }
 
 template <int M, uint32_t F, bool TF>
 __global__ void __launch_bounds__(kThreads, staged_ctas_per_sm<M, F, TF>())
 adams_nm_multi_bulk_kernel(const __grid_constant__ MultiParams p, const __grid_constant__ StepConsts c,
-                           unsigned long long* __restrict__ flip_count, unsigned long long* fail_word)
+                           unsigned long long* __restrict__ flip_count, MaskStats* __restrict__ stats, unsigned long long* fail_word)
 {
     const uint32_t tile = blockIdx.x;
     uint32_t k = p.hint[tile >> p.hint_shift];
     while (tile >= p.tile_start[k + 1]) ++k;
-    bulk_tile<M, F, TF>(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits, flip_count, fail_word);
+    bulk_tile<M, F, TF>(p.desc[k], c, (tile - p.tile_start[k]) * kTileUnits, flip_count, stats, fail_word);
 }
 
 template <int M, uint32_t F, bool TF>
 int launch_bulk_t(const StepLaunch& a)
 {
-    if (a.single) adams_nm_bulk_kernel<M, F, TF><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.fail_word);
-    else adams_nm_multi_bulk_kernel<M, F, TF><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(*a.multi, *a.c, a.flip_count, a.fail_word);
+    if (a.single) {
+        if constexpr ((F & kMaskStats) != 0) return CAST_ERR_NM;      // the statistics epilogue exists for plans only
+        else adams_nm_bulk_kernel<M, F, TF><<<tiles_of(*a.single), kThreads, 0, a.stream>>>(*a.single, *a.c, a.flip_count, a.fail_word);
+    } else {
+        adams_nm_multi_bulk_kernel<M, F, TF><<<a.multi->tile_start[a.multi->n_tensors], kThreads, 0, a.stream>>>(
+            *a.multi, *a.c, a.flip_count, a.stats, a.fail_word);
+    }
     CAST_CUDA_TRY(cudaGetLastError());
     return CAST_OK;
 }
@@ -230,11 +258,12 @@ int launch_bulk_t(const StepLaunch& a)
 //   2:4:      select (index or bitmask form), with flips, with dense emission; stored mask with pruned / dense emission
 //   general N:M in groups of 4 or 8 (4:8, 1:4, ...): select, with flips (bitmask form)
 //   2:4 also: compressed emission with index-form metadata
-// (the steps with the scale gradient or the statistics epilogue were measured in this form too and are faster plain:
-//  refresh + scale gradient 28.2 against 26.85 ms, refresh + statistics 27.9-28.1 against 27.3 ms per 7B step)
-constexpr uint32_t RS = kReselect, FL = kCountFlips, BM = kMetaBitmask, DN = kEmitDense, CP = kEmitCompressed;
+//   2:4 also: the stored-mask step with the statistics epilogue (26.6 against 27.65 ms plain)
+// (measured in this form too and faster plain: the refresh step with the statistics epilogue, 27.6 against 26.8 ms per 7B
+//  step, and the steps with the scale gradient, refresh 28.2 against 26.85 ms)
+constexpr uint32_t RS = kReselect, FL = kCountFlips, BM = kMetaBitmask, DN = kEmitDense, CP = kEmitCompressed, ST = kMaskStats;
 #define CAST_BULK_CASES_2OF4(X) X(4, RS, true) X(4, RS | FL, true) X(4, RS | BM, true) X(4, RS | BM | FL, true) X(4, RS | DN, true) \
-    X(4, RS | FL | DN, true) X(4, 0u, true) X(4, DN, true) X(4, RS | CP, true)
+    X(4, RS | FL | DN, true) X(4, 0u, true) X(4, DN, true) X(4, RS | CP, true) X(4, DN | ST, true)
 // (groups of 16 and 32 columns were measured in this form too: 31.0 / 33.1 against 26.8 / 27.8 ms on the plain path --
 // the sorted keys of the cross-lane merge end up in local memory next to the tile code -- so they stay plain)
 #define CAST_BULK_CASES_NM(X) X(4, RS | BM, false) X(4, RS | BM | FL, false) X(8, RS | BM, false) X(8, RS | BM | FL, false)

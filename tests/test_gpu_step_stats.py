@@ -107,6 +107,30 @@ def test_step_with_statistics_matches_oracle(N, M, flags, what, rows, cols):
             assert stats["flips"] == 0
 
 
+@pytest.mark.parametrize("flags,what", [(DN, "stored 2:4 mask, index form, dense emission")])
+@pytest.mark.parametrize("rows,cols", [(1, 32), (5, 96), (7, 2080), (33, 1056)])
+def test_staged_step_with_statistics_matches_oracle(flags, what, rows, cols):
+    """The same on the staged access path (the sums ride on the barrier before the tile's stores), forced by flag: a
+    plan takes it by itself only for launches of model size."""
+    inp = workloads.gen_tensor_inputs(rows, cols, seed=24, tensor_index=7, device="cpu", scale_mode="jitter")
+    if (cols // 2) % 8 != 0:
+        inp.scale = None
+    other = workloads.gen_tensor_inputs(rows, cols, seed=25, tensor_index=1, device="cpu", scale_mode="none")
+    third = workloads.gen_tensor_inputs(rows, cols, seed=26, tensor_index=2, device="cpu", scale_mode="none")
+    meta_in = U.run_oracle(other, 2, 4, Hyper(lr=0.0), RS)["meta"]
+    meta_ref = U.run_oracle(third, 2, 4, Hyper(lr=0.0), RS)["meta"]
+    h = Hyper()
+    want = U.run_oracle(inp, 2, 4, h, flags, meta_in=meta_in)
+    for ref in (meta_ref, None):
+        got, stats = step_with_stats(inp, 2, 4, h, flags | ST | B.CAST_F_BULK_STAGING, meta_in, ref)
+        U.assert_parity(got, want, f"staged {what} {rows}x{cols}")
+        check_stats(got, stats, want, ref, 4, False, f"staged {what} {rows}x{cols} ref={ref is not None}")
+        plain, plain_stats = step_with_stats(inp, 2, 4, h, flags | ST | B.CAST_F_PLAIN_ACCESS, meta_in, ref)
+        for k in ("w", "m", "v", "w_fwd", "meta"):
+            assert np.array_equal(got[k], plain[k]), f"{what}: {k} differs between the access paths"
+        assert stats["flips"] == plain_stats["flips"]
+
+
 def test_plan_step_with_statistics_accumulates_over_matrices():
     """All matrices of a plan in one launch: the accumulator holds the model-wide sums, the reference masks are the
     masks of an earlier step (the initial flip rate i_t of App. C), and the step's own results are unchanged by
