@@ -34,7 +34,7 @@ FALLBACK_HBM_GBS = 6650.0         # used only when MEASURED_PEAKS.json is absent
 # taken on); every byte is touched once, so the traffic of a launch is this figure times its parameter count.
 # Set to None when that kernel changes, until the counters are taken again; reported only for the workload and
 # configuration they were taken on (the 2:4 headline over LLaMA2-7B shapes).
-NCU_DRAM_BYTES_PER_PARAM = {"plain": 27.858, "bulk": 27.843}
+NCU_DRAM_BYTES_PER_PARAM = {"plain": 27.856, "bulk": 27.842}
 NCU_KERNEL = {"plain": "adams_nm_multi_kernel<4, 1, 1>", "bulk": "adams_nm_multi_bulk_kernel<4, 1, 1>"}
 
 METRIC = "AdamS 2:4 step params/s"
